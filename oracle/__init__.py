@@ -1,0 +1,168 @@
+"""CPU oracle for the {-1,+1}-decomposed quantized layer -- TEST INFRASTRUCTURE.
+
+This package is not part of the product.  Only the test-suite, the smoke check
+and the benchmark's CPU-baseline leg may import it.  It wraps ``qnn_oracle.c``
+(plain C, compiled here with gcc) behind numpy arrays; it shares no code with the
+CUDA library and never calls it.
+
+What each function follows in the paper:
+
+* ``quantize``     -- code space of Eq. 7 / Section 3.2, interval ownership of Table 2,
+                      clamp of Eq. 15.
+* ``pack_planes``  -- bit-plane storage of Eq. 3 / Eq. 7, one bit per element per plane.
+* ``fc`` / ``conv2d`` (and their ``_sampled`` forms) -- Op(EnC(x), EnC(w)) of Eq. 9:
+                      the plain integer product that Eq. 8 reproduces exactly.
+* ``scale``        -- the fixed scaling factor of Eq. 9 / Alg. 1 forward pass.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "qnn_oracle.c"
+_LIB = _HERE / "libqnn_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile qnn_oracle.c into libqnn_oracle.so next to it (gcc -O2, OpenMP)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        subprocess.check_call([
+            "gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+            "-Wall", "-Wextra", "-o", str(tmp), str(_SRC), "-lm",
+        ])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(str(_LIB))
+        c = ctypes
+        p = c.c_void_p
+        lib.oracle_num_threads.restype = c.c_int
+        lib.oracle_row_words.restype = c.c_size_t
+        lib.oracle_row_words.argtypes = [c.c_size_t]
+        lib.oracle_quantize.argtypes = [p, c.c_size_t, c.c_int, c.c_float, c.c_int, p]
+        lib.oracle_pack_planes.argtypes = [p, c.c_size_t, c.c_size_t, c.c_int, p]
+        lib.oracle_fc.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, p]
+        lib.oracle_fc_sampled.argtypes = [p, p, c.c_size_t, c.c_size_t, p, p, p]
+        lib.oracle_conv_out_dim.argtypes = [c.c_int] * 4
+        lib.oracle_conv2d.argtypes = [p, p] + [c.c_int] * 9 + [p]
+        lib.oracle_conv2d_sampled.argtypes = [p, p] + [c.c_int] * 9 + [c.c_size_t, p, p, p]
+        lib.oracle_scale.argtypes = [p, c.c_size_t, c.c_float, p]
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise ValueError(f"oracle {what} failed with status {rc}")
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def row_words(k: int) -> int:
+    return int(_load().oracle_row_words(k))
+
+
+def quantize(x: np.ndarray, bits: int, scale, relu: bool = False) -> np.ndarray:
+    """Real tensor -> odd integer codes (int16), same shape."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    q = np.empty(x.shape, dtype=np.int16)
+    _check(_load().oracle_quantize(_ptr(x), x.size, bits, float(np.float32(scale)), int(relu), _ptr(q)),
+           "quantize")
+    return q
+
+
+def pack_planes(q: np.ndarray, bits: int) -> np.ndarray:
+    """Codes [rows, k] -> canonical planes uint32 [rows, bits, row_words(k)]."""
+    q = np.ascontiguousarray(q, dtype=np.int16)
+    rows, k = q.shape
+    out = np.empty((rows, bits, row_words(k)), dtype=np.uint32)
+    _check(_load().oracle_pack_planes(_ptr(q), rows, k, bits, _ptr(out)), "pack_planes")
+    return out
+
+
+def fc(qa: np.ndarray, qw: np.ndarray) -> np.ndarray:
+    """qa [Mg, Kg], qw [Ng, Kg] -> int32 [Mg, Ng]."""
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    Mg, Kg = qa.shape
+    Ng, Kg2 = qw.shape
+    assert Kg == Kg2
+    acc = np.empty((Mg, Ng), dtype=np.int32)
+    _check(_load().oracle_fc(_ptr(qa), _ptr(qw), Mg, Ng, Kg, _ptr(acc)), "fc")
+    return acc
+
+
+def fc_sampled(qa: np.ndarray, qw: np.ndarray, rows, cols) -> np.ndarray:
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    assert rows.shape == cols.shape and qa.shape[1] == qw.shape[1]
+    assert rows.size == 0 or (rows.min() >= 0 and rows.max() < qa.shape[0])
+    assert cols.size == 0 or (cols.min() >= 0 and cols.max() < qw.shape[0])
+    acc = np.empty(rows.shape, dtype=np.int32)
+    _check(_load().oracle_fc_sampled(_ptr(qa), _ptr(qw), qa.shape[1], rows.size, _ptr(rows), _ptr(cols),
+                                     _ptr(acc)), "fc_sampled")
+    return acc
+
+
+def conv_out_dim(size: int, k: int, stride: int, pad: int) -> int:
+    return int(_load().oracle_conv_out_dim(size, k, stride, pad))
+
+
+def conv2d(qa: np.ndarray, qw: np.ndarray, stride: int, pad: int) -> np.ndarray:
+    """qa [N,H,W,C], qw [Cout,R,S,C] -> int32 [N,Ho,Wo,Cout]; zero padding of the codes."""
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    N, H, W, C = qa.shape
+    Cout, R, S, C2 = qw.shape
+    assert C == C2
+    Ho, Wo = conv_out_dim(H, R, stride, pad), conv_out_dim(W, S, stride, pad)
+    acc = np.empty((N, Ho, Wo, Cout), dtype=np.int32)
+    _check(_load().oracle_conv2d(_ptr(qa), _ptr(qw), N, H, W, C, Cout, R, S, stride, pad, _ptr(acc)),
+           "conv2d")
+    return acc
+
+
+def conv2d_sampled(qa: np.ndarray, qw: np.ndarray, stride: int, pad: int, rows, cols) -> np.ndarray:
+    """Outputs at (m, co) pairs, m = (n*Ho + ho)*Wo + wo."""
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    N, H, W, C = qa.shape
+    Cout, R, S, C2 = qw.shape
+    assert C == C2 and rows.shape == cols.shape
+    Ho, Wo = conv_out_dim(H, R, stride, pad), conv_out_dim(W, S, stride, pad)
+    assert rows.size == 0 or (rows.min() >= 0 and rows.max() < N * Ho * Wo)
+    assert cols.size == 0 or (cols.min() >= 0 and cols.max() < Cout)
+    acc = np.empty(rows.shape, dtype=np.int32)
+    _check(_load().oracle_conv2d_sampled(_ptr(qa), _ptr(qw), N, H, W, C, Cout, R, S, stride, pad,
+                                         rows.size, _ptr(rows), _ptr(cols), _ptr(acc)), "conv2d_sampled")
+    return acc
+
+
+def scale(acc: np.ndarray, alpha) -> np.ndarray:
+    """float32(acc) * alpha, one rounding each."""
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    out = np.empty(acc.shape, dtype=np.float32)
+    _check(_load().oracle_scale(_ptr(acc), acc.size, float(np.float32(alpha)), _ptr(out)), "scale")
+    return out

@@ -1,0 +1,226 @@
+/*
+ * qnn_oracle.c -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, obviously-correct CPU statement of what one {-1,+1}-decomposed
+ * quantized layer computes.  Only the test-suite, the smoke check and the
+ * benchmark's CPU-baseline leg may call it; the CUDA library never does, and the
+ * two share no source, header, table or helper.
+ *
+ * The paper's multi-branch product (Eq. 8) is an identity, not an approximation:
+ * the weighted sum of all plane-pair xnor/popcount products equals the ordinary
+ * integer dot product of the odd-integer codes.  The oracle is therefore the
+ * plain definition:
+ *
+ *   1. quantize each real tensor to odd codes q in {-(2^b-1), ..., -1, +1, ...,
+ *      2^b-1} (code space of Eq. 7 / Section 3.2; interval ownership of Table 2),
+ *   2. naive integer matrix product / zero-padded convolution of the codes
+ *      (Eq. 1 applied to codes; Op(EnC(x), EnC(w)) of Eq. 9),
+ *   3. one multiplication by the layer scale (Eq. 9, Alg. 1 forward step
+ *      "a_l <- r * a_hat / ((2^M-1)(2^K-1))").
+ *
+ * It also writes the canonical bit-plane storage (Eq. 3 / Eq. 7: plane m holds
+ * c_m of every element, one bit per element, +1 stored as 1) so that packed
+ * planes can be compared word for word.
+ *
+ * Floating point: the quantizer decides an integer, so it is evaluated in
+ * binary32 with one explicit fused multiply-add (the precision the kernels use);
+ * everything after it is integer until the single binary32 multiply of step 3.
+ *
+ * Parallelism: independent output rows are spread over OpenMP threads.  There is
+ * no blocking, vectorisation by hand, fusion or reordering.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_E_ARG (-1)
+#define ORACLE_E_RANGE (-3)
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/*
+ * Quantizer (Table 2 generalised to b bits; code space of Section 3.2).
+ * scale = s = r / (2^b - 1) is the distance from 0 to the first grid point; grid
+ * points are q*s for odd q.  Interval ownership follows Table 2: a value exactly
+ * half-way between two grid points goes to the one farther from zero, and 0
+ * itself belongs to the negative side ("(-2/3, 0]" maps to -1/3).
+ * Values outside [-r, r] take the end codes (the clamp of Eq. 15).
+ * Returns the unsigned code t in [0, 2^b - 1]; the odd code is q = 2t - (2^b-1).
+ */
+static int quantize_t(float x, float inv2s, int bits, int relu) {
+    const float amax = (float)((1 << bits) - 1);
+    const float half = (float)(1 << (bits - 1));
+    if (relu) x = fmaxf(x, 0.0f);
+    float v = fmaf(x, inv2s, half);              /* x/(2s) + 2^(b-1), one rounding */
+    float tf = (x > 0.0f) ? floorf(v) : ceilf(v) - 1.0f;
+    tf = fminf(fmaxf(tf, 0.0f), amax);           /* end codes; NaN -> 0 */
+    return (int)tf;
+}
+
+/* x[n] -> odd codes q[n].  relu != 0 applies max(x,0) first. */
+int oracle_quantize(const float *x, size_t n, int bits, float scale, int relu, int16_t *q) {
+    if (!x || !q || bits < 1 || bits > 8) return ORACLE_E_ARG;
+    if (!(scale > 0.0f) || isinf(scale)) return ORACLE_E_ARG;
+    const float inv2s = 1.0f / (2.0f * scale);
+    const int amax = (1 << bits) - 1;
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t i = 0; i < (ptrdiff_t)n; ++i) {
+        int t = quantize_t(x[i], inv2s, bits, relu);
+        q[i] = (int16_t)(2 * t - amax);
+    }
+    return ORACLE_OK;
+}
+
+/* Number of 32-bit words one plane of one row occupies: ceil(k/32) rounded up to 4. */
+size_t oracle_row_words(size_t k) {
+    size_t w = (k + 31) / 32;
+    return (w + 3) / 4 * 4;
+}
+
+/*
+ * Canonical bit planes of odd codes (Eq. 7: q = sum_m 2^(m-1) c_m, c_m = +-1).
+ * With t = (q + 2^b - 1)/2, c_m = +1 exactly when binary bit (m-1) of t is 1.
+ * Layout: planes[row][plane i = m-1][word], element k in bit (k mod 32) of word
+ * (k div 32); all padding bits are 0.
+ */
+int oracle_pack_planes(const int16_t *q, size_t rows, size_t k, int bits, uint32_t *planes) {
+    if (!q || !planes || bits < 1 || bits > 8) return ORACLE_E_ARG;
+    const size_t kw = oracle_row_words(k);
+    const int amax = (1 << bits) - 1;
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t r = 0; r < (ptrdiff_t)rows; ++r) {
+        for (int i = 0; i < bits; ++i) {
+            uint32_t *dst = planes + ((size_t)r * bits + i) * kw;
+            for (size_t w = 0; w < kw; ++w) dst[w] = 0u;
+            for (size_t e = 0; e < k; ++e) {
+                int t = (q[(size_t)r * k + e] + amax) / 2;
+                if ((t >> i) & 1) dst[e / 32] |= (uint32_t)1 << (e % 32);
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* acc[m][n] = sum_k qa[m][k] * qw[n][k]   (fully-connected layer on codes). */
+int oracle_fc(const int16_t *qa, const int16_t *qw, size_t Mg, size_t Ng, size_t Kg, int32_t *acc) {
+    if (!qa || !qw || !acc) return ORACLE_E_ARG;
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (ptrdiff_t m = 0; m < (ptrdiff_t)Mg; ++m) {
+        for (size_t n = 0; n < Ng; ++n) {
+            int64_t s = 0;
+            for (size_t k = 0; k < Kg; ++k)
+                s += (int64_t)qa[(size_t)m * Kg + k] * (int64_t)qw[n * Kg + k];
+            if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
+            acc[(size_t)m * Ng + n] = (int32_t)s;
+        }
+    }
+    return bad ? ORACLE_E_RANGE : ORACLE_OK;
+}
+
+/* The same dot product for a list of (row, column) pairs only. */
+int oracle_fc_sampled(const int16_t *qa, const int16_t *qw, size_t Kg, size_t count,
+                      const int64_t *rows, const int64_t *cols, int32_t *acc) {
+    if (!qa || !qw || !acc || !rows || !cols) return ORACLE_E_ARG;
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (ptrdiff_t i = 0; i < (ptrdiff_t)count; ++i) {
+        const int16_t *a = qa + (size_t)rows[i] * Kg;
+        const int16_t *w = qw + (size_t)cols[i] * Kg;
+        int64_t s = 0;
+        for (size_t k = 0; k < Kg; ++k) s += (int64_t)a[k] * (int64_t)w[k];
+        if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
+        acc[i] = (int32_t)s;
+    }
+    return bad ? ORACLE_E_RANGE : ORACLE_OK;
+}
+
+/*
+ * One output of the convolution of codes.  Activations are [N][H][W][C], weights
+ * [Cout][R][S][C]; the encoded tensor is padded with true zeros, so a tap that
+ * falls outside the image adds nothing (0 is not a code; Eq. 9 applies the layer
+ * operation to the already-encoded tensor).
+ */
+static int64_t conv_one(const int16_t *qa, const int16_t *qw, int H, int W, int C, int R, int S,
+                        int stride, int pad, int n, int ho, int wo, int co) {
+    int64_t s = 0;
+    for (int r = 0; r < R; ++r) {
+        int hi = ho * stride - pad + r;
+        if (hi < 0 || hi >= H) continue;
+        for (int t = 0; t < S; ++t) {
+            int wi = wo * stride - pad + t;
+            if (wi < 0 || wi >= W) continue;
+            const int16_t *a = qa + (((size_t)n * H + hi) * W + wi) * C;
+            const int16_t *w = qw + (((size_t)co * R + r) * S + t) * C;
+            for (int c = 0; c < C; ++c) s += (int64_t)a[c] * (int64_t)w[c];
+        }
+    }
+    return s;
+}
+
+int oracle_conv_out_dim(int in, int k, int stride, int pad) {
+    return (in + 2 * pad - k) / stride + 1;
+}
+
+/* acc[n][ho][wo][co], Ho = (H + 2 pad - R)/stride + 1, Wo likewise. */
+int oracle_conv2d(const int16_t *qa, const int16_t *qw, int N, int H, int W, int C, int Cout, int R,
+                  int S, int stride, int pad, int32_t *acc) {
+    if (!qa || !qw || !acc || stride < 1 || pad < 0) return ORACLE_E_ARG;
+    const int Ho = oracle_conv_out_dim(H, R, stride, pad);
+    const int Wo = oracle_conv_out_dim(W, S, stride, pad);
+    if (Ho < 1 || Wo < 1) return ORACLE_E_ARG;
+    int bad = 0;
+    const ptrdiff_t rows = (ptrdiff_t)N * Ho * Wo;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (ptrdiff_t m = 0; m < rows; ++m) {
+        int n = (int)(m / ((ptrdiff_t)Ho * Wo));
+        int ho = (int)((m / Wo) % Ho);
+        int wo = (int)(m % Wo);
+        for (int co = 0; co < Cout; ++co) {
+            int64_t s = conv_one(qa, qw, H, W, C, R, S, stride, pad, n, ho, wo, co);
+            if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
+            acc[(size_t)m * Cout + co] = (int32_t)s;
+        }
+    }
+    return bad ? ORACLE_E_RANGE : ORACLE_OK;
+}
+
+/* Convolution outputs for a list of (output row m = (n*Ho+ho)*Wo+wo, channel co) pairs. */
+int oracle_conv2d_sampled(const int16_t *qa, const int16_t *qw, int N, int H, int W, int C, int Cout,
+                          int R, int S, int stride, int pad, size_t count, const int64_t *rows,
+                          const int64_t *cols, int32_t *acc) {
+    if (!qa || !qw || !acc || !rows || !cols || stride < 1 || pad < 0) return ORACLE_E_ARG;
+    (void)N; (void)Cout;
+    const int Ho = oracle_conv_out_dim(H, R, stride, pad);
+    const int Wo = oracle_conv_out_dim(W, S, stride, pad);
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (ptrdiff_t i = 0; i < (ptrdiff_t)count; ++i) {
+        int64_t m = rows[i];
+        int n = (int)(m / ((int64_t)Ho * Wo));
+        int ho = (int)((m / Wo) % Ho);
+        int wo = (int)(m % Wo);
+        int64_t s = conv_one(qa, qw, H, W, C, R, S, stride, pad, n, ho, wo, (int)cols[i]);
+        if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
+        acc[i] = (int32_t)s;
+    }
+    return bad ? ORACLE_E_RANGE : ORACLE_OK;
+}
+
+/* out = float(acc) * alpha: one int->binary32 conversion (round to nearest even), one multiply. */
+int oracle_scale(const int32_t *acc, size_t n, float alpha, float *out) {
+    if (!acc || !out) return ORACLE_E_ARG;
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t i = 0; i < (ptrdiff_t)n; ++i) out[i] = (float)acc[i] * alpha;
+    return ORACLE_OK;
+}

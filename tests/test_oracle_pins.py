@@ -1,0 +1,336 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Nothing here calls the CUDA library.  Every expected value is either printed in
+the paper (Table 2, the 1/9 factor of Fig. 1), a closed form, an independent
+definition (the trigonometric encoder of Eq. 10, a bit-level evaluation of Eq. 8,
+exact rational arithmetic), or a library routine on a special case (numpy matmul,
+torch conv2d on the integer codes in float64).
+"""
+from fractions import Fraction
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+
+
+def codes_to_t(q, bits):
+    return (q.astype(np.int64) + (2 ** bits - 1)) // 2
+
+
+# ----------------------------------------------------------------------------- quantizer
+
+def _parse_frac(s):
+    return Fraction(s)
+
+
+def test_table2_intervals_and_states(golden_dir):
+    """Table 2: interval ownership, quantized numbers and encoded states for 2 bits on [-1, 1]."""
+    rows = []
+    for line in (golden_dir / "table2_2bit.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        lo, lo_c, hi, hi_c, num, den, sh, sl = line.split()
+        rows.append((_parse_frac(lo), int(lo_c), _parse_frac(hi), int(hi_c), Fraction(int(num), int(den)),
+                     int(sh), int(sl)))
+    assert len(rows) == 4
+    # r = 3 makes grid step s = 1 and every interval end exactly representable (x_table = x/3).
+    r = 3.0
+    for lo, lo_c, hi, hi_c, qv, sh, sl in rows:
+        pts = [lo + (hi - lo) * Fraction(i, 16) for i in range(17)]
+        for p in pts:
+            if (p == lo and not lo_c) or (p == hi and not hi_c):
+                continue
+            x = np.array([float(p * 3)], dtype=np.float32)
+            assert Fraction(float(x[0])) == p * 3 or p not in (lo, hi)
+            q = int(oracle.quantize(x, 2, r / 3.0)[0])
+            assert Fraction(q, 3) == qv, (p, q)
+            planes = oracle.pack_planes(np.array([[q]], dtype=np.int16), 2)
+            low = 1 if planes[0, 0, 0] & 1 else -1
+            high = 1 if planes[0, 1, 0] & 1 else -1
+            assert (high, low) == (sh, sl)
+            assert low + 2 * high == q            # x = x_1 + 2 x_2 (Section 3.2)
+
+
+def test_table2_exact_ties_at_r3():
+    x = np.array([-3, -2.5, -2, -1, -0.5, 0, 0.5, 1, 2, 2.5, 3], dtype=np.float32)
+    want = [-3, -3, -3, -1, -1, -1, 1, 1, 3, 3, 3]
+    assert oracle.quantize(x, 2, 1.0).tolist() == want
+    # -0.0 is zero: it belongs to "(-2/3, 0]"
+    assert oracle.quantize(np.array([-0.0], dtype=np.float32), 2, 1.0).tolist() == [-1]
+
+
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_grid_points_are_fixed_points_and_ties_go_outward(bits):
+    A = 2 ** bits - 1
+    s = np.float32(0.25)                       # power of two: q*s and tie points are exact
+    q = np.arange(-A, A + 1, 2, dtype=np.int64)
+    x = (q * float(s)).astype(np.float32)
+    assert oracle.quantize(x, bits, s).tolist() == q.tolist()
+    ties = np.arange(-A + 1, A, 2, dtype=np.int64)             # even integers between codes
+    got = oracle.quantize((ties * float(s)).astype(np.float32), bits, s)
+    want = np.where(ties > 0, ties + 1, ties - 1)               # away from zero; 0 -> -1
+    assert got.tolist() == want.tolist()
+
+
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_quantizer_nearest_monotone_symmetric_clamped(bits):
+    rng = np.random.default_rng(bits)
+    A = 2 ** bits - 1
+    s = np.float32(0.37)
+    r = float(s) * A
+    x = np.sort(rng.uniform(-1.3 * r, 1.3 * r, size=20000).astype(np.float32))
+    q = oracle.quantize(x, bits, s).astype(np.int64)
+    assert np.all(np.abs(q) % 2 == 1) and q.min() >= -A and q.max() <= A
+    assert np.all(np.diff(q) >= 0)                                   # monotone
+    inside = np.abs(x.astype(np.float64)) <= r
+    err = np.abs(x.astype(np.float64) - q * float(s))
+    assert np.all(err[inside] <= float(s) * (1 + 1e-6))              # nearest grid point
+    # strictly nearest grid point wherever the two closest grid points are not (almost) equidistant
+    grid = np.arange(-A, A + 1, 2)
+    d = np.abs(x.astype(np.float64)[:, None] - (grid * float(s))[None, :])
+    nearest = grid[np.argmin(d, axis=1)]
+    if A > 1:
+        ds = np.sort(d, axis=1)
+        clear = (ds[:, 1] - ds[:, 0]) > 1e-4
+    else:
+        clear = np.abs(x) > 1e-4
+    assert np.all(q[clear] == nearest[clear])
+    assert np.all(q[x > r] == A) and np.all(q[x < -r] == -A)          # end codes outside the range
+    qneg = oracle.quantize(-x, bits, s).astype(np.int64)
+    assert np.all(qneg[x != 0] == -q[x != 0])                         # odd symmetry away from 0
+
+
+def test_relu_flag_and_nonfinite():
+    x = np.array([-5.0, -0.1, 0.0, 0.1, 0.9, np.inf, -np.inf, np.nan], dtype=np.float32)
+    assert oracle.quantize(x, 2, 1.0 / 3, relu=True).tolist() == [-1, -1, -1, 1, 3, 3, -1, -1]
+    assert oracle.quantize(x, 2, 1.0 / 3, relu=False).tolist() == [-3, -1, -1, 1, 3, 3, -3, -3]
+
+
+# ----------------------------------------------------------------------------- planes
+
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_planes_match_trigonometric_encoder(bits):
+    """Eq. 10: the m-th encoder output is sign(+-sin((2^M-1)/2^m * pi * x)) for x in [-1, 1]."""
+    M = bits
+    A = 2 ** M - 1
+    rng = np.random.default_rng(100 + bits)
+    x = rng.uniform(-1, 1, size=6000)
+    # keep away from interval boundaries (even multiples of 1/A) where sign(sin) is 0
+    dist = np.abs(x * A / 2 - np.round(x * A / 2))
+    x = x[dist > 1e-3]
+    xf = x.astype(np.float32)
+    q = oracle.quantize(xf, M, np.float32(1.0) / np.float32(A))
+    planes = oracle.pack_planes(q.reshape(1, -1), M)
+    for m in range(1, M + 1):
+        arg = (2 ** M - 1) / 2 ** m * math.pi * xf.astype(np.float64)
+        phi = np.sign(np.sin(arg)) if m == M else np.sign(-np.sin(arg))
+        words = planes[0, m - 1]
+        bits_m = (words[np.arange(x.size) // 32] >> (np.arange(x.size) % 32).astype(np.uint32)) & 1
+        assert np.array_equal(np.where(bits_m == 1, 1.0, -1.0), phi), (M, m)
+
+
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_eq7_reconstruction_from_planes(bits):
+    rng = np.random.default_rng(7 + bits)
+    A = 2 ** bits - 1
+    q = (2 * rng.integers(0, A + 1, size=(5, 77)) - A).astype(np.int16)
+    planes = oracle.pack_planes(q, bits)
+    k = np.arange(77)
+    rec = np.zeros((5, 77), dtype=np.int64)
+    for i in range(bits):
+        c = ((planes[:, i, :][:, k // 32] >> (k % 32).astype(np.uint32)) & 1).astype(np.int64) * 2 - 1
+        rec += (2 ** i) * c
+    assert np.array_equal(rec, q)
+
+
+def test_plane_layout_word_and_bit_position():
+    """Element k sits in bit k%32 of word k//32; pad bits are zero; rows padded to 4 words."""
+    k = 70
+    q = -np.ones((2, k), dtype=np.int16) * 3        # t = 0 everywhere (2 bits)
+    q[1, 37] = 3                                    # t = 3: both planes set
+    q[0, 69] = 1                                    # t = 2: only plane 1
+    planes = oracle.pack_planes(q, 2)
+    assert planes.shape == (2, 2, 4) and oracle.row_words(k) == 4
+    want = np.zeros((2, 2, 4), dtype=np.uint32)
+    want[1, 0, 1] = 1 << 5
+    want[1, 1, 1] = 1 << 5
+    want[0, 1, 2] = 1 << 5
+    assert np.array_equal(planes, want)
+    ones = oracle.pack_planes(np.ones((1, k), dtype=np.int16) * 3, 2)
+    assert ones[0, 0].tolist() == [0xFFFFFFFF, 0xFFFFFFFF, 0x3F, 0]
+    assert oracle.row_words(128) == 4 and oracle.row_words(129) == 8 and oracle.row_words(1) == 4
+
+
+@pytest.mark.parametrize("bits,ratio", [(1, 32), (2, 16), (3, 10.7), (4, 8), (5, 6.4), (6, 5.3), (7, 4.6), (8, 4)])
+def test_packed_size_matches_compression_column(bits, ratio):
+    """Table 3's compression column: 32/bits relative to fp32 storage."""
+    rows, k = 16, 1024
+    planes = oracle.pack_planes(np.ones((rows, k), dtype=np.int16), bits)
+    assert abs(rows * k * 4 / planes.nbytes - ratio) < 0.05
+
+
+# ----------------------------------------------------------------------------- contraction
+
+def branch_sum_bruteforce(pa, pw, N, ab, wb):
+    """Eq. 8 evaluated literally on bit planes: sum_ij 2^(i+j) * (N - 2*popcount(a_i xor w_j))."""
+    Mg, Ng = pa.shape[0], pw.shape[0]
+    out = np.zeros((Mg, Ng), dtype=np.int64)
+    for m in range(Mg):
+        for n in range(Ng):
+            s = 0
+            for i in range(ab):
+                for j in range(wb):
+                    x = np.bitwise_xor(pa[m, i], pw[n, j])
+                    pc = sum(bin(int(v)).count("1") for v in x)
+                    s += (1 << (i + j)) * (N - 2 * pc)
+            out[m, n] = s
+    return out
+
+
+@pytest.mark.parametrize("ab,wb,Kg", [(1, 1, 40), (2, 2, 65), (3, 2, 33), (4, 4, 130), (2, 4, 7), (8, 8, 50), (5, 1, 96)])
+def test_eq8_branch_identity(ab, wb, Kg):
+    rng = np.random.default_rng(ab * 100 + wb * 10 + Kg)
+    A, B = 2 ** ab - 1, 2 ** wb - 1
+    qa = (2 * rng.integers(0, A + 1, size=(5, Kg)) - A).astype(np.int16)
+    qw = (2 * rng.integers(0, B + 1, size=(6, Kg)) - B).astype(np.int16)
+    acc = oracle.fc(qa, qw)
+    assert np.array_equal(acc, branch_sum_bruteforce(oracle.pack_planes(qa, ab), oracle.pack_planes(qw, wb), Kg, ab, wb))
+    # Eq. 6 / Eq. 18 form on the {0,1}-coded integers t
+    ta, tw = codes_to_t(qa, ab), codes_to_t(qw, wb)
+    alt = 4 * ta @ tw.T - 2 * B * ta.sum(1)[:, None] - 2 * A * tw.sum(1)[None, :] + Kg * A * B
+    assert np.array_equal(acc, alt)
+
+
+def test_fc_matches_numpy_matmul_ragged():
+    rng = np.random.default_rng(5)
+    qa = (2 * rng.integers(0, 16, size=(37, 301)) - 15).astype(np.int16)
+    qw = (2 * rng.integers(0, 8, size=(29, 301)) - 7).astype(np.int16)
+    want = qa.astype(np.float64) @ qw.astype(np.float64).T
+    got = oracle.fc(qa, qw)
+    assert np.array_equal(got.astype(np.float64), want)
+    rows = rng.integers(0, 37, size=50)
+    cols = rng.integers(0, 29, size=50)
+    assert np.array_equal(oracle.fc_sampled(qa, qw, rows, cols), got[rows, cols])
+
+
+def test_closed_forms():
+    N = 123
+    for ab, wb in [(1, 1), (2, 3), (4, 4), (8, 8)]:
+        A, B = 2 ** ab - 1, 2 ** wb - 1
+        assert oracle.fc(np.full((2, N), A, np.int16), np.full((3, N), B, np.int16)).tolist() == [[N * A * B] * 3] * 2
+        assert oracle.fc(np.full((2, N), -A, np.int16), np.full((3, N), B, np.int16)).tolist() == [[-N * A * B] * 3] * 2
+    rng = np.random.default_rng(1)
+    q = (2 * rng.integers(0, 8, size=(1, N)) - 7).astype(np.int16)
+    assert oracle.fc(q, -q)[0, 0] == -int((q.astype(np.int64) ** 2).sum())
+
+
+def test_one_bit_is_sign_xnor_popcount():
+    """1-bit x 1-bit reduces to the binarized-network product: sign vectors, 2*popc(xnor) - N."""
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((4, 100)).astype(np.float32)
+    w = rng.standard_normal((3, 100)).astype(np.float32)
+    x[x == 0] = 1
+    qa, qw = oracle.quantize(x, 1, 1.0), oracle.quantize(w, 1, 1.0)
+    assert np.array_equal(qa, np.sign(x).astype(np.int16))
+    sa, sw = x > 0, w > 0
+    want = np.array([[2 * int(np.sum(~(sa[m] ^ sw[n]))) - 100 for n in range(3)] for m in range(4)])
+    assert np.array_equal(oracle.fc(qa, qw), want)
+
+
+def test_overflow_is_reported():
+    Kg = 40000                                    # 40000 * 255 * 255 > 2^31
+    qa = np.full((1, Kg), 255, np.int16)
+    with pytest.raises(ValueError):
+        oracle.fc(qa, qa)
+
+
+# ----------------------------------------------------------------------------- scale
+
+def test_fig1_two_bit_fc_scale_one_ninth():
+    """2-bit FC on [-1,1] data: real product of the quantized numbers = integer product / 9 (Fig. 1, Eq. 19)."""
+    vals = [Fraction(-1), Fraction(-1, 3), Fraction(1, 3), Fraction(1)]
+    rng = np.random.default_rng(11)
+    xi = rng.integers(0, 4, size=(3, 24))
+    wi = rng.integers(0, 4, size=(5, 24))
+    # feed points strictly inside each Table-2 interval
+    centers = np.array([-0.9, -0.3, 0.3, 0.9], dtype=np.float32)
+    s = np.float32(1.0) / np.float32(3.0)
+    qa, qw = oracle.quantize(centers[xi], 2, s), oracle.quantize(centers[wi], 2, s)
+    acc = oracle.fc(qa, qw)
+    for m in range(3):
+        for n in range(5):
+            exact = sum(vals[xi[m, k]] * vals[wi[n, k]] for k in range(24))
+            assert Fraction(int(acc[m, n]), 9) == exact
+    out = oracle.scale(acc, np.float32(1.0) / np.float32(9.0))
+    assert np.allclose(out, acc / 9.0, rtol=2e-7)
+
+
+def test_scale_against_float_bruteforce_of_decoded_values():
+    rng = np.random.default_rng(17)
+    a = np.maximum(rng.standard_normal((6, 90)), 0).astype(np.float32)
+    w = (0.05 * rng.standard_normal((7, 90))).astype(np.float32)
+    for ab, wb in [(2, 2), (3, 4), (1, 8)]:
+        sa = np.float32(np.abs(a).max()) / np.float32(2 ** ab - 1)
+        sw = np.float32(np.abs(w).max()) / np.float32(2 ** wb - 1)
+        qa, qw = oracle.quantize(a, ab, sa), oracle.quantize(w, wb, sw)
+        alpha = np.float32(sa * sw)
+        out = oracle.scale(oracle.fc(qa, qw), alpha)
+        brute = (qa.astype(np.float64) * float(sa)) @ (qw.astype(np.float64) * float(sw)).T
+        assert np.allclose(out, brute, rtol=1e-6, atol=1e-9)
+        # the quantized layer approximates the real one (coarse sanity of grid + scale)
+        assert np.abs(out - a.astype(np.float64) @ w.astype(np.float64).T).max() <= 90 * float(sa) * float(sw) * (2 ** ab) * (2 ** wb)
+
+
+def test_scale_is_single_rounding():
+    acc = np.array([0, 1, -1, 16777217, -2147483648, 2147483647, 123456789], dtype=np.int32)
+    alpha = np.float32(0.013671875)
+    want = (acc.astype(np.float32) * alpha).astype(np.float32)
+    assert np.array_equal(oracle.scale(acc, alpha), want)
+
+
+# ----------------------------------------------------------------------------- convolution
+
+def im2col_zero(qa, R, S, stride, pad):
+    N, H, W, C = qa.shape
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    padded = np.zeros((N, H + 2 * pad, W + 2 * pad, C), dtype=qa.dtype)
+    padded[:, pad:pad + H, pad:pad + W] = qa
+    cols = np.empty((N, Ho, Wo, R, S, C), dtype=qa.dtype)
+    for r in range(R):
+        for s in range(S):
+            cols[:, :, :, r, s, :] = padded[:, r:r + stride * Ho:stride, s:s + stride * Wo:stride, :]
+    return cols.reshape(N * Ho * Wo, R * S * C), Ho, Wo
+
+
+@pytest.mark.parametrize("N,H,W,C,Cout,R,S,stride,pad", [
+    (2, 5, 6, 7, 4, 3, 3, 1, 1), (1, 7, 7, 3, 5, 3, 3, 2, 1), (2, 6, 6, 9, 3, 1, 1, 2, 0),
+    (1, 4, 5, 33, 2, 3, 3, 1, 0), (1, 9, 8, 4, 3, 5, 3, 2, 2), (2, 3, 3, 8, 8, 3, 3, 1, 1)])
+def test_conv_equals_fc_on_explicit_im2col_and_torch(N, H, W, C, Cout, R, S, stride, pad):
+    import torch
+    rng = np.random.default_rng(N * 1000 + H * 100 + C)
+    qa = (2 * rng.integers(0, 8, size=(N, H, W, C)) - 7).astype(np.int16)
+    qw = (2 * rng.integers(0, 4, size=(Cout, R, S, C)) - 3).astype(np.int16)
+    acc = oracle.conv2d(qa, qw, stride, pad)
+    cols, Ho, Wo = im2col_zero(qa, R, S, stride, pad)
+    assert acc.shape == (N, Ho, Wo, Cout)
+    assert np.array_equal(acc.reshape(-1, Cout), oracle.fc(cols, qw.reshape(Cout, -1)))
+    ref = torch.nn.functional.conv2d(torch.from_numpy(qa.astype(np.float64)).permute(0, 3, 1, 2),
+                                     torch.from_numpy(qw.astype(np.float64)).permute(0, 3, 1, 2),
+                                     stride=stride, padding=pad).permute(0, 2, 3, 1).numpy()
+    assert np.array_equal(acc.astype(np.float64), ref)
+    rows = rng.integers(0, N * Ho * Wo, size=40)
+    cc = rng.integers(0, Cout, size=40)
+    assert np.array_equal(oracle.conv2d_sampled(qa, qw, stride, pad, rows, cc), acc.reshape(-1, Cout)[rows, cc])
+
+
+def test_conv_1x1_is_gemm_and_border_counts_valid_taps():
+    rng = np.random.default_rng(2)
+    qa = (2 * rng.integers(0, 4, size=(2, 4, 4, 16)) - 3).astype(np.int16)
+    qw = (2 * rng.integers(0, 4, size=(6, 1, 1, 16)) - 3).astype(np.int16)
+    assert np.array_equal(oracle.conv2d(qa, qw, 1, 0).reshape(-1, 6), oracle.fc(qa.reshape(-1, 16), qw.reshape(6, 16)))
+    # all codes +1 (1 bit): each output counts C * (#taps inside the image); corners see 4 of 9 taps
+    ones = np.ones((1, 5, 5, 8), np.int16)
+    acc = oracle.conv2d(ones, np.ones((1, 3, 3, 8), np.int16), 1, 1)[0, :, :, 0]
+    assert acc[0, 0] == 8 * 4 and acc[0, 2] == 8 * 6 and acc[2, 2] == 8 * 9 and acc[4, 4] == 8 * 4
