@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the {-1,+1} bit-plane decomposed quantized layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--report FILE]
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+qnn_encode_pack (fp32 activations -> bit planes) followed by qnn_bgemm (all plane pairs,
+combine, scale) against weights packed offline.  Workload: square GEMM Mg = Ng = Kg = 4096,
+2-bit weights x 2-bit activations, A = min(|N(0,1)|, 4), W ~ N(0, 0.02), per-tensor scales.
+
+Prints ONE JSON line (rank 0).  `value` is binary TOPS of the whole step with inputs resident
+in HBM; `e2e` is the same metric through qnn_fc_forward_host with pinned host buffers
+(host<->device copies inside the timed region); `roofline` is for the dominant kernel
+(the contraction), timed with CUDA events inside the timed region, against the
+bit-operation peak measured by the library's register-resident probe in the same run;
+`cpu_baseline` is the CPU oracle timed on the host cores.
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same workload on its own
+batch of rows (rows are independent, weights replicated, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+N_SQ = 4096
+AB, WB = 2, 2
+NBUF = 4           # rotating input/output sets: 4 x (64 MiB in + 64 MiB out) >> 126 MB of L2
+METRIC = "binary TOPS, qnn_encode_pack + qnn_bgemm (equiv. int GOPS and % of roofline alongside)"
+UNIT = "binary TOPS"
+
+
+def binary_ops(Mg, Ng, Kg, ab, wb):
+    return 2.0 * Mg * Ng * Kg * ab * wb
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        inside = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.1] or [r for (_, r) in self.rows]
+        for r in inside:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ----------------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on the host cores
+# ----------------------------------------------------------------------------------------------------------
+
+def oracle_step_sample(rows_per_step: int, seed: int = 0):
+    """Returns (fn, macs) where fn() runs quantize+FC of `rows_per_step` activation rows against all 4096 columns."""
+    import oracle
+    from paper_2106_09886_b200 import workloads as wl
+    c = wl.gemm_config3(seed, N_SQ, WB, AB)
+    sa, sw = wl.per_tensor_scale(c.a, AB), wl.per_tensor_scale(c.w, WB)
+    alpha = np.float32(sa * sw)
+    qw = oracle.quantize(c.w, WB, sw)          # offline, like the packed weights of the GPU arm
+    a = c.a
+
+    def fn(step: int):
+        r0 = (step * rows_per_step) % (N_SQ - rows_per_step + 1)
+        qa = oracle.quantize(a[r0:r0 + rows_per_step], AB, sa)
+        acc = oracle.fc(qa, qw)
+        return oracle.scale(acc, alpha)
+
+    return fn, oracle.num_threads()
+
+
+def run_reference(args):
+    rank, world, _ = dist_setup(args.gpus)
+    if rank != 0:
+        return
+    rows = 256
+    fn, cores = oracle_step_sample(rows)
+    for s in range(args.warmup):
+        fn(s)
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        fn(s)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = binary_ops(rows, N_SQ, N_SQ, AB, WB) / dt / 1e12
+    sample = f"{rows} of {N_SQ} activation rows per step (quantize + naive int FC against all {N_SQ} columns + scale)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": f"qnn_bgemm {N_SQ}x{N_SQ}x{N_SQ} w{WB}a{AB} (square GEMM sweep, 2x2 bits)", "sample": sample},
+        "equiv_int_gops": 2.0 * rows * N_SQ * N_SQ / dt / 1e9,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------------------------------------
+
+def measure_peaks(torch, qnn, dev):
+    """In-run peaks: bit-operation probes (both instruction mixes) and a plain device copy."""
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    sink = torch.empty(sms * 8 * 256, dtype=torch.int32, device=dev)
+    res = {}
+    for variant, name in ((0, "xor_popc_add"), (1, "csa_3to2")):
+        best = 0.0
+        for _ in range(4):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ops = qnn.probe_bitops(variant, 4000, sms * 8, sink)
+            e1.record()
+            e1.synchronize()
+            best = max(best, ops / (e0.elapsed_time(e1) * 1e-3))
+        res[name] = best * 64.0 / 1e12            # word-ops/s -> binary TOPS (32 MACs x 2 ops per word)
+    nbytes = 1 << 30
+    src = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    dst = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    src.zero_()
+    best = 0.0
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        qnn.probe_copy(dst, src)
+        e1.record()
+        e1.synchronize()
+        best = max(best, 2.0 * nbytes / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    res["copy_gbs"] = best
+    del src, dst
+    return res
+
+
+def load_measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return json.loads(p.read_text()), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
+
+
+def cpu_baseline_leg():
+    rows = 1024
+    fn, cores = oracle_step_sample(rows)
+    fn(0)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        fn(reps)
+        reps += 1
+        if time.perf_counter() - t0 > 10.0 or reps >= 8:
+            break
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": binary_ops(rows, N_SQ, N_SQ, AB, WB) / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{rows} of {N_SQ} activation rows (quantize + naive int FC against all {N_SQ} columns + scale), "
+                      f"{reps} repetitions, {dt:.2f} s each",
+            "equiv_int_gops": 2.0 * rows * N_SQ * N_SQ / dt / 1e9}
+
+
+def run_gpu(args):
+    import torch
+    from paper_2106_09886_b200 import qnn
+    from paper_2106_09886_b200 import workloads as wl
+
+    rank, world, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- workload: per-rank batch of rows (seeded per rank), replicated weights, packed offline
+    c = wl.gemm_config3(0, N_SQ, WB, AB, variant=rank)
+    sa, sw = wl.per_tensor_scale(c.a, AB), wl.per_tensor_scale(c.w, WB)
+    alpha = float(np.float32(sa * sw))
+    Mg = Ng = Kg = N_SQ
+    w_d = torch.from_numpy(c.w).to(dev)
+    packed = qnn.pack_weights(w_d, Ng, 1, Kg, qnn.W_NTC, WB, sw)
+    del w_d
+    a_host = torch.from_numpy(c.a).pin_memory()
+    a_bufs = [a_host.to(dev) for _ in range(NBUF)]
+    out_bufs = [torch.empty((Mg, Ng), dtype=torch.float32, device=dev) for _ in range(NBUF)]
+    planes = [torch.empty((Mg, AB, qnn.row_words(Kg)), dtype=torch.int32, device=dev) for _ in range(NBUF)]
+    out_host = torch.empty((Mg, Ng), dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+
+    def step(i):
+        b = i % NBUF
+        qnn.encode_pack(a_bufs[b], AB, sa, 0, planes=planes[b])
+        qnn.bgemm(planes[b], AB, packed, WB, Mg, Ng, Kg, alpha, out=out_bufs[b])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = measure_peaks(torch, qnn, dev) if rank == 0 else None
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    t_wall0 = time.time()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(args.steps):
+        b = i % NBUF
+        ev[i][0].record()
+        qnn.encode_pack(a_bufs[b], AB, sa, 0, planes=planes[b])
+        ev[i][1].record()
+        qnn.bgemm(planes[b], AB, packed, WB, Mg, Ng, Kg, alpha, out=out_bufs[b])
+        ev[i][2].record()
+    stop.record()
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    ms_total = start.elapsed_time(stop)
+    enc_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+
+    # ---- end to end through the host-buffer entry point
+    def e2e_step(i):
+        b = i % NBUF
+        qnn.fc_forward_host(a_host, AB, sa, 0, packed, WB, Ng, alpha, out_host, a_bufs[b], planes[b], out_bufs[b])
+
+    e2e_steps = max(3, min(args.steps, 10))
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    s2, t2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    t2.record()
+    barrier()
+    e2e_ms_total = s2.elapsed_time(t2)
+    checksum = float(out_host[0, 0])
+
+    times = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
+    if use_dist:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_total = (float(v) for v in times.cpu())
+
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        ops_step = binary_ops(Mg, Ng, Kg, AB, WB) * world
+        value = ops_step / (ms_step * 1e-3) / 1e12
+        e2e_ms = e2e_ms_total / e2e_steps
+        mp, mp_kind = load_measured_peaks()
+        kernel_peak = max(peaks["xor_popc_add"], peaks["csa_3to2"]) if qnn.version() >= 110 else peaks["xor_popc_add"]
+        achieved = binary_ops(Mg, Ng, Kg, AB, WB) / (gemm_ms * 1e-3) / 1e12
+        alg_bytes_gemm = Mg * Kg * AB / 8 + Ng * Kg * WB / 8 + Mg * Ng * 4
+        enc_bytes = Mg * Kg * 4 + Mg * Kg * AB / 8
+        traffic = None
+        tfile = ROOT / "profiles" / "traffic.json"
+        if tfile.exists():
+            try:
+                traffic = json.loads(tfile.read_text()).get("bgemm_4096_w2a2_dram_bytes_per_launch")
+            except Exception:
+                traffic = None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32", "data": "synthetic",
+            "config": {"workload": f"qnn_bgemm {N_SQ}x{N_SQ}x{N_SQ} w{WB}a{AB} per GPU (square GEMM sweep, 2x2 bits), "
+                                   "step = qnn_encode_pack + qnn_bgemm, weights packed offline",
+                       "l2": f"{NBUF} rotating input/output sets of 128 MiB each (larger than L2)",
+                       "parallelism": f"replicas x{world}, rows sharded, no collective"},
+            "equiv_int_gops": 2.0 * Mg * Ng * Kg * world / (ms_step * 1e-3) / 1e9,
+            "kernel_ms": {"qnn_encode_pack": enc_ms, "qnn_bgemm": gemm_ms},
+            "gpu_launches": 2 * args.steps,
+            "e2e": {"value": ops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": Mg * Kg * 4, "d2h_bytes_per_step": Mg * Ng * 4, "steps": e2e_steps,
+                    "api": "qnn_fc_forward_host (pinned host buffers)", "checksum": checksum},
+            "roofline": {"kernel": "qnn_bgemm", "bound": "alu", "achieved": achieved, "peak": kernel_peak,
+                         "unit": UNIT, "frac": achieved / kernel_peak, "traffic": traffic,
+                         "peak_source": "register-resident bit-op probe of the library, same run (of measured)",
+                         "probe_xor_popc_add": peaks["xor_popc_add"], "probe_csa_3to2": peaks["csa_3to2"],
+                         "algorithmic_bytes": alg_bytes_gemm,
+                         "hbm_time_ms": alg_bytes_gemm / (mp["hbm_gbs"] * 1e9) * 1e3,
+                         "hbm_peak_gbs": mp["hbm_gbs"], "hbm_peak_kind": mp_kind, "copy_probe_gbs": peaks["copy_gbs"]},
+            "roofline_encode": {"kernel": "qnn_encode_pack", "bound": "hbm", "achieved": enc_bytes / (enc_ms * 1e-3) / 1e9,
+                                "peak": mp["hbm_gbs"], "unit": "GB/s",
+                                "frac": enc_bytes / (enc_ms * 1e-3) / 1e9 / mp["hbm_gbs"], "peak_kind": mp_kind},
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline_leg()
+        print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["graft", "reference"], default="graft")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,174 @@
+/*
+ * qnn.h -- C ABI of libqnn: one quantized layer computed through the {-1,+1}
+ * bit-plane decomposition (arXiv 2106.09886), for NVIDIA B200 (sm_100a).
+ *
+ * Pipeline of one layer (Alg. 1, forward pass; Fig. 1):
+ *
+ *   real activations --qnn_encode_pack--> activation bit planes  \
+ *                                                                  qnn_bgemm / qnn_bconv2d --> fp32 outputs
+ *   real weights ------qnn_pack_weights-> weight bit planes      /   (all plane pairs, 2^(i+j) combine, scale)
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The caller
+ *     owns every buffer; the library allocates nothing, never frees, and never
+ *     modifies an input.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     only enqueue work; they return before it has run.
+ *   - Every call returns a qnn_status.  Argument errors are found on the host
+ *     before anything is enqueued; no exception or abort crosses this boundary.
+ *   - Bit widths are 1..8.  "ab"/"wb" = activation / weight bits.
+ *     A = 2^ab - 1 and B = 2^wb - 1 are the largest odd codes.
+ *   - Mg, Ng, Kg = rows of activations, output features, reduction length.
+ *
+ * Encoding (Eq. 7, Section 3.2, Table 2).  A real x with grid step `scale`
+ * (= r/(2^b - 1) for data in [-r, r]) becomes the odd integer q in
+ * {-(2^b-1), ..., -1, +1, ..., 2^b-1} nearest to x/scale; a value half-way
+ * between two codes goes to the one farther from zero, 0 goes to -1, values
+ * outside [-r, r] take the end codes, NaN takes the most negative code.
+ * q = sum_{i<b} 2^i c_i with c_i in {-1,+1}; with t = (q + 2^b - 1)/2, c_i = +1
+ * exactly when bit i of t is 1.  Plane i stores c_i of every element, 1 bit each
+ * (bit 1 means +1).
+ *
+ * Plane storage.  uint32 planes[row][plane i][word]; element k of a row is bit
+ * (k mod 32) of word (k div 32); a row of k elements occupies
+ * qnn_row_words(k) = ceil(k/32) rounded up to a multiple of 4 words per plane;
+ * all padding bits are 0.  Plane buffers must be 16-byte aligned.
+ */
+#ifndef QNN_H
+#define QNN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum qnn_status {
+    QNN_OK = 0,
+    QNN_E_ARG = -1,    /* null pointer, non-positive size, bits outside 1..8, unknown flag/layout */
+    QNN_E_ALIGN = -2,  /* a plane/packed buffer is not 16-byte aligned, fp32 buffer not 4-byte aligned */
+    QNN_E_RANGE = -3,  /* Kg*A*B does not fit int32, or an index does not fit the kernels' 32-bit tile arithmetic */
+    QNN_E_SCALE = -4,  /* scale or alpha not finite, or scale <= 0 */
+    QNN_E_CUDA = -5,   /* the CUDA runtime refused a launch or copy (cudaGetLastError is consumed) */
+    QNN_E_DEVICE = -6  /* a kernel reported an internal error through its status word */
+} qnn_status;
+
+/* flags of qnn_encode_pack */
+#define QNN_RELU 1u /* apply max(x, 0) before quantizing (the ReLU between layers of a stack) */
+
+/* source layouts of qnn_pack_weights; element (n, tap, c) of the logical weight tensor is read from */
+#define QNN_W_NTC 0 /* w[(n*taps + tap)*c_in + c]   : FC [Ng][Kg] (taps = 1) or conv [Cout][R][S][Cin] */
+#define QNN_W_TCN 1 /* w[(tap*c_in + c)*n_out + n]  : FC stored k-major [Kg][Ng], conv [R][S][Cin][Cout] */
+#define QNN_W_NCT 2 /* w[(n*c_in + c)*taps + tap]   : conv [Cout][Cin][R][S] */
+
+const char *qnn_status_string(int status);
+int qnn_version(void);
+
+/* Words per (row, plane) for a row of k elements: ceil(k/32) rounded up to 4. */
+size_t qnn_row_words(int64_t k);
+/* Bytes of a plane buffer: rows * bits * qnn_row_words(k) * 4. */
+size_t qnn_planes_bytes(int64_t rows, int64_t k, int bits);
+/* Bytes of the packed-weights blob written by qnn_pack_weights (layout below). */
+size_t qnn_weights_bytes(int n_out, int taps, int c_in, int bits);
+/* Words per (output feature, plane) inside the packed-weights blob: taps*ceil(c_in/32) rounded up to 4. */
+size_t qnn_weights_row_words(int taps, int c_in);
+
+/*
+ * Quantize, encode and bit-plane-pack activations in one pass (Eq. 7; Table 2;
+ * the encoder stage of Fig. 1; Alg. 1 forward "MBitEncoder" step, evaluated
+ * as the look-up form of Section 3.3).
+ *   x       fp32 [rows][ldx], row r starts at x + r*ldx, first k entries used (ldx >= k).
+ *           For a convolution input in NHWC, rows = N*H*W and k = C.
+ *   scale   grid step s = r/(2^bits - 1), finite and > 0.
+ *   flags   0 or QNN_RELU.
+ *   planes  out, uint32 [rows][bits][qnn_row_words(k)], fully written (padding = 0).
+ *   rowsum  optional out (may be NULL), int32 [rows]: sum over the row of t = (q + 2^bits - 1)/2.
+ */
+int qnn_encode_pack(const float *x, int64_t rows, int k, int64_t ldx, int bits, float scale, unsigned flags,
+                    uint32_t *planes, int32_t *rowsum, void *stream);
+
+/*
+ * Offline weight decomposition: quantize real weights to odd codes and store
+ * their bit planes (Section 4.2: the quantized network's weights are
+ * transformed into bit-encoded binary weights used at inference; Eq. 21).
+ *   w        fp32, n_out*taps*c_in elements in one of the QNN_W_* layouts.
+ *            FC: taps = 1, c_in = Kg.  Convolution: taps = R*S, c_in = Cin.
+ *   packed   out, qnn_weights_bytes(...) bytes, 16-byte aligned:
+ *              uint32 planes[n_out][bits][qnn_weights_row_words(taps, c_in)]
+ *                 word tap*ceil(c_in/32) + c/32, bit c%32 holds element (tap, c);
+ *                 each tap starts on a word boundary, padding bits are 0;
+ *              followed by int32 tapsum[n_out][taps] = sum_c t(n, tap, c), which the
+ *                 convolution needs for taps that fall outside the image.
+ */
+int qnn_pack_weights(const float *w, int n_out, int taps, int c_in, int layout, int bits, float scale,
+                     void *packed, void *stream);
+
+/*
+ * Fully-connected layer on packed planes (Eq. 8 and Eq. 9; Alg. 1 forward,
+ * the weighted branch sum and the scale): for every output (m, n)
+ *   X_ij   = popcount over the row of (a_i[m] xor w_j[n])      for all ab*wb plane pairs,
+ *   acc    = Kg*A*B - 2 * sum_ij 2^(i+j) X_ij                   (= sum_k q_a[m][k]*q_w[n][k], exact int32),
+ *   out    = float(acc) * alpha                                 (alpha = scale_a * scale_w).
+ * All pairs, the combine and the scale happen in one launch.
+ *   a_planes  uint32 [Mg][ab][qnn_row_words(Kg)]
+ *   w_packed  blob of qnn_pack_weights(n_out = Ng, taps = 1, c_in = Kg, bits = wb)
+ *   out       fp32 [Mg][ldo] (ldo >= Ng), may be NULL if acc is given
+ *   acc       optional int32 [Mg][Ng] (dense), the exact accumulators
+ * QNN_E_RANGE if Kg*A*B >= 2^31.
+ */
+int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg,
+              float alpha, float *out, int64_t ldo, int32_t *acc, void *stream);
+
+/*
+ * Convolution lowered by implicit im2col onto the same plane-pair contraction
+ * (Section 3.2: the decomposition applies to convolution layers as to
+ * fully-connected ones; Eq. 9 applies the layer operation to the encoded
+ * tensors).  The encoded activation tensor is padded with true zeros: a tap
+ * outside the image adds nothing, so for each output pixel only the taps inside
+ * the image are counted.
+ *   a_planes  uint32 [N*H*W][ab][qnn_row_words(C)]   (NHWC pixels as rows)
+ *   w_packed  blob of qnn_pack_weights(n_out = Cout, taps = R*S, c_in = C, bits = wb)
+ *   out       fp32 [N][Ho][Wo][Cout], Ho = (H + 2*pad - R)/stride + 1, Wo likewise; may be NULL if acc given
+ *   acc       optional int32, same shape as out
+ */
+int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
+                int Cout, int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc,
+                void *stream);
+
+/*
+ * max_i |x[i]| into *out (device fp32), for workloads whose grid step is derived
+ * from the tensor's range.  Not a step of the paper's method (its range r is a
+ * fixed or learned constant, Eq. 9 / Eq. 15).  NaNs are ignored.
+ */
+int qnn_absmax_f32(const float *x, size_t n, float *out, void *stream);
+
+/*
+ * One FC layer from host memory: copies x_host to x_dev, runs qnn_encode_pack
+ * and qnn_bgemm, copies the fp32 result to out_host, all on `stream`.
+ * Device work buffers are the caller's: x_dev [Mg*Kg] fp32, planes_dev
+ * qnn_planes_bytes(Mg, Kg, ab), out_dev [Mg*Ng] fp32.  x_host / out_host should be
+ * pinned for the copies to be asynchronous.  The result is in out_host once the
+ * stream has been synchronized.
+ */
+int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float scale_a, unsigned flags,
+                        const void *w_packed, int wb, int Ng, float alpha, float *out_host, float *x_dev,
+                        uint32_t *planes_dev, float *out_dev, void *stream);
+
+/*
+ * Peak probes used to state a roofline next to a measurement.
+ * qnn_probe_bitops enqueues a register-resident kernel that does nothing but the
+ * contraction's instruction mix and returns (in *word_ops) how many 32-bit
+ * xor-popcount-accumulate word operations it performs; divide by its measured time.
+ *   variant 0: xor + popc + add per word;  variant 1: the 3:2 carry-save form
+ *   (3 xor, 2 three-input logic ops, 2 popc per 3 words).
+ *   sink: device int32 [blocks*256], written once at the end.
+ * qnn_probe_copy enqueues a plain 16-byte-vector device copy of `bytes` (multiple of 16).
+ */
+int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream);
+int qnn_probe_copy(void *dst, const void *src, size_t bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QNN_H */

@@ -1,0 +1,148 @@
+// qnn_bgemm / qnn_bconv2d: all plane-pair xor+popcount contractions of one layer,
+// the 2^(i+j) combine and the scale, in one launch.
+#include "qnn_internal.cuh"
+
+namespace {
+
+struct ConvGeom {
+    int N, H, W, C, Cout, R, S, stride, pad, Ho, Wo;
+    int cw;        // words per tap: ceil(C/32)
+    int a_pitch;   // words per (pixel, plane) in the activation planes: qnn_row_words(C)
+    int w_pitch;   // words per (feature, plane) in the packed weights
+};
+
+__device__ __forceinline__ void store_out(float *out, int64_t ldo, int32_t *acc, int64_t m, int n, int Ng, int32_t v,
+                                          float alpha) {
+    if (acc) acc[m * Ng + n] = v;
+    if (out) out[m * ldo + n] = __fmul_rn(__int2float_rn(v), alpha);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Generic path (any ab, wb in 1..8): one thread per output.  Used for bit widths that have no
+// tiled specialisation; correct for every shape, not tuned.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+bgemm_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__restrict__ w, int wb, int64_t Mg, int Ng,
+                     int Kg, int kw, float alpha, float *__restrict__ out, int64_t ldo, int32_t *__restrict__ acc) {
+    const int n = blockIdx.x * 16 + (threadIdx.x & 15);
+    const int64_t m = (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
+    if (n >= Ng || m >= Mg) return;
+    const uint4 *arow = reinterpret_cast<const uint4 *>(a + m * ab * (int64_t)kw);
+    const uint4 *wrow = reinterpret_cast<const uint4 *>(w + (int64_t)n * wb * kw);
+    const int kq = kw / 4;
+    int32_t s = 0;
+    for (int i = 0; i < ab; ++i) {
+        for (int j = 0; j < wb; ++j) {
+            int32_t x = 0;
+            for (int q = 0; q < kq; ++q) {
+                uint4 av = arow[i * kq + q], wv = wrow[j * kq + q];
+                x += __popc(av.x ^ wv.x) + __popc(av.y ^ wv.y) + __popc(av.z ^ wv.z) + __popc(av.w ^ wv.w);
+            }
+            s += x << (i + j);
+        }
+    }
+    const int32_t AB = ((1 << ab) - 1) * ((1 << wb) - 1);
+    store_out(out, ldo, acc, m, n, Ng, Kg * AB - 2 * s, alpha);
+}
+
+__global__ void __launch_bounds__(256)
+bconv_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__restrict__ w, int wb, ConvGeom g,
+                     float alpha, float *__restrict__ out, int32_t *__restrict__ acc) {
+    const int co = blockIdx.x * 16 + (threadIdx.x & 15);
+    const int64_t m = (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
+    const int64_t Mg = (int64_t)g.N * g.Ho * g.Wo;
+    if (co >= g.Cout || m >= Mg) return;
+    const int wo = (int)(m % g.Wo);
+    const int ho = (int)((m / g.Wo) % g.Ho);
+    const int n = (int)(m / ((int64_t)g.Wo * g.Ho));
+    int32_t s = 0;
+    int valid = 0;
+    for (int r = 0; r < g.R; ++r) {
+        const int hi = ho * g.stride - g.pad + r;
+        if (hi < 0 || hi >= g.H) continue;
+        for (int t = 0; t < g.S; ++t) {
+            const int wi = wo * g.stride - g.pad + t;
+            if (wi < 0 || wi >= g.W) continue;
+            ++valid;
+            const uint32_t *ap = a + (((int64_t)n * g.H + hi) * g.W + wi) * ab * g.a_pitch;
+            const uint32_t *wp = w + (int64_t)co * wb * g.w_pitch + (r * g.S + t) * g.cw;
+            for (int i = 0; i < ab; ++i)
+                for (int j = 0; j < wb; ++j) {
+                    int32_t x = 0;
+                    for (int c = 0; c < g.cw; ++c) x += __popc(ap[i * g.a_pitch + c] ^ wp[j * g.w_pitch + c]);
+                    s += x << (i + j);
+                }
+        }
+    }
+    const int32_t AB = ((1 << ab) - 1) * ((1 << wb) - 1);
+    store_out(out, g.Cout, acc, m, co, g.Cout, valid * g.C * AB - 2 * s, alpha);
+}
+
+}  // namespace
+
+extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg,
+                         float alpha, float *out, int64_t ldo, int32_t *acc, void *stream) {
+    if (!a_planes || !w_packed || (!out && !acc) || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
+    if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb) || (out && ldo < Ng)) return QNN_E_ARG;
+    if (!isfinite(alpha)) return QNN_E_SCALE;
+    if (!qnn_aligned(a_planes, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(out, 4) || !qnn_aligned(acc, 4))
+        return QNN_E_ALIGN;
+    const int64_t AB = (int64_t)((1 << ab) - 1) * ((1 << wb) - 1);
+    if ((int64_t)Kg * AB >= ((int64_t)1 << 31)) return QNN_E_RANGE;
+    if (Mg > ((int64_t)1 << 31) - 1 || qnn_ceil_div(Mg, 16) > 65535 * (int64_t)16) return QNN_E_RANGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int kw = (int)qnn_row_words_i(Kg);
+    const uint32_t *w = static_cast<const uint32_t *>(w_packed);
+    dim3 grid((unsigned)qnn_ceil_div(Ng, 16), (unsigned)qnn_ceil_div(Mg, 16));
+    if (grid.y > 65535) return QNN_E_RANGE;
+    bgemm_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, Mg, Ng, Kg, kw, alpha, out, ldo, acc);
+    return qnn_launch_status();
+}
+
+extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
+                           int Cout, int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc,
+                           void *stream) {
+    if (!a_planes || !w_packed || (!out && !acc)) return QNN_E_ARG;
+    if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || Cout <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0) return QNN_E_ARG;
+    if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb)) return QNN_E_ARG;
+    if (!isfinite(alpha)) return QNN_E_SCALE;
+    if (!qnn_aligned(a_planes, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(out, 4) || !qnn_aligned(acc, 4))
+        return QNN_E_ALIGN;
+    ConvGeom g;
+    g.N = N; g.H = H; g.W = W; g.C = C; g.Cout = Cout; g.R = R; g.S = S; g.stride = stride; g.pad = pad;
+    g.Ho = (H + 2 * pad - R) / stride + 1;
+    g.Wo = (W + 2 * pad - S) / stride + 1;
+    if (H + 2 * pad < R || W + 2 * pad < S || g.Ho <= 0 || g.Wo <= 0) return QNN_E_ARG;
+    g.cw = (C + 31) / 32;
+    g.a_pitch = (int)qnn_row_words_i(C);
+    g.w_pitch = (int)qnn_w_row_words_i(R * S, C);
+    const int64_t AB = (int64_t)((1 << ab) - 1) * ((1 << wb) - 1);
+    if ((int64_t)R * S * C * AB >= ((int64_t)1 << 31)) return QNN_E_RANGE;
+    const int64_t Mg = (int64_t)N * g.Ho * g.Wo;
+    if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t *w = static_cast<const uint32_t *>(w_packed);
+    dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
+    if (grid.y > 65535) {
+        // fold rows into x for very tall problems
+        return QNN_E_RANGE;
+    }
+    bconv_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, g, alpha, out, acc);
+    return qnn_launch_status();
+}
+
+extern "C" int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float scale_a, unsigned flags,
+                                   const void *w_packed, int wb, int Ng, float alpha, float *out_host, float *x_dev,
+                                   uint32_t *planes_dev, float *out_dev, void *stream) {
+    if (!x_host || !out_host || !x_dev || !planes_dev || !out_dev || Mg <= 0 || Kg <= 0 || Ng <= 0) return QNN_E_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)Mg * Kg * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return QNN_E_CUDA;
+    int rc = qnn_encode_pack(x_dev, Mg, Kg, Kg, ab, scale_a, flags, planes_dev, nullptr, stream);
+    if (rc != QNN_OK) return rc;
+    rc = qnn_bgemm(planes_dev, ab, w_packed, wb, Mg, Ng, Kg, alpha, out_dev, Ng, nullptr, stream);
+    if (rc != QNN_OK) return rc;
+    if (cudaMemcpyAsync(out_host, out_dev, (size_t)Mg * Ng * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return QNN_E_CUDA;
+    return QNN_OK;
+}

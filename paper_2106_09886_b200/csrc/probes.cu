@@ -1,0 +1,108 @@
+// Peak probes: a register-resident kernel with the contraction's instruction mix, and a plain copy.
+#include "qnn_internal.cuh"
+
+namespace {
+
+// R x C register tile of xor + popc + add, operands perturbed once per iteration.
+template <int R, int C>
+__global__ void __launch_bounds__(256) probe_popc_kernel(int iters, int32_t *sink) {
+    uint32_t a[R], w[C];
+    int acc[R][C];
+#pragma unroll
+    for (int r = 0; r < R; ++r) a[r] = (threadIdx.x + 1u) * 2654435761u + r * 40503u + blockIdx.x;
+#pragma unroll
+    for (int c = 0; c < C; ++c) w[c] = (threadIdx.x + 7u) * 2246822519u + c * 2654435769u;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < C; ++c) acc[r][c] = 0;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int c = 0; c < C; ++c) acc[r][c] += __popc(a[r] ^ w[c]);
+#pragma unroll
+        for (int r = 0; r < R; ++r) a[r] += 0x9e3779b9u;
+#pragma unroll
+        for (int c = 0; c < C; ++c) w[c] += 0x7f4a7c15u;
+    }
+    int s = 0;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < C; ++c) s += acc[r][c];
+    sink[blockIdx.x * 256 + threadIdx.x] = s;
+}
+
+// Carry-save form: three xor words are compressed to a sum word and a carry word (two 3-input
+// logic ops), so 3 words cost 2 popcounts.
+template <int R, int C>
+__global__ void __launch_bounds__(256) probe_csa_kernel(int iters, int32_t *sink) {
+    uint32_t a[3][R], w[3][C];
+    int acc[R][C];
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) a[k][r] = (threadIdx.x + 1u) * 2654435761u + (k * R + r) * 40503u + blockIdx.x;
+#pragma unroll
+        for (int c = 0; c < C; ++c) w[k][c] = (threadIdx.x + 7u) * 2246822519u + (k * C + c) * 2654435769u;
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < C; ++c) acc[r][c] = 0;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                uint32_t x0 = a[0][r] ^ w[0][c], x1 = a[1][r] ^ w[1][c], x2 = a[2][r] ^ w[2][c];
+                uint32_t s = x0 ^ x1 ^ x2;
+                uint32_t cy = (x0 & x1) | (x2 & (x0 ^ x1));
+                acc[r][c] += __popc(s) + 2 * __popc(cy);
+            }
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) a[k][r] += 0x9e3779b9u;
+#pragma unroll
+            for (int c = 0; c < C; ++c) w[k][c] += 0x7f4a7c15u;
+        }
+    }
+    int s = 0;
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int c = 0; c < C; ++c) s += acc[r][c];
+    sink[blockIdx.x * 256 + threadIdx.x] = s;
+}
+
+__global__ void __launch_bounds__(256) probe_copy_kernel(uint4 *__restrict__ dst, const uint4 *__restrict__ src, size_t n) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = src[i];
+}
+
+}  // namespace
+
+extern "C" int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream) {
+    if (!sink || iters <= 0 || blocks <= 0 || (variant != 0 && variant != 1)) return QNN_E_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double per_thread_iter;
+    if (variant == 0) {
+        probe_popc_kernel<8, 4><<<blocks, 256, 0, st>>>(iters, sink);
+        per_thread_iter = 32.0;
+    } else {
+        probe_csa_kernel<4, 4><<<blocks, 256, 0, st>>>(iters, sink);
+        per_thread_iter = 48.0;
+    }
+    if (word_ops) *word_ops = per_thread_iter * iters * 256.0 * blocks;
+    return qnn_launch_status();
+}
+
+extern "C" int qnn_probe_copy(void *dst, const void *src, size_t bytes, void *stream) {
+    if (!dst || !src || bytes == 0 || bytes % 16) return QNN_E_ARG;
+    if (!qnn_aligned(dst, 16) || !qnn_aligned(src, 16)) return QNN_E_ALIGN;
+    probe_copy_kernel<<<148 * 16, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint4 *>(dst),
+                                                                           static_cast<const uint4 *>(src), bytes / 16);
+    return qnn_launch_status();
+}

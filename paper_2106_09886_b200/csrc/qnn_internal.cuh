@@ -1,0 +1,29 @@
+// Internal helpers shared by the CUDA translation units of libqnn.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <math.h>
+#include "qnn.h"
+
+#define QNN_VERSION_NUMBER 100
+
+static inline bool qnn_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+static inline bool qnn_bits_ok(int b) { return b >= 1 && b <= 8; }
+static inline int64_t qnn_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline int64_t qnn_row_words_i(int64_t k) { return qnn_ceil_div(qnn_ceil_div(k, 32), 4) * 4; }
+static inline int64_t qnn_w_row_words_i(int taps, int c_in) {
+    return qnn_ceil_div((int64_t)taps * qnn_ceil_div(c_in, 32), 4) * 4;
+}
+static inline int qnn_launch_status() { return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA; }
+
+// Unsigned code t in [0, 2^bits - 1] of a real value (odd code q = 2t - (2^bits - 1)).
+// inv2s = 1/(2*scale), half = 2^(bits-1), amax = 2^bits - 1.
+// One fused multiply-add, then floor for positive x and ceil-1 otherwise, so that
+// a value half-way between two codes moves away from zero and 0 maps to q = -1.
+__device__ __forceinline__ int qnn_code_t(float x, float inv2s, float half, float amax, bool relu) {
+    if (relu) x = fmaxf(x, 0.0f);
+    float v = __fmaf_rn(x, inv2s, half);
+    float tf = (x > 0.0f) ? floorf(v) : ceilf(v) - 1.0f;
+    tf = fminf(fmaxf(tf, 0.0f), amax);
+    return __float2int_rz(tf);
+}

@@ -1,0 +1,203 @@
+"""ctypes binding of libqnn.so: same names as the C ABI (include/qnn.h), torch tensors in and out.
+
+Argument marshalling only -- every step runs inside the library's CUDA kernels.  The
+library must have been built (``python -m paper_2106_09886_b200.build``); importing this
+module without it raises ImportError, and there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libqnn.so"
+
+OK, E_ARG, E_ALIGN, E_RANGE, E_SCALE, E_CUDA, E_DEVICE = 0, -1, -2, -3, -4, -5, -6
+RELU = 1
+W_NTC, W_TCN, W_NCT = 0, 1, 2
+
+EXPORTS = [
+    "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
+    "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
+    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_probe_bitops", "qnn_probe_copy",
+]
+
+
+class QnnError(RuntimeError):
+    def __init__(self, status: int, call: str):
+        self.status = status
+        super().__init__(f"{call} failed: {status_string(status)} ({status})")
+
+
+def _load() -> C.CDLL:
+    if not _LIB_PATH.exists():
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2106_09886_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(str(_LIB_PATH))
+    p, i, i64, f, u, sz = C.c_void_p, C.c_int, C.c_int64, C.c_float, C.c_uint, C.c_size_t
+    lib.qnn_status_string.restype = C.c_char_p
+    lib.qnn_status_string.argtypes = [i]
+    lib.qnn_version.restype = i
+    lib.qnn_row_words.restype = sz
+    lib.qnn_row_words.argtypes = [i64]
+    lib.qnn_planes_bytes.restype = sz
+    lib.qnn_planes_bytes.argtypes = [i64, i64, i]
+    lib.qnn_weights_bytes.restype = sz
+    lib.qnn_weights_bytes.argtypes = [i, i, i, i]
+    lib.qnn_weights_row_words.restype = sz
+    lib.qnn_weights_row_words.argtypes = [i, i]
+    lib.qnn_encode_pack.argtypes = [p, i64, i, i64, i, f, u, p, p, p]
+    lib.qnn_pack_weights.argtypes = [p, i, i, i, i, i, f, p, p]
+    lib.qnn_bgemm.argtypes = [p, i, p, i, i64, i, i, f, p, i64, p, p]
+    lib.qnn_bconv2d.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, p]
+    lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
+    lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
+    lib.qnn_probe_bitops.argtypes = [i, i, i, p, C.POINTER(C.c_double), p]
+    lib.qnn_probe_copy.argtypes = [p, p, sz, p]
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.qnn_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib.qnn_version())
+
+
+def row_words(k: int) -> int:
+    return int(lib.qnn_row_words(k))
+
+
+def planes_bytes(rows: int, k: int, bits: int) -> int:
+    return int(lib.qnn_planes_bytes(rows, k, bits))
+
+
+def weights_bytes(n_out: int, taps: int, c_in: int, bits: int) -> int:
+    return int(lib.qnn_weights_bytes(n_out, taps, c_in, bits))
+
+
+def weights_row_words(taps: int, c_in: int) -> int:
+    return int(lib.qnn_weights_row_words(taps, c_in))
+
+
+def _stream(stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _check(rc: int, call: str):
+    if rc != OK:
+        raise QnnError(rc, call)
+
+
+def _dev(t: torch.Tensor, dtype, name: str):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous {dtype}")
+    return t
+
+
+def encode_pack(x: torch.Tensor, bits: int, scale: float, flags: int = 0, planes: torch.Tensor | None = None,
+                rowsum: torch.Tensor | None = None, k: int | None = None, stream=None) -> torch.Tensor:
+    """x fp32 [rows, ldx] (first k columns used) -> planes int32-typed storage [rows, bits, row_words(k)]."""
+    _dev(x, torch.float32, "x")
+    rows, ldx = x.shape[0] if x.dim() == 2 else x.numel() // x.shape[-1], x.shape[-1]
+    k = ldx if k is None else k
+    if planes is None:
+        planes = torch.empty((rows, bits, row_words(k)), dtype=torch.int32, device=x.device)
+    _check(lib.qnn_encode_pack(_ptr(x), rows, k, ldx, bits, float(scale), flags, _ptr(planes), _ptr(rowsum),
+                               _stream(stream)), "qnn_encode_pack")
+    return planes
+
+
+def pack_weights(w: torch.Tensor, n_out: int, taps: int, c_in: int, layout: int, bits: int, scale: float,
+                 packed: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Real weights (any of the W_* layouts, n_out*taps*c_in elements) -> packed blob (uint8 tensor)."""
+    _dev(w, torch.float32, "w")
+    if w.numel() != n_out * taps * c_in:
+        raise ValueError("w has the wrong number of elements")
+    if packed is None:
+        packed = torch.empty(weights_bytes(n_out, taps, c_in, bits), dtype=torch.uint8, device=w.device)
+    _check(lib.qnn_pack_weights(_ptr(w), n_out, taps, c_in, layout, bits, float(scale), _ptr(packed),
+                                _stream(stream)), "qnn_pack_weights")
+    return packed
+
+
+def bgemm(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, Mg: int, Ng: int, Kg: int,
+          alpha: float, out: torch.Tensor | None = None, acc: torch.Tensor | None = None, want_acc: bool = False,
+          stream=None):
+    if out is None:
+        out = torch.empty((Mg, Ng), dtype=torch.float32, device=a_planes.device)
+    if acc is None and want_acc:
+        acc = torch.empty((Mg, Ng), dtype=torch.int32, device=a_planes.device)
+    _check(lib.qnn_bgemm(_ptr(a_planes), ab, _ptr(w_packed), wb, Mg, Ng, Kg, float(alpha), _ptr(out),
+                         out.stride(0), _ptr(acc), _stream(stream)), "qnn_bgemm")
+    return (out, acc) if (want_acc or acc is not None) else out
+
+
+def conv_out_dim(size: int, k: int, stride: int, pad: int) -> int:
+    return (size + 2 * pad - k) // stride + 1
+
+
+def bconv2d(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N: int, H: int, W: int, Cin: int,
+            Cout: int, R: int, S: int, stride: int, pad: int, alpha: float, out: torch.Tensor | None = None,
+            acc: torch.Tensor | None = None, want_acc: bool = False, stream=None):
+    Ho, Wo = conv_out_dim(H, R, stride, pad), conv_out_dim(W, S, stride, pad)
+    if out is None:
+        out = torch.empty((N, Ho, Wo, Cout), dtype=torch.float32, device=a_planes.device)
+    if acc is None and want_acc:
+        acc = torch.empty((N, Ho, Wo, Cout), dtype=torch.int32, device=a_planes.device)
+    _check(lib.qnn_bconv2d(_ptr(a_planes), ab, _ptr(w_packed), wb, N, H, W, Cin, Cout, R, S, stride, pad,
+                           float(alpha), _ptr(out), _ptr(acc), _stream(stream)), "qnn_bconv2d")
+    return (out, acc) if (want_acc or acc is not None) else out
+
+
+def absmax_f32(x: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    _dev(x, torch.float32, "x")
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=x.device)
+    _check(lib.qnn_absmax_f32(_ptr(x), x.numel(), _ptr(out), _stream(stream)), "qnn_absmax_f32")
+    return out
+
+
+def fc_forward_host(x_host: torch.Tensor, ab: int, scale_a: float, flags: int, w_packed: torch.Tensor, wb: int,
+                    Ng: int, alpha: float, out_host: torch.Tensor, x_dev: torch.Tensor, planes_dev: torch.Tensor,
+                    out_dev: torch.Tensor, stream=None) -> torch.Tensor:
+    Mg, Kg = x_host.shape
+    _check(lib.qnn_fc_forward_host(_ptr(x_host), Mg, Kg, ab, float(scale_a), flags, _ptr(w_packed), wb, Ng,
+                                   float(alpha), _ptr(out_host), _ptr(x_dev), _ptr(planes_dev), _ptr(out_dev),
+                                   _stream(stream)), "qnn_fc_forward_host")
+    return out_host
+
+
+def probe_bitops(variant: int, iters: int, blocks: int, sink: torch.Tensor, stream=None) -> float:
+    """Enqueue the register-resident bit-op probe; returns the number of 32-bit word operations it performs."""
+    ops = C.c_double(0.0)
+    _check(lib.qnn_probe_bitops(variant, iters, blocks, _ptr(sink), C.byref(ops), _stream(stream)),
+           "qnn_probe_bitops")
+    return ops.value
+
+
+def probe_copy(dst: torch.Tensor, src: torch.Tensor, stream=None) -> int:
+    nbytes = src.numel() * src.element_size()
+    _check(lib.qnn_probe_copy(_ptr(dst), _ptr(src), nbytes, _stream(stream)), "qnn_probe_copy")
+    return nbytes
+
+
+def weights_views(packed: torch.Tensor, n_out: int, taps: int, c_in: int, bits: int):
+    """Split a packed-weights blob into (planes int32 [n_out, bits, row_words], tapsum int32 [n_out, taps])."""
+    kw = weights_row_words(taps, c_in)
+    nplane = n_out * bits * kw
+    as_i32 = packed.view(torch.int32)
+    return as_i32[:nplane].view(n_out, bits, kw), as_i32[nplane:nplane + n_out * taps].view(n_out, taps)

@@ -1,0 +1,108 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every declared symbol, and its host-side
+argument validation and size queries behave as the header says.  No kernel is launched here."""
+import ctypes
+import re
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import oracle
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def qnn():
+    from paper_2106_09886_b200 import build
+    build.build()
+    from paper_2106_09886_b200 import qnn as q
+    return q
+
+
+def declared_functions():
+    text = (ROOT / "include" / "qnn.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(qnn_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(qnn):
+    names = declared_functions()
+    assert "qnn_bgemm" in names and "qnn_bconv2d" in names and "qnn_encode_pack" in names and "qnn_pack_weights" in names
+    for name in names:
+        assert hasattr(qnn.lib, name), name
+    assert sorted(qnn.EXPORTS) == names
+
+
+def test_size_queries_match_layout(qnn):
+    for k in [1, 31, 32, 33, 127, 128, 129, 512, 4096, 4097]:
+        assert qnn.row_words(k) == oracle.row_words(k)
+        assert qnn.planes_bytes(7, k, 3) == 7 * 3 * oracle.row_words(k) * 4
+    assert qnn.row_words(0) == 0 and qnn.planes_bytes(0, 5, 2) == 0 and qnn.planes_bytes(5, 5, 9) == 0
+    # conv weights: every tap starts on a word boundary
+    assert qnn.weights_row_words(9, 256) == 72 and qnn.weights_row_words(9, 3) == 12 and qnn.weights_row_words(1, 64) == 4
+    assert qnn.weights_bytes(256, 9, 256, 2) == 256 * 2 * 72 * 4 + 256 * 9 * 4
+    assert qnn.weights_bytes(5, 1, 40, 3) == 5 * 3 * 4 * 4 + 32       # tapsum rounded up to 16 bytes
+    # Table 3's compression column: 32/bits
+    for bits in range(1, 9):
+        assert qnn.planes_bytes(64, 4096, bits) * bits == 64 * 4096 * 4 * bits * bits // 32
+
+
+def test_status_strings_and_version(qnn):
+    assert qnn.version() >= 100
+    seen = {qnn.status_string(s) for s in range(0, -7, -1)}
+    assert len(seen) == 7 and qnn.status_string(0) == "ok" and qnn.status_string(-99) == "unknown status"
+
+
+def test_argument_errors_are_reported_before_any_launch(qnn):
+    lib = qnn.lib
+    buf = (ctypes.c_char * 4096)()
+    base = ctypes.addressof(buf)
+    p = ctypes.c_void_p((base + 15) // 16 * 16)                    # aligned, never dereferenced by these calls
+    mis = ctypes.c_void_p(p.value + 4)
+    assert lib.qnn_encode_pack(None, 4, 64, 64, 2, 1.0, 0, p, None, None) == qnn.E_ARG
+    assert lib.qnn_encode_pack(p, 4, 64, 32, 2, 1.0, 0, p, None, None) == qnn.E_ARG       # ldx < k
+    assert lib.qnn_encode_pack(p, 4, 64, 64, 9, 1.0, 0, p, None, None) == qnn.E_ARG
+    assert lib.qnn_encode_pack(p, 4, 64, 64, 2, 1.0, 2, p, None, None) == qnn.E_ARG       # unknown flag
+    assert lib.qnn_encode_pack(p, 4, 64, 64, 2, 0.0, 0, p, None, None) == qnn.E_SCALE
+    assert lib.qnn_encode_pack(p, 4, 64, 64, 2, float("nan"), 0, p, None, None) == qnn.E_SCALE
+    assert lib.qnn_encode_pack(p, 4, 64, 64, 2, 1.0, 0, mis, None, None) == qnn.E_ALIGN
+    assert lib.qnn_pack_weights(p, 4, 1, 64, 7, 2, 1.0, p, None) == qnn.E_ARG            # unknown layout
+    assert lib.qnn_pack_weights(p, 4, 1, 64, 0, 2, -1.0, p, None) == qnn.E_SCALE
+    assert lib.qnn_pack_weights(p, 4, 1, 64, 0, 2, 1.0, mis, None) == qnn.E_ALIGN
+    assert lib.qnn_bgemm(p, 2, p, 2, 4, 4, 64, 1.0, None, 4, None, None) == qnn.E_ARG    # no output at all
+    assert lib.qnn_bgemm(p, 0, p, 2, 4, 4, 64, 1.0, p, 4, None, None) == qnn.E_ARG
+    assert lib.qnn_bgemm(p, 2, p, 2, 4, 4, 64, 1.0, p, 3, None, None) == qnn.E_ARG       # ldo < Ng
+    assert lib.qnn_bgemm(p, 2, p, 2, 4, 4, 64, float("inf"), p, 4, None, None) == qnn.E_SCALE
+    assert lib.qnn_bgemm(mis, 2, p, 2, 4, 4, 64, 1.0, p, 4, None, None) == qnn.E_ALIGN
+    assert lib.qnn_bgemm(p, 8, p, 8, 4, 4, 33026, 1.0, p, 4, None, None) == qnn.E_RANGE  # 33026*255*255 >= 2^31
+    assert lib.qnn_bconv2d(p, 2, p, 2, 1, 4, 4, 8, 8, 3, 3, 0, 1, 1.0, p, None, None) == qnn.E_ARG   # stride 0
+    assert lib.qnn_bconv2d(p, 2, p, 2, 1, 2, 2, 8, 8, 5, 5, 1, 0, 1.0, p, None, None) == qnn.E_ARG   # kernel > image
+    assert lib.qnn_bconv2d(p, 8, p, 8, 1, 8, 8, 4096, 8, 3, 3, 1, 1, 1.0, p, None, None) == qnn.E_RANGE
+    assert lib.qnn_absmax_f32(None, 4, p, None) == qnn.E_ARG
+    assert lib.qnn_probe_copy(p, p, 24, None) == qnn.E_ARG
+
+
+def test_importing_binding_without_library_fails_loudly(tmp_path, monkeypatch):
+    import importlib.util
+    src = (ROOT / "paper_2106_09886_b200" / "qnn.py").read_text()
+    mod_path = tmp_path / "qnn_copy.py"
+    mod_path.write_text(src)
+    spec = importlib.util.spec_from_file_location("qnn_copy", mod_path)
+    with pytest.raises(ImportError):
+        spec.loader.exec_module(importlib.util.module_from_spec(spec))
+
+
+def test_workloads_are_seeded_and_shaped():
+    from paper_2106_09886_b200 import workloads as wl
+    c1, c1b = wl.fc_config1(0), wl.fc_config1(0)
+    assert np.array_equal(c1.a, c1b.a) and c1.a.shape == (64, 512) and c1.w.shape == (512, 256) and c1.k_major
+    assert c1.a.min() >= 0 and c1.a.max() <= 3.0 and (c1.Mg, c1.Ng, c1.Kg) == (64, 256, 512)
+    c2 = wl.conv_config2(0, batch=2)
+    assert c2.a.shape == (2, 14, 14, 256) and c2.w.shape == (256, 3, 3, 256) and c2.a.min() >= 0
+    assert wl.conv_config2(0).shape.Mg == 6272 and wl.conv_config2(0).shape.Kg == 2304
+    r = wl.resnet18_shapes()
+    assert len(r) == 19 and sum(s.int_macs for s in r) // 10 ** 9 == 434
+    v = wl.vgg16_shapes()
+    assert len(v) == 13 and sum(s.int_macs for s in v) // 10 ** 9 == 982
+    assert v[0].Kg == 27 and v[0].Mg == 3211264

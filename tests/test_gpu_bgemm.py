@@ -1,0 +1,120 @@
+"""GPU parity: qnn_bgemm against the CPU oracle -- int32 accumulators bit-exact, fp32 outputs within 1e-6 relative."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import assert_fp32_close, gpu_fc, oracle_fc, oracle_fc_codes, scales_for
+from paper_2106_09886_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def run_case(a, w, k_major, ab, wb, relu=False):
+    sa, sw, alpha = scales_for(a, w, ab, wb)
+    qa, qw, acc, out = oracle_fc(a, w, k_major, ab, wb, sa, sw, alpha, relu)
+    got = gpu_fc(a, w, k_major, ab, wb, sa, sw, alpha, relu, want_planes=True)
+    assert np.array_equal(got["a_planes"], oracle.pack_planes(qa, ab))
+    assert np.array_equal(got["w_planes"], oracle.pack_planes(qw, wb))
+    assert np.array_equal(got["acc"], acc)
+    assert_fp32_close(got["out"], out)
+    return got
+
+
+BITS = [(a, w) for a in range(1, 5) for w in range(1, 5)] + [(8, 8), (5, 3), (1, 7), (6, 2)]
+
+
+@pytest.mark.parametrize("ab,wb", BITS)
+def test_bgemm_bit_widths(ab, wb):
+    rng = np.random.default_rng(ab * 10 + wb)
+    a = np.maximum(rng.standard_normal((150, 700)), 0).astype(np.float32)
+    w = (0.02 * rng.standard_normal((83, 700))).astype(np.float32)
+    run_case(a, w, False, ab, wb)
+
+
+@pytest.mark.parametrize("Mg,Ng,Kg", [(1, 1, 1), (1, 5, 31), (63, 17, 32), (64, 64, 128), (65, 100, 129),
+                                      (130, 33, 1000), (257, 129, 520), (5, 300, 4097), (200, 8, 96)])
+def test_bgemm_ragged_shapes(Mg, Ng, Kg):
+    rng = np.random.default_rng(Mg * 7 + Ng * 3 + Kg)
+    a = rng.standard_normal((Mg, Kg)).astype(np.float32)
+    w = rng.standard_normal((Ng, Kg)).astype(np.float32)
+    for ab, wb in [(2, 2), (3, 2)]:
+        run_case(a, w, False, ab, wb)
+
+
+def test_bgemm_closed_forms_and_extremes():
+    Kg = 777
+    for ab, wb in [(1, 1), (2, 2), (4, 4), (8, 8)]:
+        A, B = 2 ** ab - 1, 2 ** wb - 1
+        a = np.full((70, Kg), 1e6, np.float32)         # far outside the range: end codes
+        w = np.full((66, Kg), 1e6, np.float32)
+        got = gpu_fc(a, w, False, ab, wb, np.float32(1), np.float32(1), np.float32(1))
+        assert np.all(got["acc"] == Kg * A * B)
+        got = gpu_fc(-a, w, False, ab, wb, np.float32(1), np.float32(1), np.float32(1))
+        assert np.all(got["acc"] == -Kg * A * B)
+    # largest reduction that still fits int32 at 8x8 bits
+    Kg = 33025
+    a = np.full((3, Kg), 1e9, np.float32)
+    got = gpu_fc(a, a[:2], False, 8, 8, np.float32(1), np.float32(1), np.float32(1))
+    assert np.all(got["acc"] == Kg * 255 * 255)
+
+
+def test_bgemm_k_major_weights_relu_and_strided_output():
+    import torch
+    from paper_2106_09886_b200 import qnn
+    rng = np.random.default_rng(12)
+    a = rng.standard_normal((90, 300)).astype(np.float32)
+    w = (0.05 * rng.standard_normal((300, 70))).astype(np.float32)       # [Kg][Ng]
+    run_case(a, w, True, 2, 3, relu=True)
+    # out only / acc only / padded leading dimension
+    sa, sw, alpha = scales_for(a, w, 2, 2)
+    _, _, acc, out = oracle_fc(a, w, True, 2, 2, sa, sw, alpha)
+    dev = torch.device("cuda:0")
+    planes = qnn.encode_pack(torch.from_numpy(a).to(dev), 2, sa)
+    packed = qnn.pack_weights(torch.from_numpy(w).to(dev), 70, 1, 300, qnn.W_TCN, 2, sw)
+    wide = torch.full((90, 96), 123.0, dtype=torch.float32, device=dev)
+    qnn.bgemm(planes, 2, packed, 2, 90, 70, 300, alpha, out=wide[:, :70])
+    assert_fp32_close(wide[:, :70].cpu().numpy(), out)
+    assert torch.all(wide[:, 70:] == 123.0)
+    acc_d = torch.empty((90, 70), dtype=torch.int32, device=dev)
+    assert qnn.lib.qnn_bgemm(planes.data_ptr(), 2, packed.data_ptr(), 2, 90, 70, 300, float(alpha), None, 70,
+                             acc_d.data_ptr(), None) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(acc_d.cpu().numpy(), acc)
+
+
+def test_bgemm_is_deterministic():
+    rng = np.random.default_rng(3)
+    a = rng.standard_normal((300, 2048)).astype(np.float32)
+    w = rng.standard_normal((200, 2048)).astype(np.float32)
+    r1 = gpu_fc(a, w, False, 3, 3, np.float32(0.3), np.float32(0.3), np.float32(0.09))
+    r2 = gpu_fc(a, w, False, 3, 3, np.float32(0.3), np.float32(0.3), np.float32(0.09))
+    assert np.array_equal(r1["acc"], r2["acc"]) and np.array_equal(r1["out"].view(np.uint32), r2["out"].view(np.uint32))
+
+
+def test_config1_fc_layer():
+    c = wl.fc_config1(0)
+    got = run_case(c.a, c.w, c.k_major, c.ab, c.wb)
+    assert got["out"].shape == (64, 256)
+
+
+@pytest.mark.parametrize("wb,ab", wl.GEMM_SWEEP_BITS)
+def test_config3_gemm_4096_sampled(wb, ab):
+    """Full-size square GEMM; the oracle evaluates complete rows spread over the matrix plus random entries."""
+    c = wl.gemm_config3(0, 4096, wb, ab)
+    sa, sw, alpha = scales_for(c.a, c.w, ab, wb)
+    qa, qw = oracle_fc_codes(c.a, c.w, False, ab, wb, sa, sw)
+    got = gpu_fc(c.a, c.w, False, ab, wb, sa, sw, alpha, want_planes=True)
+    assert np.array_equal(got["a_planes"], oracle.pack_planes(qa, ab))
+    assert np.array_equal(got["w_planes"], oracle.pack_planes(qw, wb))
+    if (wb, ab) == (2, 2):
+        # the headline configuration is compared in full: all 16.7 M accumulators and outputs
+        want = oracle.fc(qa, qw)
+        assert np.array_equal(got["acc"], want)
+        assert_fp32_close(got["out"], oracle.scale(want, alpha))
+    else:
+        rows, cols = wl.sample_pairs(0, 4096, 4096, 200000, full_rows=24)
+        want = oracle.fc_sampled(qa, qw, rows, cols)
+        assert np.array_equal(got["acc"][rows, cols], want)
+        assert_fp32_close(got["out"][rows, cols], oracle.scale(want, alpha))
+    # property that holds at any size: every accumulator has the parity of Kg and is bounded by Kg*A*B
+    assert np.all((got["acc"] & 1) == 0) and np.abs(got["acc"]).max() <= 4096 * (2 ** ab - 1) * (2 ** wb - 1)
