@@ -1,6 +1,7 @@
 // qnn_bgemm / qnn_bconv2d: all plane-pair xor+popcount contractions of one layer,
 // the 2^(i+j) combine and the scale, in one launch.
 #include "qnn_internal.cuh"
+#include "bgemm_tiled.cuh"
 
 namespace {
 
@@ -93,6 +94,15 @@ extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int kw = (int)qnn_row_words_i(Kg);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
+    if (ab <= 4 && wb <= 4 && qnn_ceil_div(Ng, qnn_tiled::kBN) <= 65535) {
+        qnn_tiled::Params p = {};
+        p.a = a_planes; p.w = w; p.tapsum = nullptr;
+        p.Mg = Mg; p.Ng = Ng;
+        p.a_pitch = kw; p.w_pitch = kw; p.kwords = kw;
+        p.nstages = (int)qnn_ceil_div(kw, qnn_tiled::kStageWords);
+        p.n_elems = Kg; p.alpha = alpha; p.out = out; p.ldo = ldo; p.acc = acc;
+        return qnn_tiled::dispatch_tiled<false>(ab, wb, p, st);
+    }
     dim3 grid((unsigned)qnn_ceil_div(Ng, 16), (unsigned)qnn_ceil_div(Mg, 16));
     if (grid.y > 65535) return QNN_E_RANGE;
     bgemm_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, Mg, Ng, Kg, kw, alpha, out, ldo, acc);
@@ -122,11 +132,20 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
     if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
-    if (grid.y > 65535) {
-        // fold rows into x for very tall problems
-        return QNN_E_RANGE;
+    if (ab <= 4 && wb <= 4 && qnn_ceil_div(Cout, qnn_tiled::kBN) <= 65535) {
+        qnn_tiled::Params p = {};
+        p.a = a_planes; p.w = w;
+        p.tapsum = reinterpret_cast<const int32_t *>(w + (int64_t)Cout * wb * g.w_pitch);
+        p.Mg = Mg; p.Ng = Cout;
+        p.a_pitch = g.a_pitch; p.w_pitch = g.w_pitch; p.kwords = R * S * g.cw;
+        p.nstages = (int)qnn_ceil_div(p.kwords, qnn_tiled::kStageWords);
+        p.n_elems = R * S * C; p.alpha = alpha; p.out = out; p.ldo = Cout; p.acc = acc;
+        p.H = H; p.W = W; p.C = C; p.R = R; p.S = S; p.stride = stride; p.pad = pad; p.Ho = g.Ho; p.Wo = g.Wo;
+        p.cw = g.cw; p.piece = (g.cw % 4 == 0) ? 4 : ((g.cw % 2 == 0) ? 2 : 1);
+        return qnn_tiled::dispatch_tiled<true>(ab, wb, p, st);
     }
+    dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
+    if (grid.y > 65535) return QNN_E_RANGE;
     bconv_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, g, alpha, out, acc);
     return qnn_launch_status();
 }

@@ -1,0 +1,334 @@
+// Tiled xor+popcount contraction for ab, wb in 1..4 (FC and implicit-im2col convolution).
+//
+// CTA tile: BM activation rows x 64 output features, 256 threads, each thread a TM x 4 block of
+// outputs (rows ty + 16r, features tx + 16c) for ALL ab*wb plane pairs; TM = 4 (BM = 64) for
+// ab <= 2 and TM = 2 (BM = 32) for ab = 3, 4, so that the TM*ab*8 re-coded activation words of a
+// group stay in registers while the weight words stream past them.  The reduction runs in
+// stages of 16 words (512 elements) per (row, plane), double buffered in shared memory with
+// cp.async; the operand words of a stage are re-coded in place before use (see below).
+//
+// Carry-save contraction.  popcount issues at 16 lanes/clk/SM, 3-input logic at 64, so counting
+// every xor word separately is popcount-bound.  Eight xor words x0..x7 of one (output, plane pair)
+// are instead compressed with full adders on bit columns (a 7:3 counter: ones, twos, fours) and
+// only 4 words are counted: popc(ones) + popc(x7) + 2 popc(twos) + 4 popc(fours).
+// Because xor distributes over the operands, the sum output of an adder whose inputs are
+// x_p ^ x_q ^ x_r equals (a_p^a_q^a_r) ^ (w_p^w_q^w_r): the operand-side xors are computed ONCE
+// per staged word (not per output), so shared memory holds, per group of 8 words,
+//   T = [a0, a1, a0^a1^a2, a3, a4, a3^a4^a5, a0^...^a6, a7]
+// and the per-output work is 8 xors + 5 three-input logic ops + 4 popcounts + 4 multiply-adds.
+#pragma once
+#include "qnn_internal.cuh"
+
+namespace qnn_tiled {
+
+constexpr int kBN = 64, kThreads = 256;
+template <int AB> struct TileM { static constexpr int TM = (AB <= 2) ? 4 : 2, BM = 16 * TM; };
+constexpr int kStageChunks = 2;                   // groups of 8 words per stage
+constexpr int kStageWords = 8 * kStageChunks;     // words per (row, plane) per stage
+
+struct Params {
+    const uint32_t *a;
+    const uint32_t *w;
+    const int32_t *tapsum;   // conv only: [Ng][taps]
+    int64_t Mg;
+    int Ng;
+    int a_pitch, w_pitch;    // words per (row|pixel, plane) and per (feature, plane)
+    int kwords;              // words to contract per plane: FC = a_pitch, conv = taps*cw
+    int nstages;
+    int n_elems;             // FC: Kg (true reduction length)
+    float alpha;
+    float *out;
+    int64_t ldo;
+    int32_t *acc;
+    // convolution geometry
+    int H, W, C, R, S, stride, pad, Ho, Wo, cw, piece;   // piece = words per copy (4, 2 or 1)
+};
+
+__device__ __forceinline__ uint32_t lop3_xor3(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t lop3_maj(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// carry of the full adder with inputs (u, v, z) given u, v and the adder's SUM s = u^v^z
+__device__ __forceinline__ uint32_t lop3_carry_from_sum(uint32_t u, uint32_t v, uint32_t s) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xD4;" : "=r"(d) : "r"(u), "r"(v), "r"(s));
+    return d;
+}
+
+__device__ __forceinline__ void cp_async(uint32_t dst_smem, const void *src, int bytes_total, bool valid) {
+    // 16-, 8- or 4-byte asynchronous copy; an invalid source is replaced by zeros (src-size 0)
+    const int n = valid ? bytes_total : 0;
+    if (bytes_total == 16)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
+    else if (bytes_total == 8)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst_smem), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+// One (output, plane pair) over 8 re-coded words: returns nothing, adds the weighted count.
+// `shift` = i + j is a compile-time constant after unrolling.
+__device__ __forceinline__ void pair8(const uint32_t (&ta)[8], const uint32_t (&tw)[8], const int shift, int &acc) {
+    const uint32_t u = ta[0] ^ tw[0], v = ta[1] ^ tw[1], s1 = ta[2] ^ tw[2];
+    const uint32_t c1 = lop3_carry_from_sum(u, v, s1);
+    const uint32_t u2 = ta[3] ^ tw[3], v2 = ta[4] ^ tw[4], s2 = ta[5] ^ tw[5];
+    const uint32_t c2 = lop3_carry_from_sum(u2, v2, s2);
+    const uint32_t ones = ta[6] ^ tw[6];                       // x0^...^x6 = s1^s2^x6
+    const uint32_t c3 = lop3_carry_from_sum(s1, s2, ones);     // carry of (s1, s2, x6)
+    const uint32_t twos = lop3_xor3(c1, c2, c3), fours = lop3_maj(c1, c2, c3);
+    const uint32_t x7 = ta[7] ^ tw[7];
+    acc += __popc(ones) * (1 << shift);
+    acc += __popc(x7) * (1 << shift);
+    acc += __popc(twos) * (2 << shift);
+    acc += __popc(fours) * (4 << shift);
+}
+
+template <int AB, int WB, bool CONV>
+__global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p) {
+    constexpr int TM = TileM<AB>::TM, kBM = TileM<AB>::BM;
+    constexpr int A_UNITS = kBM * AB * kStageChunks;      // (row, plane, chunk) units per stage
+    constexpr int W_UNITS = kBN * WB * kStageChunks;
+    constexpr int A_VEC = kStageChunks * 2 * AB * kBM;    // uint4 per stage, A region
+    constexpr int W_VEC = kStageChunks * 2 * WB * kBN;
+    extern __shared__ uint4 smem[];                       // [2 buffers][A_VEC + W_VEC]
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int64_t m0 = (int64_t)blockIdx.x * kBM;
+    const int n0 = blockIdx.y * kBN;
+    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
+
+    // ---- per-thread staging bookkeeping: unit u = tid + 256*q  ->  row = tid % BM (A) or tid % 64 (W) for every q
+    const int srow = tid % kBM, wrow = tid % kBN;
+    const int64_t am = m0 + srow;
+    const bool arow_ok = am < p.Mg;
+    const bool wrow_ok = (n0 + wrow) < p.Ng;
+    int h0 = 0, w0 = 0;
+    int64_t pixbase = 0;
+    if (CONV) {
+        const int64_t mm = arow_ok ? am : 0;
+        const int wo = (int)(mm % p.Wo);
+        const int ho = (int)((mm / p.Wo) % p.Ho);
+        const int64_t n = mm / ((int64_t)p.Wo * p.Ho);
+        h0 = ho * p.stride - p.pad;
+        w0 = wo * p.stride - p.pad;
+        pixbase = n * p.H * p.W;
+    }
+
+    auto issue_stage = [&](int stage, int buf) {
+        const uint32_t a_smem = smem_base + (uint32_t)buf * (A_VEC + W_VEC) * 16u;
+        const uint32_t w_smem = a_smem + A_VEC * 16u;
+        const int kbase = stage * kStageWords;
+#pragma unroll
+        for (int q = 0; q < (A_UNITS + kThreads - 1) / kThreads; ++q) {
+            const int u = tid + q * kThreads;
+            if ((A_UNITS % kThreads) != 0 && u >= A_UNITS) break;
+            const int rp = u % (kBM * AB), ch = u / (kBM * AB);
+            const int plane = rp / kBM;                    // row == srow
+            const int kw0 = kbase + ch * 8;
+            if (!CONV) {
+                const uint32_t *src = p.a + ((int64_t)am * AB + plane) * p.a_pitch;
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    const int kw = kw0 + 4 * g;
+                    const bool ok = arow_ok && kw < p.kwords;
+                    const uint32_t dst = a_smem + (uint32_t)((((ch * 2 + g) * AB + plane) * kBM + srow) * 16);
+                    cp_async(dst, ok ? (const void *)(src + kw) : (const void *)p.a, 16, ok);
+                }
+            } else {
+                const int piece = p.piece;
+                for (int off = 0; off < 8; off += piece) {
+                    const int kw = kw0 + off;
+                    const int tap = kw / p.cw;
+                    const int cword = kw - tap * p.cw;
+                    const int r = tap / p.S, s = tap - r * p.S;
+                    const int hi = h0 + r, wi = w0 + s;
+                    const bool ok = arow_ok && kw < p.kwords && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                    const uint32_t *src = p.a + ((pixbase + (int64_t)hi * p.W + wi) * AB + plane) * p.a_pitch + cword;
+                    const int g = off >> 2;
+                    const uint32_t dst = a_smem + (uint32_t)((((ch * 2 + g) * AB + plane) * kBM + srow) * 16) + (uint32_t)(off & 3) * 4u;
+                    cp_async(dst, ok ? (const void *)src : (const void *)p.a, piece * 4, ok);
+                }
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < (W_UNITS + kThreads - 1) / kThreads; ++q) {
+            const int u = tid + q * kThreads;
+            if ((W_UNITS % kThreads) != 0 && u >= W_UNITS) break;
+            const int rp = u % (kBN * WB), ch = u / (kBN * WB);
+            const int plane = rp / kBN;
+            const int kw0 = kbase + ch * 8;
+            const uint32_t *src = p.w + ((int64_t)(n0 + wrow) * WB + plane) * p.w_pitch;
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                const int kw = kw0 + 4 * g;
+                const bool ok = wrow_ok && kw < p.kwords && kw < p.w_pitch;
+                const uint32_t dst = w_smem + (uint32_t)((((ch * 2 + g) * WB + plane) * kBN + wrow) * 16);
+                cp_async(dst, ok ? (const void *)(src + kw) : (const void *)p.w, 16, ok);
+            }
+        }
+        cp_async_commit();
+    };
+
+    // re-code the words this thread copied: [x0..x7] -> [x0, x1, x0^x1^x2, x3, x4, x3^x4^x5, x0^..^x6, x7]
+    auto recode_stage = [&](int buf) {
+        uint4 *a_s = smem + (size_t)buf * (A_VEC + W_VEC);
+        uint4 *w_s = a_s + A_VEC;
+        auto recode = [](uint4 *lo, uint4 *hi) {
+            uint4 x = *lo, y = *hi;
+            const uint32_t t2 = lop3_xor3(x.x, x.y, x.z);
+            const uint32_t t5 = lop3_xor3(x.w, y.x, y.y);
+            const uint32_t t6 = lop3_xor3(t2, t5, y.z);
+            *lo = make_uint4(x.x, x.y, t2, x.w);
+            *hi = make_uint4(y.x, t5, t6, y.w);
+        };
+#pragma unroll
+        for (int q = 0; q < (A_UNITS + kThreads - 1) / kThreads; ++q) {
+            const int u = tid + q * kThreads;
+            if ((A_UNITS % kThreads) != 0 && u >= A_UNITS) break;
+            const int rp = u % (kBM * AB), ch = u / (kBM * AB);
+            const int plane = rp / kBM;
+            recode(a_s + ((ch * 2 + 0) * AB + plane) * kBM + srow, a_s + ((ch * 2 + 1) * AB + plane) * kBM + srow);
+        }
+#pragma unroll
+        for (int q = 0; q < (W_UNITS + kThreads - 1) / kThreads; ++q) {
+            const int u = tid + q * kThreads;
+            if ((W_UNITS % kThreads) != 0 && u >= W_UNITS) break;
+            const int rp = u % (kBN * WB), ch = u / (kBN * WB);
+            const int plane = rp / kBN;
+            recode(w_s + ((ch * 2 + 0) * WB + plane) * kBN + wrow, w_s + ((ch * 2 + 1) * WB + plane) * kBN + wrow);
+        }
+    };
+
+    int acc[TM][4];
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = 0;
+
+    issue_stage(0, 0);
+    cp_async_wait_all();
+    recode_stage(0);
+    __syncthreads();
+
+    for (int stage = 0; stage < p.nstages; ++stage) {
+        const int buf = stage & 1;
+        if (stage + 1 < p.nstages) issue_stage(stage + 1, buf ^ 1);
+        const uint4 *a_s = smem + (size_t)buf * (A_VEC + W_VEC);
+        const uint4 *w_s = a_s + A_VEC;
+#pragma unroll 1
+        for (int ch = 0; ch < kStageChunks; ++ch) {
+            uint32_t ta[TM][AB][8];
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int i = 0; i < AB; ++i)
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const uint4 v = a_s[((ch * 2 + g) * AB + i) * kBM + ty + 16 * r];
+                        ta[r][i][4 * g + 0] = v.x; ta[r][i][4 * g + 1] = v.y;
+                        ta[r][i][4 * g + 2] = v.z; ta[r][i][4 * g + 3] = v.w;
+                    }
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int j = 0; j < WB; ++j) {
+                    uint32_t tw[8];
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const uint4 v = w_s[((ch * 2 + g) * WB + j) * kBN + tx + 16 * c];
+                        tw[4 * g + 0] = v.x; tw[4 * g + 1] = v.y; tw[4 * g + 2] = v.z; tw[4 * g + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int i = 0; i < AB; ++i) pair8(ta[r][i], tw, i + j, acc[r][c]);
+                }
+        }
+        if (stage + 1 < p.nstages) {
+            cp_async_wait_all();
+            recode_stage(buf ^ 1);
+        }
+        __syncthreads();
+    }
+
+    // ---- epilogue: acc holds S = sum_ij 2^(i+j) X_ij.  out = n_valid*A*B - 2*S (Eq. 8), times alpha (Eq. 9).
+    constexpr int AMAX = (1 << AB) - 1, PROD = AMAX * ((1 << WB) - 1);
+#pragma unroll
+    for (int r = 0; r < TM; ++r) {
+        const int64_t m = m0 + ty + 16 * r;
+        if (m >= p.Mg) continue;
+        int n_valid = p.n_elems;
+        int corr[4] = {0, 0, 0, 0};
+        if (CONV) {
+            // Taps outside the image were staged as zero words: each contributed popc(w_j) to X_ij, i.e.
+            // AMAX * tapsum[n][tap] to S, and must not be counted in the length.
+            const int wo = (int)(m % p.Wo);
+            const int ho = (int)((m / p.Wo) % p.Ho);
+            const int hh = ho * p.stride - p.pad, ww = wo * p.stride - p.pad;
+            int valid_taps = 0;
+            const bool interior = hh >= 0 && ww >= 0 && hh + p.R <= p.H && ww + p.S <= p.W;
+            if (interior) {
+                valid_taps = p.R * p.S;
+            } else {
+                for (int rr = 0; rr < p.R; ++rr)
+                    for (int ss = 0; ss < p.S; ++ss) {
+                        const int hi = hh + rr, wi = ww + ss;
+                        if (hi >= 0 && hi < p.H && wi >= 0 && wi < p.W) {
+                            ++valid_taps;
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const int n = n0 + tx + 16 * c;
+                                if (n < p.Ng) corr[c] += __ldg(p.tapsum + (int64_t)n * (p.R * p.S) + rr * p.S + ss);
+                            }
+                        }
+                    }
+            }
+            n_valid = valid_taps * p.C;
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int n = n0 + tx + 16 * c;
+            if (n >= p.Ng) continue;
+            const int32_t v = n_valid * PROD - 2 * (acc[r][c] - AMAX * corr[c]);
+            if (p.acc) p.acc[m * p.Ng + n] = v;
+            if (p.out) p.out[m * p.ldo + n] = __fmul_rn(__int2float_rn(v), p.alpha);
+        }
+    }
+}
+
+
+template <int AB, int WB, bool CONV>
+inline int launch_tiled(const Params &p, cudaStream_t st) {
+    constexpr int kBM = TileM<AB>::BM;
+    constexpr size_t smem = 2u * kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u;
+    if (smem > 48u * 1024u &&
+        cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+        return QNN_E_CUDA;
+    dim3 grid((unsigned)((p.Mg + kBM - 1) / kBM), (unsigned)((p.Ng + kBN - 1) / kBN));
+    bgemm_tiled_kernel<AB, WB, CONV><<<grid, kThreads, smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA;
+}
+
+template <bool CONV>
+inline int dispatch_tiled(int ab, int wb, const Params &p, cudaStream_t st) {
+#define QNN_T(A_, W_) \
+    if (ab == A_ && wb == W_) return launch_tiled<A_, W_, CONV>(p, st);
+    QNN_T(1, 1) QNN_T(1, 2) QNN_T(1, 3) QNN_T(1, 4)
+    QNN_T(2, 1) QNN_T(2, 2) QNN_T(2, 3) QNN_T(2, 4)
+    QNN_T(3, 1) QNN_T(3, 2) QNN_T(3, 3) QNN_T(3, 4)
+    QNN_T(4, 1) QNN_T(4, 2) QNN_T(4, 3) QNN_T(4, 4)
+#undef QNN_T
+    return QNN_E_ARG;
+}
+
+}  // namespace qnn_tiled
