@@ -160,8 +160,11 @@ int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float s
  * qnn_probe_bitops enqueues a register-resident kernel that does nothing but the
  * contraction's instruction mix and returns (in *word_ops) how many 32-bit
  * xor-popcount-accumulate word operations it performs; divide by its measured time.
- *   variant 0: xor + popc + add per word;  variant 1: the 3:2 carry-save form
- *   (3 xor, 2 three-input logic ops, 2 popc per 3 words).
+ *   variant 0: xor + popc + add per word, operands in registers (this is popcount-issue bound and so
+ *              measures the popcount pipe: one popcount per word);
+ *   variant 1: the 3:2 carry-save form in registers (3 xor, 2 three-input logic ops, 2 popc per 3 words);
+ *   variant 2: the tiled kernel's own inner loop (7:3 bit-column counters on re-coded operands: 8 xor,
+ *              5 three-input logic ops, 4 popc, 4 multiply-adds per 8 words) fed from shared memory.
  *   sink: device int32 [blocks*256], written once at the end.
  * qnn_probe_copy enqueues a plain 16-byte-vector device copy of `bytes` (multiple of 16).
  */

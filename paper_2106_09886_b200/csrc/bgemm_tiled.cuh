@@ -306,6 +306,64 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
 }
 
 
+// Peak probe: the inner loop of bgemm_tiled_kernel<2, 2> (same pair8, same register tile, same shared
+// memory layout) running `iters` times over one resident stage: no global traffic, barriers or epilogue.
+static __global__ void __launch_bounds__(kThreads, 2) probe_csa73_kernel(int iters, int32_t *sink) {
+    constexpr int AB = 2, WB = 2, TM = 4, kBM = 64;
+    constexpr int A_VEC = kStageChunks * 2 * AB * kBM, W_VEC = kStageChunks * 2 * WB * kBN;
+    __shared__ uint4 sm[A_VEC + W_VEC];
+    for (int i = threadIdx.x; i < A_VEC + W_VEC; i += kThreads) {
+        const uint32_t h = (uint32_t)(i + 1) * 2654435761u + blockIdx.x * 40503u;
+        sm[i] = make_uint4(h, h * 2246822519u, h ^ (h >> 7), h * 3266489917u + 1u);
+    }
+    __syncthreads();
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const uint4 *a_s = sm, *w_s = sm + A_VEC;
+    int acc[TM][4];
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = 0;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll 1
+        for (int ch = 0; ch < kStageChunks; ++ch) {
+            uint32_t ta[TM][AB][8];
+#pragma unroll
+            for (int r = 0; r < TM; ++r)
+#pragma unroll
+                for (int i = 0; i < AB; ++i)
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const uint4 v = a_s[((ch * 2 + g) * AB + i) * kBM + ty + 16 * r];
+                        ta[r][i][4 * g + 0] = v.x; ta[r][i][4 * g + 1] = v.y;
+                        ta[r][i][4 * g + 2] = v.z; ta[r][i][4 * g + 3] = v.w;
+                    }
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int j = 0; j < WB; ++j) {
+                    uint32_t tw[8];
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const uint4 v = w_s[((ch * 2 + g) * WB + j) * kBN + tx + 16 * c];
+                        tw[4 * g + 0] = v.x; tw[4 * g + 1] = v.y; tw[4 * g + 2] = v.z; tw[4 * g + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int r = 0; r < TM; ++r)
+#pragma unroll
+                        for (int i = 0; i < AB; ++i) pair8(ta[r][i], tw, i + j, acc[r][c]);
+                }
+        }
+    }
+    int s = 0;
+#pragma unroll
+    for (int r = 0; r < TM; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s += acc[r][c] * (r * 4 + c + 1);
+    sink[blockIdx.x * kThreads + threadIdx.x] = s;
+}
+constexpr double kProbeCsa73WordsPerThreadIter = 8.0 * kStageChunks * 4 * 4 * 2 * 2;
+
 template <int AB, int WB, bool CONV>
 inline int launch_tiled(const Params &p, cudaStream_t st) {
     constexpr int kBM = TileM<AB>::BM;

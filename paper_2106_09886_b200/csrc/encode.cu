@@ -11,52 +11,104 @@ namespace {
 
 constexpr int kEncThreads = 256;
 
-template <int BITS>
+// A unit is 128 consecutive elements: four ballots per plane give four canonical words.  For rows
+// longer than 64 elements a unit is a 128-element segment of one row (RPU = 1); for shorter rows
+// (NHWC activations with few channels) a unit spans RPU = 2 (k <= 64) or 4 (k <= 32) whole rows so
+// that the lanes stay busy.  UN units are loaded before the first ballot, so 4*UN independent
+// 128-byte requests per warp are in flight.  Unit indices advance incrementally (no division in the loop).
+template <int BITS, int UN, int RPU>
 __global__ void __launch_bounds__(kEncThreads)
-encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, bool relu,
-                   uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum, int segs_per_row, int kw) {
+encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, float lo,
+                   uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum, int groups_per_row, int segs_per_row,
+                   int kw, int64_t first_row_step, int first_grp_step) {
     const float half = (float)(1 << (BITS - 1));
-    const float amax = (float)((1 << BITS) - 1);
+    constexpr int amax = (1 << BITS) - 1;
+    constexpr int SPAN = 128 / RPU;                       // elements of one row inside a unit (RPU > 1)
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = ((int64_t)blockIdx.x * kEncThreads + threadIdx.x) >> 5;
-    const int64_t nwarps = ((int64_t)gridDim.x * kEncThreads) >> 5;
-    const int64_t units = rows * segs_per_row;
-    for (int64_t u = warp0; u < units; u += nwarps) {
-        const int64_t row = u / segs_per_row;
-        const int seg = (int)(u - row * segs_per_row);
-        const float *src = x + row * ldx;
-        const int k0 = seg * 128 + lane;
-        float v[4];
+    // group g = (row-unit, group of UN segments); RPU > 1 has one group per row-unit
+    int64_t ru = warp0 / groups_per_row;                  // row (RPU = 1) or index of a bundle of RPU rows
+    int grp = (int)(warp0 - ru * groups_per_row);
+    const int64_t n_ru = (RPU == 1) ? rows : ((rows + RPU - 1) / RPU + UN - 1) / UN;
+    for (; ru < n_ru;) {
+        float v[UN][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            int kk = k0 + 32 * j;
-            v[j] = (kk < k) ? __ldcs(src + kk) : 0.0f;
-        }
-        int t[4];
+        for (int q = 0; q < UN; ++q) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            int kk = k0 + 32 * j;
-            t[j] = (kk < k) ? qnn_code_t(v[j], inv2s, half, amax, relu) : 0;   // padding bits are 0
+            for (int j = 0; j < 4; ++j) {
+                int64_t row;
+                int kk;
+                if (RPU == 1) {
+                    row = ru;
+                    kk = (grp * UN + q) * 128 + 32 * j + lane;
+                } else {
+                    row = (ru * UN + q) * RPU + (32 * j) / SPAN;
+                    kk = (32 * j) % SPAN + lane;
+                }
+                const bool live = (RPU == 1) ? ((grp * UN + q) < segs_per_row) : (row < rows);
+                v[q][j] = (live && kk < k) ? __ldcs(x + row * ldx + kk) : 0.0f;
+            }
         }
-        uint4 mine = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int i = 0; i < BITS; ++i) {
-            uint32_t b0 = __ballot_sync(0xffffffffu, (t[0] >> i) & 1);
-            uint32_t b1 = __ballot_sync(0xffffffffu, (t[1] >> i) & 1);
-            uint32_t b2 = __ballot_sync(0xffffffffu, (t[2] >> i) & 1);
-            uint32_t b3 = __ballot_sync(0xffffffffu, (t[3] >> i) & 1);
-            if (lane == i) mine = make_uint4(b0, b1, b2, b3);
-        }
-        if (lane < BITS) {
-            uint4 *dst = reinterpret_cast<uint4 *>(planes + (row * BITS + lane) * (int64_t)kw + seg * 4);
-            *dst = mine;
-        }
-        if (rowsum != nullptr) {
-            int s = t[0] + t[1] + t[2] + t[3];
+        for (int q = 0; q < UN; ++q) {
+            const int seg = grp * UN + q;
+            if (RPU == 1 && seg >= segs_per_row) break;                            // warp-uniform
+            int t[4];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0) atomicAdd(rowsum + row, s);
+            for (int j = 0; j < 4; ++j) {
+                const int kk = (RPU == 1) ? seg * 128 + 32 * j + lane : (32 * j) % SPAN + lane;
+                const int code = qnn_code_t(v[q][j], inv2s, half, amax, lo);
+                t[j] = (kk < k) ? code : 0;                                        // padding bits are 0
+            }
+            uint32_t b[BITS][4];
+#pragma unroll
+            for (int i = 0; i < BITS; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) b[i][j] = __ballot_sync(0xffffffffu, t[j] & (1 << i));
+            if (RPU == 1) {
+                uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int i = 0; i < BITS; ++i)
+                    if (lane == i) mine = make_uint4(b[i][0], b[i][1], b[i][2], b[i][3]);
+                if (lane < BITS)
+                    *reinterpret_cast<uint4 *>(planes + (ru * BITS + lane) * (int64_t)kw + seg * 4) = mine;
+                if (rowsum != nullptr) {
+                    int s = t[0] + t[1] + t[2] + t[3];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                    if (lane == 0) atomicAdd(rowsum + ru, s);
+                }
+            } else {
+                // lane r*BITS + i stores plane i of bundle row r: words [b(r-th span)...], rest 0 (kw == 4)
+                constexpr int WPR = SPAN / 32;            // ballots per row: 2 or 1
+                uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int r = 0; r < RPU; ++r)
+#pragma unroll
+                    for (int i = 0; i < BITS; ++i)
+                        if (lane == r * BITS + i)
+                            mine = make_uint4(b[i][r * WPR], WPR == 2 ? b[i][r * WPR + 1] : 0u, 0u, 0u);
+                const int64_t row = (ru * UN + q) * RPU + lane / BITS;
+                if (lane < RPU * BITS && row < rows)
+                    *reinterpret_cast<uint4 *>(planes + (row * BITS + lane % BITS) * (int64_t)kw) = mine;
+                if (rowsum != nullptr) {
+#pragma unroll
+                    for (int r = 0; r < RPU; ++r) {
+                        int s = 0;
+#pragma unroll
+                        for (int jj = 0; jj < WPR; ++jj) s += t[r * WPR + jj];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                        const int64_t rr = (ru * UN + q) * RPU + r;
+                        if (lane == 0 && rr < rows) rowsum[rr] = s;
+                    }
+                }
+            }
         }
+        // advance by the number of warps in the grid without dividing
+        grp += first_grp_step;
+        ru += first_row_step;
+        if (grp >= groups_per_row) { grp -= groups_per_row; ++ru; }
     }
 }
 
@@ -67,7 +119,7 @@ __global__ void __launch_bounds__(kEncThreads)
 pack_weights_kernel(const float *__restrict__ w, int n_out, int taps, int c_in, int layout, float inv2s,
                     uint32_t *__restrict__ planes, int kw, int cw) {
     const float half = (float)(1 << (BITS - 1));
-    const float amax = (float)((1 << BITS) - 1);
+    constexpr int amax = (1 << BITS) - 1;
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = ((int64_t)blockIdx.x * kEncThreads + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * kEncThreads) >> 5;
@@ -88,7 +140,7 @@ pack_weights_kernel(const float *__restrict__ w, int n_out, int taps, int c_in, 
                 if (layout == QNN_W_NTC) idx = ((int64_t)n * taps + tap) * c_in + c;
                 else if (layout == QNN_W_TCN) idx = ((int64_t)tap * c_in + c) * n_out + n;
                 else idx = ((int64_t)n * c_in + c) * taps + tap;
-                t[j] = qnn_code_t(w[idx], inv2s, half, amax, false);
+                t[j] = qnn_code_t(w[idx], inv2s, half, amax, -INFINITY);
             }
         }
         uint4 mine = make_uint4(0u, 0u, 0u, 0u);
@@ -148,10 +200,33 @@ int grid_for(int64_t warps_needed) {
 template <int BITS>
 void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float inv2s, bool relu, uint32_t *planes,
                    int32_t *rowsum, cudaStream_t st) {
+    constexpr int UN = 4;
+    const float lo = relu ? 0.0f : -INFINITY;
     const int kw = (int)qnn_row_words_i(k);
     const int segs = kw / 4;
-    encode_pack_kernel<BITS><<<grid_for(rows * segs), kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, relu, planes,
-                                                                          rowsum, segs, kw);
+    int groups;
+    int64_t total;                                   // warp-level work items
+    const int rpu = (k <= 32 && 4 * BITS <= 32) ? 4 : (k <= 64 ? 2 : 1);
+    if (rpu == 1) {
+        groups = (int)qnn_ceil_div(segs, UN);
+        total = rows * groups;
+    } else {
+        groups = 1;
+        total = qnn_ceil_div(qnn_ceil_div(rows, rpu), UN);
+    }
+    const int grid = grid_for(total);
+    const int64_t nwarps = (int64_t)grid * (kEncThreads / 32);
+    const int64_t row_step = nwarps / groups;
+    const int grp_step = (int)(nwarps % groups);
+    if (rpu == 1)
+        encode_pack_kernel<BITS, UN, 1><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, planes, rowsum, groups,
+                                                                    segs, kw, row_step, grp_step);
+    else if (rpu == 2)
+        encode_pack_kernel<BITS, UN, 2><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, planes, rowsum, groups,
+                                                                    segs, kw, row_step, grp_step);
+    else
+        encode_pack_kernel<BITS, UN, 4><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, planes, rowsum, groups,
+                                                                    segs, kw, row_step, grp_step);
 }
 
 template <int BITS>
@@ -186,7 +261,8 @@ extern "C" int qnn_encode_pack(const float *x, int64_t rows, int k, int64_t ldx,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float inv2s = 1.0f / (2.0f * scale);
     const bool relu = (flags & QNN_RELU) != 0;
-    if (rowsum && cudaMemsetAsync(rowsum, 0, (size_t)rows * sizeof(int32_t), st) != cudaSuccess) return QNN_E_CUDA;
+    if (rowsum && k > 64 && cudaMemsetAsync(rowsum, 0, (size_t)rows * sizeof(int32_t), st) != cudaSuccess)
+        return QNN_E_CUDA;
 #define CALL(B) launch_encode<B>(x, rows, k, ldx, inv2s, relu, planes, rowsum, st)
     QNN_DISPATCH_BITS(bits, CALL)
 #undef CALL

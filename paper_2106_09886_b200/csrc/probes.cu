@@ -1,5 +1,6 @@
 // Peak probes: a register-resident kernel with the contraction's instruction mix, and a plain copy.
 #include "qnn_internal.cuh"
+#include "bgemm_tiled.cuh"
 
 namespace {
 
@@ -85,15 +86,18 @@ __global__ void __launch_bounds__(256) probe_copy_kernel(uint4 *__restrict__ dst
 }  // namespace
 
 extern "C" int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream) {
-    if (!sink || iters <= 0 || blocks <= 0 || (variant != 0 && variant != 1)) return QNN_E_ARG;
+    if (!sink || iters <= 0 || blocks <= 0 || (variant < 0 || variant > 2)) return QNN_E_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double per_thread_iter;
     if (variant == 0) {
         probe_popc_kernel<8, 4><<<blocks, 256, 0, st>>>(iters, sink);
         per_thread_iter = 32.0;
-    } else {
+    } else if (variant == 1) {
         probe_csa_kernel<4, 4><<<blocks, 256, 0, st>>>(iters, sink);
         per_thread_iter = 48.0;
+    } else {
+        qnn_tiled::probe_csa73_kernel<<<blocks, 256, 0, st>>>(iters, sink);
+        per_thread_iter = qnn_tiled::kProbeCsa73WordsPerThreadIter;
     }
     if (word_ops) *word_ops = per_thread_iter * iters * 256.0 * blocks;
     return qnn_launch_status();

@@ -17,13 +17,16 @@ static inline int64_t qnn_w_row_words_i(int taps, int c_in) {
 static inline int qnn_launch_status() { return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA; }
 
 // Unsigned code t in [0, 2^bits - 1] of a real value (odd code q = 2t - (2^bits - 1)).
-// inv2s = 1/(2*scale), half = 2^(bits-1), amax = 2^bits - 1.
-// One fused multiply-add, then floor for positive x and ceil-1 otherwise, so that
-// a value half-way between two codes moves away from zero and 0 maps to q = -1.
-__device__ __forceinline__ int qnn_code_t(float x, float inv2s, float half, float amax, bool relu) {
-    if (relu) x = fmaxf(x, 0.0f);
-    float v = __fmaf_rn(x, inv2s, half);
-    float tf = (x > 0.0f) ? floorf(v) : ceilf(v) - 1.0f;
-    tf = fminf(fmaxf(tf, 0.0f), amax);
-    return __float2int_rz(tf);
+// inv2s = 1/(2*scale), half = 2^(bits-1), amax = 2^bits - 1, lo = 0 for a fused ReLU else -inf.
+// v = x/(2s) + 2^(b-1) with one fused multiply-add; t = floor(v) for x > 0 and ceil(v) - 1 otherwise,
+// so that a value half-way between two codes moves away from zero and 0 maps to q = -1.
+// ceil(v) - 1 = -floor(-v) - 1 = ~floor(-v): one saturating float->int conversion (round down)
+// serves both branches; NaN converts to 0 and ends at t = 0, infinities saturate and are clamped.
+__device__ __forceinline__ int qnn_code_t(float x, float inv2s, float half, int amax, float lo) {
+    x = fmaxf(x, lo);
+    const float v = __fmaf_rn(x, inv2s, half);
+    const bool pos = x > 0.0f;
+    const int f = __float2int_rd(pos ? v : -v);
+    const int t = pos ? f : ~f;
+    return min(max(t, 0), amax);
 }

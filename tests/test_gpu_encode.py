@@ -97,3 +97,22 @@ def test_absmax(env):
             x[3] = np.nan
         got = qnn.absmax_f32(torch.from_numpy(x).to(dev)).cpu().numpy()[0]
         assert got == np.float32(17.25)
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("rows,k", [(1, 3), (7, 3), (1001, 3), (5, 32), (1000, 32), (3, 33), (999, 64), (1234, 40),
+                                    (6, 65), (4097, 64), (50000, 16)])
+def test_encode_pack_short_rows(env, bits, rows, k):
+    """Rows of at most 64 elements (NHWC activations with few channels) take the multi-row path."""
+    torch, qnn, dev = env
+    rng = np.random.default_rng(bits * 100 + rows + k)
+    x = rng.standard_normal((rows, k)).astype(np.float32)
+    scale = np.float32(np.abs(x).max()) / np.float32(2 ** bits - 1)
+    for relu in (False, True):
+        q = oracle.quantize(x, bits, scale, relu)
+        want = oracle.pack_planes(q, bits)
+        rowsum = torch.full((rows,), -7, dtype=torch.int32, device=dev)
+        got = qnn.encode_pack(torch.from_numpy(x).to(dev), bits, scale, qnn.RELU if relu else 0, rowsum=rowsum)
+        torch.cuda.synchronize()
+        assert np.array_equal(got.cpu().numpy().view(np.uint32), want)
+        assert np.array_equal(rowsum.cpu().numpy(), ((q.astype(np.int64) + 2 ** bits - 1) // 2).sum(axis=1))
