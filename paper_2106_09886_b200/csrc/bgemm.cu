@@ -94,12 +94,11 @@ extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int kw = (int)qnn_row_words_i(Kg);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    if (ab <= 4 && wb <= 4 && qnn_ceil_div(Ng, qnn_tiled::kBN) <= 65535) {
+    if (ab <= 4 && wb <= 4) {
         qnn_tiled::Params p = {};
         p.a = a_planes; p.w = w; p.tapsum = nullptr;
         p.Mg = Mg; p.Ng = Ng;
         p.a_pitch = kw; p.w_pitch = kw; p.kwords = kw;
-        p.nstages = (int)qnn_ceil_div(kw, qnn_tiled::kStageWords);
         p.n_elems = Kg; p.alpha = alpha; p.out = out; p.ldo = ldo; p.acc = acc;
         return qnn_tiled::dispatch_tiled<false>(ab, wb, p, st);
     }
@@ -132,13 +131,16 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
     if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    if (ab <= 4 && wb <= 4 && qnn_ceil_div(Cout, qnn_tiled::kBN) <= 65535) {
+    // the tiled kernel divides by cw and S with a 20-bit multiply-shift: exact while kwords*cw and taps*S < 2^20
+    if (ab <= 4 && wb <= 4 && (int64_t)R * S * g.cw * g.cw < (1 << 20) && (int64_t)R * S * S < (1 << 20) &&
+        (int64_t)R * S * g.cw < 4096) {
         qnn_tiled::Params p = {};
         p.a = a_planes; p.w = w;
         p.tapsum = reinterpret_cast<const int32_t *>(w + (int64_t)Cout * wb * g.w_pitch);
         p.Mg = Mg; p.Ng = Cout;
         p.a_pitch = g.a_pitch; p.w_pitch = g.w_pitch; p.kwords = R * S * g.cw;
-        p.nstages = (int)qnn_ceil_div(p.kwords, qnn_tiled::kStageWords);
+        p.cw_magic = (1u << 20) / (uint32_t)g.cw + 1u;
+        p.s_magic = (1u << 20) / (uint32_t)S + 1u;
         p.n_elems = R * S * C; p.alpha = alpha; p.out = out; p.ldo = Cout; p.acc = acc;
         p.H = H; p.W = W; p.C = C; p.R = R; p.S = S; p.stride = stride; p.pad = pad; p.Ho = g.Ho; p.Wo = g.Wo;
         p.cw = g.cw; p.piece = (g.cw % 4 == 0) ? 4 : ((g.cw % 2 == 0) ? 2 : 1);
