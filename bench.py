@@ -44,6 +44,20 @@ UNIT = "binary TOPS"
 POPC_PER_WORD = 0.5   # popcounts the tiled kernel issues per 32-bit xor word (7:3 bit-column counters)
 
 
+# DRAM read+write of one qnn_bgemm 4096^3 w2a2 launch from the ncu capture summarised in
+# profiles/bgemm_tiled_4096_w2a2.md, valid for the kernel source with this digest only.
+NCU_TRAFFIC = {"bytes": None, "kernel_sha256": None}
+
+
+def ncu_traffic_bytes():
+    import hashlib
+    src = ROOT / "paper_2106_09886_b200" / "csrc" / "bgemm_tiled.cuh"
+    if NCU_TRAFFIC["bytes"] is None or not src.exists():
+        return None
+    digest = hashlib.sha256(src.read_bytes()).hexdigest()
+    return NCU_TRAFFIC["bytes"] if digest == NCU_TRAFFIC["kernel_sha256"] else None
+
+
 def binary_ops(Mg, Ng, Kg, ab, wb):
     return 2.0 * Mg * Ng * Kg * ab * wb
 
@@ -109,6 +123,27 @@ def dist_setup(n_gpus: int):
     return rank, world, local
 
 
+def max_over_ranks(values, device, use_dist: bool):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if use_dist:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_value(ms_per_step: float, world: int):
+    """Binary TOPS of the whole job: every rank processes its own 4096-row batch per step (weak scaling)."""
+    return binary_ops(N_SQ, N_SQ, N_SQ, AB, WB) * world / (ms_per_step * 1e-3) / 1e12
+
+
+def rank_workload(rank: int):
+    """Per-rank inputs: the weights are the same on every rank, the activation batch is drawn per rank."""
+    from paper_2106_09886_b200 import workloads as wl
+    return wl.gemm_config3(0, N_SQ, WB, AB, variant=rank)
+
+
 # ----------------------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle on the host cores
 # ----------------------------------------------------------------------------------------------------------
@@ -168,12 +203,13 @@ def measure_peaks(torch, qnn, dev):
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     sink = torch.empty(sms * 8 * 256, dtype=torch.int32, device=dev)
     res = {}
-    for variant, name in ((0, "xor_popc_add"), (1, "csa_3to2"), (2, "kernel_mix_smem")):
+    for variant, name, iters in ((0, "xor_popc_add", 4000), (1, "csa_3to2", 4000), (2, "kernel_mix_smem", 100),
+                                 (3, "mma_sync_b1_and_popc", 500), (4, "mma_sync_b1_xor_popc", 500)):
         best = 0.0
         for _ in range(4):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            ops = qnn.probe_bitops(variant, 4000, sms * 8, sink)
+            ops = qnn.probe_bitops(variant, iters, sms * 8, sink)
             e1.record()
             e1.synchronize()
             best = max(best, ops / (e0.elapsed_time(e1) * 1e-3))
@@ -239,7 +275,7 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=dev)
 
     # ---- workload: per-rank batch of rows (seeded per rank), replicated weights, packed offline
-    c = wl.gemm_config3(0, N_SQ, WB, AB, variant=rank)
+    c = rank_workload(rank)
     sa, sw = wl.per_tensor_scale(c.a, AB), wl.per_tensor_scale(c.w, WB)
     alpha = float(np.float32(sa * sw))
     Mg = Ng = Kg = N_SQ
@@ -311,15 +347,12 @@ def run_gpu(args):
     e2e_ms_total = s2.elapsed_time(t2)
     checksum = float(out_host[0, 0])
 
-    times = torch.tensor([ms_total, e2e_ms_total], dtype=torch.float64, device=dev)
-    if use_dist:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms_total = (float(v) for v in times.cpu())
+    ms_total, e2e_ms_total = max_over_ranks([ms_total, e2e_ms_total], dev, use_dist)
 
     if rank == 0:
         ms_step = ms_total / args.steps
         ops_step = binary_ops(Mg, Ng, Kg, AB, WB) * world
-        value = ops_step / (ms_step * 1e-3) / 1e12
+        value = whole_job_value(ms_step, world)
         e2e_ms = e2e_ms_total / e2e_steps
         mp, mp_kind = load_measured_peaks()
         # The plain probe is popcount-issue bound (one popcount per word), so it measures the popcount
@@ -330,13 +363,7 @@ def run_gpu(args):
         achieved = binary_ops(Mg, Ng, Kg, AB, WB) / (gemm_ms * 1e-3) / 1e12
         alg_bytes_gemm = Mg * Kg * AB / 8 + Ng * Kg * WB / 8 + Mg * Ng * 4
         enc_bytes = Mg * Kg * 4 + Mg * Kg * AB / 8
-        traffic = None
-        tfile = ROOT / "profiles" / "traffic.json"
-        if tfile.exists():
-            try:
-                traffic = json.loads(tfile.read_text()).get("bgemm_4096_w2a2_dram_bytes_per_launch")
-            except Exception:
-                traffic = None
+        traffic = ncu_traffic_bytes()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -359,6 +386,8 @@ def run_gpu(args):
                          "peak_analytic": peak_analytic,
                          "probe_xor_popc_add": peaks["xor_popc_add"], "probe_csa_3to2": peaks["csa_3to2"],
                          "probe_kernel_mix_smem": peaks["kernel_mix_smem"],
+                         "probe_mma_sync_b1_and_popc": peaks["mma_sync_b1_and_popc"],
+                         "probe_mma_sync_b1_xor_popc": peaks["mma_sync_b1_xor_popc"],
                          "frac_of_kernel_mix_probe": achieved / peaks["kernel_mix_smem"],
                          "algorithmic_bytes": alg_bytes_gemm,
                          "hbm_time_ms": alg_bytes_gemm / (mp["hbm_gbs"] * 1e9) * 1e3,

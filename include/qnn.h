@@ -164,7 +164,9 @@ int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float s
  *              measures the popcount pipe: one popcount per word);
  *   variant 1: the 3:2 carry-save form in registers (3 xor, 2 three-input logic ops, 2 popc per 3 words);
  *   variant 2: the tiled kernel's own inner loop (7:3 bit-column counters on re-coded operands: 8 xor,
- *              5 three-input logic ops, 4 popc, 4 multiply-adds per 8 words) fed from shared memory.
+ *              5 three-input logic ops, 4 popc, 4 multiply-adds per 8 words) fed from shared memory;
+ *   variant 3 / 4: warp-level 1-bit tensor-core instruction mma.sync m16n8k256 with and.popc / xor.popc,
+ *              operands in registers (word_ops counts 32 binary multiply-accumulates as one word operation).
  *   sink: device int32 [blocks*256], written once at the end.
  * qnn_probe_copy enqueues a plain 16-byte-vector device copy of `bytes` (multiple of 16).
  */

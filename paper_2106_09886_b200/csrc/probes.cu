@@ -78,6 +78,42 @@ __global__ void __launch_bounds__(256) probe_csa_kernel(int iters, int32_t *sink
     sink[blockIdx.x * 256 + threadIdx.x] = s;
 }
 
+// Warp-level 1-bit MMA (m16n8k256), eight independent accumulator tiles per warp, fixed operands.
+// XOR = false: and.popc, true: xor.popc.  One instruction is 16*8*256 binary multiply-accumulates.
+template <bool XOR>
+__global__ void __launch_bounds__(256) probe_bmma_kernel(int iters, int32_t *sink) {
+    const uint32_t h = (threadIdx.x + 1u) * 2654435761u + blockIdx.x;
+    const uint32_t a0 = h, a1 = h * 2246822519u, a2 = h ^ (h >> 5), a3 = h * 3266489917u, b0 = ~h, b1 = h * 40503u;
+    int d[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) d[i][j] = 0;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (XOR)
+                asm volatile(
+                    "mma.sync.aligned.m16n8k256.row.col.s32.b1.b1.s32.xor.popc {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                    "{%0,%1,%2,%3};"
+                    : "+r"(d[i][0]), "+r"(d[i][1]), "+r"(d[i][2]), "+r"(d[i][3])
+                    : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+            else
+                asm volatile(
+                    "mma.sync.aligned.m16n8k256.row.col.s32.b1.b1.s32.and.popc {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                    "{%0,%1,%2,%3};"
+                    : "+r"(d[i][0]), "+r"(d[i][1]), "+r"(d[i][2]), "+r"(d[i][3])
+                    : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        }
+    }
+    int s = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s += d[i][j];
+    sink[blockIdx.x * 256 + threadIdx.x] = s;
+}
+
 __global__ void __launch_bounds__(256) probe_copy_kernel(uint4 *__restrict__ dst, const uint4 *__restrict__ src, size_t n) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
         dst[i] = src[i];
@@ -86,7 +122,7 @@ __global__ void __launch_bounds__(256) probe_copy_kernel(uint4 *__restrict__ dst
 }  // namespace
 
 extern "C" int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream) {
-    if (!sink || iters <= 0 || blocks <= 0 || (variant < 0 || variant > 2)) return QNN_E_ARG;
+    if (!sink || iters <= 0 || blocks <= 0 || (variant < 0 || variant > 4)) return QNN_E_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double per_thread_iter;
     if (variant == 0) {
@@ -95,9 +131,13 @@ extern "C" int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sin
     } else if (variant == 1) {
         probe_csa_kernel<4, 4><<<blocks, 256, 0, st>>>(iters, sink);
         per_thread_iter = 48.0;
-    } else {
+    } else if (variant == 2) {
         qnn_tiled::probe_csa73_kernel<<<blocks, 256, 0, st>>>(iters, sink);
         per_thread_iter = qnn_tiled::kProbeCsa73WordsPerThreadIter;
+    } else {
+        if (variant == 3) probe_bmma_kernel<false><<<blocks, 256, 0, st>>>(iters, sink);
+        else probe_bmma_kernel<true><<<blocks, 256, 0, st>>>(iters, sink);
+        per_thread_iter = 8.0 * 16 * 8 * 256 / 32.0 / 32.0;   // 8 MMAs per warp iteration, in 32-bit word-ops per thread
     }
     if (word_ops) *word_ops = per_thread_iter * iters * 256.0 * blocks;
     return qnn_launch_status();
