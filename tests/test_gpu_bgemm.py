@@ -118,3 +118,24 @@ def test_config3_gemm_4096_sampled(wb, ab):
         assert_fp32_close(got["out"][rows, cols], oracle.scale(want, alpha))
     # property that holds at any size: every accumulator has the parity of Kg and is bounded by Kg*A*B
     assert np.all((got["acc"] & 1) == 0) and np.abs(got["acc"]).max() <= 4096 * (2 ** ab - 1) * (2 ** wb - 1)
+
+
+def test_fc_forward_host_matches_oracle():
+    """qnn_fc_forward_host: pinned host buffers in and out, device staging buffers supplied by the caller."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(21)
+    a = np.abs(rng.standard_normal((300, 1000))).astype(np.float32)
+    w = (0.02 * rng.standard_normal((200, 1000))).astype(np.float32)
+    sa, sw, alpha = scales_for(a, w, 2, 2)
+    _, _, acc, out = oracle_fc(a, w, False, 2, 2, sa, sw, alpha)
+    packed = qnn.pack_weights(torch.from_numpy(w).to(dev), 200, 1, 1000, qnn.W_NTC, 2, sw)
+    x_host = torch.from_numpy(a).pin_memory()
+    out_host = torch.zeros((300, 200), dtype=torch.float32).pin_memory()
+    x_dev = torch.empty((300, 1000), dtype=torch.float32, device=dev)
+    planes = torch.empty((300, 2, qnn.row_words(1000)), dtype=torch.int32, device=dev)
+    out_dev = torch.empty((300, 200), dtype=torch.float32, device=dev)
+    qnn.fc_forward_host(x_host, 2, sa, 0, packed, 2, 200, alpha, out_host, x_dev, planes, out_dev)
+    torch.cuda.synchronize()
+    assert_fp32_close(out_host.numpy(), out)
