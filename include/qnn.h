@@ -156,6 +156,40 @@ int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float s
                         uint32_t *planes_dev, float *out_dev, void *stream);
 
 /*
+ * One FC layer for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * packaging of qnn_encode_pack + qnn_bgemm, not a step of the method.)
+ *
+ * Some callers only ever hold the pointers they were given: a plug-in callback inside a host framework
+ * that owns all device memory and forbids allocation from callbacks, a real-time loop whose memory was
+ * fixed at start-up, a plain C program without an allocator.  They cannot supply the activation-planes
+ * buffer that sits between the encoder and the contraction.  This call keeps that buffer inside the
+ * library, as a fixed array of QNN_NOALLOC_SCRATCH_BYTES in the GPU's global memory (each GPU that loads
+ * the library holds it until the process exits), and calls neither cudaMalloc nor cudaFree nor any
+ * routine that allocates.
+ *
+ *   x         fp32 [Mg][ldx] (device), first Kg entries of each row used
+ *   w_packed  blob of qnn_pack_weights(n_out = Ng, taps = 1, c_in = Kg, bits = wb) (device)
+ *   out       fp32 [Mg][ldo] (device), ldo >= Ng
+ * Computes exactly what qnn_encode_pack followed by qnn_bgemm computes (same kernels, same bits).
+ *
+ * Limit: qnn_planes_bytes(Mg, Kg, ab) must not exceed QNN_NOALLOC_SCRATCH_BYTES (e.g. 4096 x 4096 at
+ * up to 4 bits, or 16384 x 4096 at 1 bit); larger problems are refused with QNN_E_RANGE before anything
+ * is enqueued.  Other argument errors are reported as by the two underlying calls.
+ *
+ * First call on a device: the library looks up the device address of its array once per device, with
+ * that device current (a host-side runtime query, no allocation).  Make that first call outside any
+ * stream capture; later calls only enqueue the two kernels on `stream`.
+ *
+ * Sharing: every call on a device uses the same array and leaves its planes there.  Nothing needs to
+ * start at zero (the encoder overwrites every word it will read, padding included), so consecutive calls
+ * on one stream are safe; two calls whose kernels can overlap on the GPU (different streams, or different
+ * host threads on different streams) race on the array and must be ordered by the caller.
+ */
+#define QNN_NOALLOC_SCRATCH_BYTES (8u << 20)
+int qnn_fc_forward_noalloc(const float *x, int64_t Mg, int Kg, int64_t ldx, int ab, float scale_a, unsigned flags,
+                           const void *w_packed, int wb, int Ng, float alpha, float *out, int64_t ldo, void *stream);
+
+/*
  * Peak probes used to state a roofline next to a measurement.
  * qnn_probe_bitops enqueues a register-resident kernel that does nothing but the
  * contraction's instruction mix and returns (in *word_ops) how many 32-bit

@@ -20,8 +20,9 @@ W_NTC, W_TCN, W_NCT = 0, 1, 2
 EXPORTS = [
     "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
-    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_probe_bitops", "qnn_probe_copy",
+    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
+NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 class QnnError(RuntimeError):
@@ -53,6 +54,7 @@ def _load() -> C.CDLL:
     lib.qnn_bconv2d.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
+    lib.qnn_fc_forward_noalloc.argtypes = [p, i64, i, i64, i, f, u, p, i, i, f, p, i64, p]
     lib.qnn_probe_bitops.argtypes = [i, i, i, p, C.POINTER(C.c_double), p]
     lib.qnn_probe_copy.argtypes = [p, p, sz, p]
     return lib
@@ -179,6 +181,20 @@ def fc_forward_host(x_host: torch.Tensor, ab: int, scale_a: float, flags: int, w
                                    float(alpha), _ptr(out_host), _ptr(x_dev), _ptr(planes_dev), _ptr(out_dev),
                                    _stream(stream)), "qnn_fc_forward_host")
     return out_host
+
+
+def fc_forward_noalloc(x: torch.Tensor, ab: int, scale_a: float, flags: int, w_packed: torch.Tensor, wb: int, Ng: int,
+                       alpha: float, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """FC layer for callers that cannot allocate: the activation planes live in the library's built-in
+    buffer (at most NOALLOC_SCRATCH_BYTES of planes).  Only `out`, if not given, is allocated here, by torch."""
+    _dev(x, torch.float32, "x")
+    Mg, Kg = x.shape
+    if out is None:
+        out = torch.empty((Mg, Ng), dtype=torch.float32, device=x.device)
+    _check(lib.qnn_fc_forward_noalloc(_ptr(x), Mg, Kg, x.stride(0), ab, float(scale_a), flags, _ptr(w_packed), wb, Ng,
+                                      float(alpha), _ptr(out), out.stride(0), _stream(stream)),
+           "qnn_fc_forward_noalloc")
+    return out
 
 
 def probe_bitops(variant: int, iters: int, blocks: int, sink: torch.Tensor, stream=None) -> float:
