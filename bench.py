@@ -231,6 +231,48 @@ def measure_peaks(torch, qnn, dev):
     return res
 
 
+def int8_tensor_comparison(torch, qnn, dev, a_dev, w_host, sa, sw, planes, packed, alpha):
+    """Comparison only: the same integer product computed as ONE int8 tensor-core GEMM on the unpacked odd
+    codes (library call: cuBLASLt through torch._int_mm), i.e. what the binary decomposition competes with
+    on this GPU.  The codes are rebuilt from the library's own bit planes, and the int32 result is checked
+    to be identical to qnn_bgemm's accumulators."""
+    try:
+        Mg, Kg = a_dev.shape
+        def codes_from_planes(pl, bits, k):
+            # pl: int32 [rows, bits, kw]; q = 2t - (2^bits - 1), bit i of t = plane i
+            rows = pl.shape[0]
+            shifts = torch.arange(32, device=dev, dtype=torch.int32)
+            t = torch.zeros((rows, pl.shape[2] * 32), dtype=torch.int32, device=dev)
+            for i in range(bits):
+                bitsv = (pl[:, i, :].unsqueeze(-1) >> shifts) & 1
+                t += bitsv.reshape(rows, -1) << i
+            return (2 * t[:, :k] - (2 ** bits - 1)).to(torch.int8).contiguous()
+        wp, _ = qnn.weights_views(packed, N_SQ, 1, N_SQ, WB)
+        qa = codes_from_planes(planes, AB, Kg)
+        qw = codes_from_planes(wp, WB, Kg)
+        qwt = qw.t().contiguous().t()          # column-major operand, as cuBLASLt's int8 path wants
+        ref = torch._int_mm(qa, qw.t())
+        _, acc = qnn.bgemm(planes, AB, packed, WB, Mg, N_SQ, Kg, alpha, want_acc=True)
+        torch.cuda.synchronize()
+        same = bool(torch.equal(ref, acc))
+        for _ in range(3):
+            torch._int_mm(qa, qw.t())
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._int_mm(qa, qw.t())
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        return {"what": "int8 tensor-core GEMM on the unpacked odd codes, cuBLASLt via torch._int_mm (library call, comparison only)",
+                "ms": ms, "equiv_int_gops": 2.0 * Mg * N_SQ * Kg / (ms * 1e-3) / 1e9, "int32_result_identical_to_qnn_bgemm": same}
+    except Exception as exc:   # comparison only: never fail the benchmark over it
+        return {"what": "int8 tensor-core GEMM comparison", "unavailable": f"{type(exc).__name__}: {exc}"[:200]}
+
+
 def load_measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -301,6 +343,10 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     peaks = measure_peaks(torch, qnn, dev) if rank == 0 else None
+    comparison = None
+    if rank == 0 and world == 1:
+        qnn.encode_pack(a_bufs[0], AB, sa, 0, planes=planes[0])
+        comparison = int8_tensor_comparison(torch, qnn, dev, a_bufs[0], c.w, sa, sw, planes[0], packed, alpha)
 
     for i in range(args.warmup):
         step(i)
@@ -397,6 +443,8 @@ def run_gpu(args):
                                 "frac": enc_bytes / (enc_ms * 1e-3) / 1e9 / mp["hbm_gbs"], "peak_kind": mp_kind},
             "clocks": clocks,
         }
+        if comparison is not None:
+            line["comparison_int8_tensor"] = comparison
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg()
         print(json.dumps(line), flush=True)
