@@ -49,7 +49,7 @@ typedef enum qnn_status {
     QNN_E_ARG = -1,    /* null pointer, non-positive size, bits outside 1..8, unknown flag/layout */
     QNN_E_ALIGN = -2,  /* a plane/packed buffer is not 16-byte aligned, fp32 buffer not 4-byte aligned */
     QNN_E_RANGE = -3,  /* Kg*A*B does not fit int32, or an index does not fit the kernels' 32-bit tile arithmetic */
-    QNN_E_SCALE = -4,  /* scale or alpha not finite, or scale <= 0 */
+    QNN_E_SCALE = -4,  /* scale outside [1e-30, 1e30] (or NaN), or alpha not finite */
     QNN_E_CUDA = -5,   /* the CUDA runtime refused a launch or copy (cudaGetLastError is consumed) */
     QNN_E_DEVICE = -6  /* a kernel reported an internal error through its status word */
 } qnn_status;
@@ -80,7 +80,7 @@ size_t qnn_weights_row_words(int taps, int c_in);
  * as the look-up form of Section 3.3).
  *   x       fp32 [rows][ldx], row r starts at x + r*ldx, first k entries used (ldx >= k).
  *           For a convolution input in NHWC, rows = N*H*W and k = C.
- *   scale   grid step s = r/(2^bits - 1), finite and > 0.
+ *   scale   grid step s = r/(2^bits - 1), in [1e-30, 1e30] (QNN_E_SCALE otherwise).
  *   flags   0 or QNN_RELU.
  *   planes  out, uint32 [rows][bits][qnn_row_words(k)], fully written (padding = 0).
  *   rowsum  optional out (may be NULL), int32 [rows]: sum over the row of t = (q + 2^bits - 1)/2.

@@ -24,7 +24,9 @@
 namespace qnn_tiled {
 
 constexpr int kBN = 64, kThreads = 256;
-template <int AB> struct TileM { static constexpr int TM = (AB <= 2) ? 4 : 2, BM = 16 * TM; };
+// default rows per thread: 4 (BM = 64) for ab <= 2, 2 (BM = 32) for ab = 3, 4; ab <= 2 also has a TM = 2
+// instantiation, used when halving the tile fills the SMs' CTA slots more evenly.
+template <int AB> struct TileM { static constexpr int TM = (AB <= 2) ? 4 : 2; };
 constexpr int kStageChunks = 2;                   // groups of 8 words per stage
 constexpr int kStageWords = 8 * kStageChunks;     // words per (row, plane) per stage
 
@@ -106,9 +108,9 @@ __device__ __forceinline__ void pair8(const uint32_t (&ta)[8], const uint32_t (&
     acc += __popc(fours) * (4 << shift);
 }
 
-template <int AB, int WB, bool CONV>
+template <int AB, int WB, bool CONV, int TM>
 __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p) {
-    constexpr int TM = TileM<AB>::TM, kBM = TileM<AB>::BM;
+    constexpr int kBM = 16 * TM;
     constexpr int A_UNITS = kBM * AB * kStageChunks;      // (row, plane, group) units per stage
     constexpr int W_UNITS = kBN * WB * kStageChunks;
     constexpr int A_VEC = kStageChunks * 2 * AB * kBM;    // uint4 per stage, A region
@@ -441,13 +443,13 @@ static __global__ void __launch_bounds__(kThreads, 2) probe_csa73_kernel(int ite
 }
 constexpr double kProbeCsa73WordsPerThreadIter = 8.0 * kStageChunks * 4 * 4 * 2 * 2;
 
-template <int AB, int WB, bool CONV>
-inline int launch_tiled(const Params &p, cudaStream_t st) {
-    constexpr int kBM = TileM<AB>::BM;
+template <int AB, int WB, bool CONV, int TM>
+inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
+    constexpr int kBM = 16 * TM;
     constexpr size_t smem = 2u * kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u;
     if (smem > 48u * 1024u &&
-        cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess)
+        cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV, TM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem) != cudaSuccess)
         return QNN_E_CUDA;
     Params q = p;
     const int64_t tiles_m = (q.Mg + kBM - 1) / kBM, tiles_n = (q.Ng + kBN - 1) / kBN;
@@ -455,17 +457,40 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
     q.tiles_m = (int)tiles_m;
     q.ntiles = (int)(tiles_m * tiles_n);
     set_k_split(q);
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return QNN_E_CUDA;
     // Short reductions: two persistent CTAs per SM walk the tiles and prefetch across tile boundaries, which
     // hides the first-stage latency that would otherwise dominate.  Long reductions: one CTA per tile measured
     // about 5% faster (the hardware's dynamic block placement balances better than the static walk).
     const bool persistent = q.nstages <= 3;
     const int grid = (persistent && q.ntiles > 2 * sms) ? 2 * sms : q.ntiles;
-    bgemm_tiled_kernel<AB, WB, CONV><<<grid, kThreads, smem, st>>>(q);
+    bgemm_tiled_kernel<AB, WB, CONV, TM><<<grid, kThreads, smem, st>>>(q);
     return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA;
+}
+
+// Share of the SMs' time spent on useful work when `tiles` equal tiles are handed out dynamically: an SM
+// works through its tiles at the same rate whether one or two CTAs are resident, so the makespan is
+// ceil(tiles / sms) tile-times.
+inline double wave_efficiency(int64_t tiles, int64_t sms) {
+    const int64_t rounds = (tiles + sms - 1) / sms;
+    return (double)tiles / (double)(rounds * sms);
+}
+
+template <int AB, int WB, bool CONV>
+inline int launch_tiled(const Params &p, cudaStream_t st) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return QNN_E_CUDA;
+    if constexpr (AB <= 2) {
+        // 64-row tiles reuse each weight word for four rows per thread; 32-row tiles measured ~5% slower per
+        // operation but give twice as many tiles.  Take them only when that fills the SMs better (small problems).
+        const int64_t tn = (p.Ng + kBN - 1) / kBN;
+        const int64_t t64 = ((p.Mg + 63) / 64) * tn, t32 = ((p.Mg + 31) / 32) * tn;
+        if (wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
+            return launch_tiled_tm<AB, WB, CONV, 2>(p, sms, st);
+        return launch_tiled_tm<AB, WB, CONV, 4>(p, sms, st);
+    } else {
+        return launch_tiled_tm<AB, WB, CONV, 2>(p, sms, st);
+    }
 }
 
 template <bool CONV>

@@ -16,13 +16,12 @@ constexpr int kEncThreads = 256;
 // (NHWC activations with few channels) a unit spans RPU = 2 (k <= 64) or 4 (k <= 32) whole rows so
 // that the lanes stay busy.  UN units are loaded before the first ballot, so 4*UN independent
 // 128-byte requests per warp are in flight.  Unit indices advance incrementally (no division in the loop).
-template <int BITS, int UN, int RPU>
+template <int BITS, int UN, int RPU, bool FULL>
 __global__ void __launch_bounds__(kEncThreads)
-encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, float lo,
+encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, float lo, float hi,
                    uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum, int groups_per_row, int segs_per_row,
                    int kw, int64_t first_row_step, int first_grp_step) {
     const float half = (float)(1 << (BITS - 1));
-    constexpr int amax = (1 << BITS) - 1;
     constexpr int SPAN = 128 / RPU;                       // elements of one row inside a unit (RPU > 1)
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = ((int64_t)blockIdx.x * kEncThreads + threadIdx.x) >> 5;
@@ -46,7 +45,7 @@ encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx
                     kk = (32 * j) % SPAN + lane;
                 }
                 const bool live = (RPU == 1) ? ((grp * UN + q) < segs_per_row) : (row < rows);
-                v[q][j] = (live && kk < k) ? __ldcs(x + row * ldx + kk) : 0.0f;
+                v[q][j] = (live && (FULL || kk < k)) ? __ldcs(x + row * ldx + kk) : 0.0f;
             }
         }
 #pragma unroll
@@ -57,8 +56,8 @@ encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int kk = (RPU == 1) ? seg * 128 + 32 * j + lane : (32 * j) % SPAN + lane;
-                const int code = qnn_code_t(v[q][j], inv2s, half, amax, lo);
-                t[j] = (kk < k) ? code : 0;                                        // padding bits are 0
+                const int code = qnn_code_t(v[q][j], inv2s, half, lo, hi);
+                t[j] = (FULL || kk < k) ? code : 0;                                // padding bits are 0
             }
             uint32_t b[BITS][4];
 #pragma unroll
@@ -66,9 +65,9 @@ encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx
 #pragma unroll
                 for (int j = 0; j < 4; ++j) b[i][j] = __ballot_sync(0xffffffffu, t[j] & (1 << i));
             if (RPU == 1) {
-                uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+                uint4 mine = make_uint4(b[0][0], b[0][1], b[0][2], b[0][3]);
 #pragma unroll
-                for (int i = 0; i < BITS; ++i)
+                for (int i = 1; i < BITS; ++i)
                     if (lane == i) mine = make_uint4(b[i][0], b[i][1], b[i][2], b[i][3]);
                 if (lane < BITS)
                     *reinterpret_cast<uint4 *>(planes + (ru * BITS + lane) * (int64_t)kw + seg * 4) = mine;
@@ -116,10 +115,9 @@ encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx
 // covers 32 input channels of one tap; the source index follows the layout flag.
 template <int BITS>
 __global__ void __launch_bounds__(kEncThreads)
-pack_weights_kernel(const float *__restrict__ w, int n_out, int taps, int c_in, int layout, float inv2s,
-                    uint32_t *__restrict__ planes, int kw, int cw) {
+pack_weights_kernel(const float *__restrict__ w, int n_out, int taps, int c_in, int layout, float inv2s, float lo,
+                    float hi, uint32_t *__restrict__ planes, int kw, int cw) {
     const float half = (float)(1 << (BITS - 1));
-    constexpr int amax = (1 << BITS) - 1;
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = ((int64_t)blockIdx.x * kEncThreads + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * kEncThreads) >> 5;
@@ -140,7 +138,7 @@ pack_weights_kernel(const float *__restrict__ w, int n_out, int taps, int c_in, 
                 if (layout == QNN_W_NTC) idx = ((int64_t)n * taps + tap) * c_in + c;
                 else if (layout == QNN_W_TCN) idx = ((int64_t)tap * c_in + c) * n_out + n;
                 else idx = ((int64_t)n * c_in + c) * taps + tap;
-                t[j] = qnn_code_t(w[idx], inv2s, half, amax, -INFINITY);
+                t[j] = qnn_code_t(w[idx], inv2s, half, lo, hi);
             }
         }
         uint4 mine = make_uint4(0u, 0u, 0u, 0u);
@@ -198,15 +196,17 @@ int grid_for(int64_t warps_needed) {
 }
 
 template <int BITS>
-void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float inv2s, bool relu, uint32_t *planes,
+void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale, bool relu, uint32_t *planes,
                    int32_t *rowsum, cudaStream_t st) {
     constexpr int UN = 4;
-    const float lo = relu ? 0.0f : -INFINITY;
+    const float inv2s = 1.0f / (2.0f * scale);
+    float lo, hi;
+    qnn_clamp_bounds(BITS, scale, relu, &lo, &hi);
     const int kw = (int)qnn_row_words_i(k);
     const int segs = kw / 4;
     int groups;
     int64_t total;                                   // warp-level work items
-    const int rpu = (k <= 32 && 4 * BITS <= 32) ? 4 : (k <= 64 ? 2 : 1);
+    const int rpu = (k <= 32) ? 4 : (k <= 64 ? 2 : 1);
     if (rpu == 1) {
         groups = (int)qnn_ceil_div(segs, UN);
         total = rows * groups;
@@ -218,24 +218,29 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float inv2s
     const int64_t nwarps = (int64_t)grid * (kEncThreads / 32);
     const int64_t row_step = nwarps / groups;
     const int grp_step = (int)(nwarps % groups);
-    if (rpu == 1)
-        encode_pack_kernel<BITS, UN, 1><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, planes, rowsum, groups,
-                                                                    segs, kw, row_step, grp_step);
-    else if (rpu == 2)
-        encode_pack_kernel<BITS, UN, 2><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, planes, rowsum, groups,
-                                                                    segs, kw, row_step, grp_step);
-    else
-        encode_pack_kernel<BITS, UN, 4><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, planes, rowsum, groups,
-                                                                    segs, kw, row_step, grp_step);
+#define QNN_ENC(RPU_, FULL_)                                                                                       \
+    encode_pack_kernel<BITS, UN, RPU_, FULL_><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, hi, planes, \
+                                                                           rowsum, groups, segs, kw, row_step, grp_step)
+    if (rpu == 1) {
+        if (k % 128 == 0) QNN_ENC(1, true); else QNN_ENC(1, false);
+    } else if (rpu == 2) {
+        if (k == 64) QNN_ENC(2, true); else QNN_ENC(2, false);
+    } else {
+        if (k == 32) QNN_ENC(4, true); else QNN_ENC(4, false);
+    }
+#undef QNN_ENC
 }
 
 template <int BITS>
-void launch_pack_w(const float *w, int n_out, int taps, int c_in, int layout, float inv2s, uint32_t *planes,
+void launch_pack_w(const float *w, int n_out, int taps, int c_in, int layout, float scale, uint32_t *planes,
                    cudaStream_t st) {
     const int kw = (int)qnn_w_row_words_i(taps, c_in);
     const int cw = (c_in + 31) / 32;
+    const float inv2s = 1.0f / (2.0f * scale);
+    float lo, hi;
+    qnn_clamp_bounds(BITS, scale, false, &lo, &hi);
     pack_weights_kernel<BITS><<<grid_for((int64_t)n_out * (kw / 4)), kEncThreads, 0, st>>>(w, n_out, taps, c_in, layout,
-                                                                                      inv2s, planes, kw, cw);
+                                                                                      inv2s, lo, hi, planes, kw, cw);
 }
 
 }  // namespace
@@ -255,15 +260,14 @@ void launch_pack_w(const float *w, int n_out, int taps, int c_in, int layout, fl
 extern "C" int qnn_encode_pack(const float *x, int64_t rows, int k, int64_t ldx, int bits, float scale,
                                unsigned flags, uint32_t *planes, int32_t *rowsum, void *stream) {
     if (!x || !planes || rows <= 0 || k <= 0 || ldx < k || !qnn_bits_ok(bits) || (flags & ~QNN_RELU)) return QNN_E_ARG;
-    if (!(scale > 0.0f) || !isfinite(scale)) return QNN_E_SCALE;
+    if (!(scale >= 1e-30f) || !(scale <= 1e30f)) return QNN_E_SCALE;   // also rejects NaN, 0, negatives, infinities
     if (!qnn_aligned(planes, 16) || !qnn_aligned(x, 4) || (rowsum && !qnn_aligned(rowsum, 4))) return QNN_E_ALIGN;
     if (k > (1 << 30) || rows > ((int64_t)1 << 40)) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const float inv2s = 1.0f / (2.0f * scale);
     const bool relu = (flags & QNN_RELU) != 0;
     if (rowsum && k > 64 && cudaMemsetAsync(rowsum, 0, (size_t)rows * sizeof(int32_t), st) != cudaSuccess)
         return QNN_E_CUDA;
-#define CALL(B) launch_encode<B>(x, rows, k, ldx, inv2s, relu, planes, rowsum, st)
+#define CALL(B) launch_encode<B>(x, rows, k, ldx, scale, relu, planes, rowsum, st)
     QNN_DISPATCH_BITS(bits, CALL)
 #undef CALL
     return qnn_launch_status();
@@ -273,15 +277,14 @@ extern "C" int qnn_pack_weights(const float *w, int n_out, int taps, int c_in, i
                                 void *packed, void *stream) {
     if (!w || !packed || n_out <= 0 || taps <= 0 || c_in <= 0 || !qnn_bits_ok(bits)) return QNN_E_ARG;
     if (layout != QNN_W_NTC && layout != QNN_W_TCN && layout != QNN_W_NCT) return QNN_E_ARG;
-    if (!(scale > 0.0f) || !isfinite(scale)) return QNN_E_SCALE;
+    if (!(scale >= 1e-30f) || !(scale <= 1e30f)) return QNN_E_SCALE;   // also rejects NaN, 0, negatives, infinities
     if (!qnn_aligned(packed, 16) || !qnn_aligned(w, 4)) return QNN_E_ALIGN;
     const int64_t kw = qnn_w_row_words_i(taps, c_in);
     if (kw > (1 << 26) || (int64_t)n_out * bits * kw > ((int64_t)1 << 40)) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const float inv2s = 1.0f / (2.0f * scale);
     uint32_t *planes = static_cast<uint32_t *>(packed);
     int32_t *tapsum = reinterpret_cast<int32_t *>(planes + (int64_t)n_out * bits * kw);
-#define CALL(B) launch_pack_w<B>(w, n_out, taps, c_in, layout, inv2s, planes, st)
+#define CALL(B) launch_pack_w<B>(w, n_out, taps, c_in, layout, scale, planes, st)
     QNN_DISPATCH_BITS(bits, CALL)
 #undef CALL
     if (cudaGetLastError() != cudaSuccess) return QNN_E_CUDA;

@@ -17,16 +17,25 @@ static inline int64_t qnn_w_row_words_i(int taps, int c_in) {
 static inline int qnn_launch_status() { return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA; }
 
 // Unsigned code t in [0, 2^bits - 1] of a real value (odd code q = 2t - (2^bits - 1)).
-// inv2s = 1/(2*scale), half = 2^(bits-1), amax = 2^bits - 1, lo = 0 for a fused ReLU else -inf.
+// inv2s = 1/(2*scale), half = 2^(bits-1); [lo, hi] is a pre-clamp of x (see qnn_clamp_bounds).
 // v = x/(2s) + 2^(b-1) with one fused multiply-add; t = floor(v) for x > 0 and ceil(v) - 1 otherwise,
 // so that a value half-way between two codes moves away from zero and 0 maps to q = -1.
-// ceil(v) - 1 = -floor(-v) - 1 = ~floor(-v): one saturating float->int conversion (round down)
-// serves both branches; NaN converts to 0 and ends at t = 0, infinities saturate and are clamped.
-__device__ __forceinline__ int qnn_code_t(float x, float inv2s, float half, int amax, float lo) {
-    x = fmaxf(x, lo);
+// ceil(v) - 1 = -floor(-v) - 1 = ~floor(-v): one float->int conversion (round down) serves both branches.
+__device__ __forceinline__ int qnn_code_t(float x, float inv2s, float half, float lo, float hi) {
+    x = fminf(fmaxf(x, lo), hi);          // NaN -> lo; no integer clamp is needed afterwards
     const float v = __fmaf_rn(x, inv2s, half);
     const bool pos = x > 0.0f;
     const int f = __float2int_rd(pos ? v : -v);
-    const int t = pos ? f : ~f;
-    return min(max(t, 0), amax);
+    return pos ? f : ~f;
+}
+
+// Pre-clamp bounds that make the integer clamp of the code unnecessary.  hi = 2^bits * scale * (1 - 2^-10)
+// lies between the range end r = (2^bits - 1) * scale and the point where v would reach 2^bits, with a margin
+// (2^-11 relative) far above the rounding of inv2s and of the multiply-add: every x in [r, hi] gives
+// floor(v) = 2^bits - 1 and every x in [-hi, -r] gives ceil(v) - 1 = 0, exactly the end codes that the
+// unclamped formula followed by a clamp of t produces for any |x| >= r.  lo = -hi, or 0 for a fused ReLU
+// (also what a NaN input turns into, matching max(NaN, 0) = 0 and NaN -> most negative code).
+static inline void qnn_clamp_bounds(int bits, float scale, bool relu, float *lo, float *hi) {
+    *hi = (float)(1 << bits) * scale * (1.0f - 0.0009765625f);
+    *lo = relu ? 0.0f : -*hi;
 }
