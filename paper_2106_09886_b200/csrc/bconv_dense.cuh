@@ -1,0 +1,147 @@
+// Convolutions whose whole patch fits one 32-bit word per plane (R*S*C <= 32, e.g. a 3x3 first layer on
+// 3 channels: 27 bits).  The plane storage keeps every tap on a word boundary, so the general kernel would
+// spend a full word operation per tap on C useful bits.  Here the patch word of an output pixel is assembled on
+// the fly, bit (tap*C + c), from the taps' plane words (implicit im2col at bit granularity), and the same is
+// done once per CTA for the weights.
+//
+// Mapping: lane <-> output feature (32 consecutive features per pass), so every store is one coalesced
+// 128-byte row segment; a warp takes 32 output pixels at a time, lane L assembles pixel L's ab patch words,
+// and the pixels' words are then handed round with shuffles.  Per output: ab*wb (xor, popc, multiply-add).
+// Taps outside the image are left as zero bits and corrected with tapsum exactly as in the tiled kernel.
+#pragma once
+#include "qnn_internal.cuh"
+
+namespace qnn_dense {
+
+constexpr int kThreads = 256;
+
+struct Params {
+    const uint32_t *a;
+    const uint32_t *w;
+    const int32_t *tapsum;   // [Ng][taps]
+    int64_t Mg;
+    int Ng;
+    int a_pitch, w_pitch;
+    float alpha;
+    float *out;
+    int32_t *acc;
+    int H, W, C, R, S, stride, pad, Ho, Wo;
+};
+
+template <int AB, int WB>
+__global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) {
+    extern __shared__ uint32_t smem_u32[];
+    const int taps = p.R * p.S;
+    uint32_t *wd_s = smem_u32;                                          // [WB][Ng] dense weight words
+    int32_t *ts_s = reinterpret_cast<int32_t *>(smem_u32 + WB * p.Ng);  // [taps][Ng]
+    for (int idx = threadIdx.x; idx < WB * p.Ng; idx += kThreads) {
+        const int j = idx / p.Ng, n = idx - j * p.Ng;
+        const uint32_t *src = p.w + ((int64_t)n * WB + j) * p.w_pitch;
+        uint32_t word = 0;
+        for (int t = 0; t < taps; ++t) word |= src[t] << (t * p.C);
+        wd_s[idx] = word;
+    }
+    for (int idx = threadIdx.x; idx < taps * p.Ng; idx += kThreads) {
+        const int t = idx / p.Ng, n = idx - t * p.Ng;
+        ts_s[idx] = p.tapsum[(int64_t)n * taps + t];
+    }
+    __syncthreads();
+
+    constexpr int AMAX = (1 << AB) - 1, PROD = AMAX * ((1 << WB) - 1);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * kThreads) >> 5;
+    const int64_t nbatches = (p.Mg + 31) / 32;
+    const int ncb = (p.Ng + 31) / 32;
+
+    for (int64_t batch = warp0; batch < nbatches; batch += nwarps) {
+        // ---- lane assembles the patch words of output pixel m = batch*32 + lane
+        const int64_t m = batch * 32 + lane;
+        uint32_t mine[AB];
+#pragma unroll
+        for (int i = 0; i < AB; ++i) mine[i] = 0u;
+        uint32_t invalid = 0u;                                           // bit t set: tap t lies outside the image
+        if (m < p.Mg) {
+            const int wo = (int)(m % p.Wo);
+            const int ho = (int)((m / p.Wo) % p.Ho);
+            const int64_t n_img = m / ((int64_t)p.Wo * p.Ho);
+            const int h0 = ho * p.stride - p.pad, w0 = wo * p.stride - p.pad;
+            int t = 0;
+            for (int r = 0; r < p.R; ++r)
+                for (int s = 0; s < p.S; ++s, ++t) {
+                    const int hi = h0 + r, wi = w0 + s;
+                    if (hi >= 0 && hi < p.H && wi >= 0 && wi < p.W) {
+                        const uint32_t *src = p.a + ((n_img * p.H + hi) * p.W + wi) * (int64_t)(AB * p.a_pitch);
+#pragma unroll
+                        for (int i = 0; i < AB; ++i) mine[i] |= __ldg(src + i * p.a_pitch) << (t * p.C);
+                    } else {
+                        invalid |= 1u << t;
+                    }
+                }
+        }
+        const int rows_here = (int)((p.Mg - batch * 32) < 32 ? (p.Mg - batch * 32) : 32);
+        for (int cb = 0; cb < ncb; ++cb) {
+            const int n = cb * 32 + lane;
+            const bool n_ok = n < p.Ng;
+            uint32_t wreg[WB];
+#pragma unroll
+            for (int j = 0; j < WB; ++j) wreg[j] = n_ok ? wd_s[j * p.Ng + n] : 0u;
+            for (int rr = 0; rr < rows_here; ++rr) {
+                int s_acc = 0;
+#pragma unroll
+                for (int i = 0; i < AB; ++i) {
+                    const uint32_t ai = __shfl_sync(0xffffffffu, mine[i], rr);
+#pragma unroll
+                    for (int j = 0; j < WB; ++j) s_acc += __popc(ai ^ wreg[j]) * (1 << (i + j));
+                }
+                uint32_t inv = __shfl_sync(0xffffffffu, invalid, rr);
+                int n_valid = (taps - __popc(inv)) * p.C;
+                int corr = 0;
+                while (inv != 0u) {                                       // warp-uniform: the row is the same for all lanes
+                    const int t = __ffs(inv) - 1;
+                    inv &= inv - 1u;
+                    if (n_ok) corr += ts_s[t * p.Ng + n];
+                }
+                if (n_ok) {
+                    const int32_t v = n_valid * PROD - 2 * (s_acc - AMAX * corr);
+                    const int64_t o = (batch * 32 + rr) * (int64_t)p.Ng + n;
+                    if (p.acc) p.acc[o] = v;
+                    if (p.out) p.out[o] = __fmul_rn(__int2float_rn(v), p.alpha);
+                }
+            }
+        }
+    }
+}
+
+template <int AB, int WB>
+inline int launch_dense1(const Params &p, cudaStream_t st) {
+    const size_t smem = ((size_t)WB * p.Ng + (size_t)p.R * p.S * p.Ng) * 4u;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return QNN_E_CUDA;
+    const int64_t nbatches = (p.Mg + 31) / 32;
+    int64_t blocks = (nbatches + kThreads / 32 - 1) / (kThreads / 32);
+    if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+    bconv_dense1_kernel<AB, WB><<<(int)blocks, kThreads, smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA;
+}
+
+// usable when the patch fits one word and the per-CTA tables fit the default shared memory
+inline bool dense1_applicable(int ab, int wb, int R, int S, int C, int Cout) {
+    return ab <= 4 && wb <= 4 && (int64_t)R * S * C <= 32 && C < 32 &&
+           ((int64_t)wb * Cout + (int64_t)R * S * Cout) * 4 <= 40 * 1024;
+}
+
+inline int dispatch_dense1(int ab, int wb, const Params &p, cudaStream_t st) {
+#define QNN_D(A_, W_) \
+    if (ab == A_ && wb == W_) return launch_dense1<A_, W_>(p, st);
+    QNN_D(1, 1) QNN_D(1, 2) QNN_D(1, 3) QNN_D(1, 4)
+    QNN_D(2, 1) QNN_D(2, 2) QNN_D(2, 3) QNN_D(2, 4)
+    QNN_D(3, 1) QNN_D(3, 2) QNN_D(3, 3) QNN_D(3, 4)
+    QNN_D(4, 1) QNN_D(4, 2) QNN_D(4, 3) QNN_D(4, 4)
+#undef QNN_D
+    return QNN_E_ARG;
+}
+
+}  // namespace qnn_dense

@@ -2,6 +2,7 @@
 // the 2^(i+j) combine and the scale, in one launch.
 #include "qnn_internal.cuh"
 #include "bgemm_tiled.cuh"
+#include "bconv_dense.cuh"
 
 namespace {
 
@@ -131,6 +132,15 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
     if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
+    if (qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout)) {
+        qnn_dense::Params d = {};
+        d.a = a_planes; d.w = w;
+        d.tapsum = reinterpret_cast<const int32_t *>(w + (int64_t)Cout * wb * g.w_pitch);
+        d.Mg = Mg; d.Ng = Cout; d.a_pitch = g.a_pitch; d.w_pitch = g.w_pitch;
+        d.alpha = alpha; d.out = out; d.acc = acc;
+        d.H = H; d.W = W; d.C = C; d.R = R; d.S = S; d.stride = stride; d.pad = pad; d.Ho = g.Ho; d.Wo = g.Wo;
+        return qnn_dense::dispatch_dense1(ab, wb, d, st);
+    }
     // the tiled kernel divides by cw and S with a 20-bit multiply-shift: exact while kwords*cw and taps*S < 2^20
     if (ab <= 4 && wb <= 4 && (int64_t)R * S * g.cw * g.cw < (1 << 20) && (int64_t)R * S * S < (1 << 20) &&
         (int64_t)R * S * g.cw < 4096) {
