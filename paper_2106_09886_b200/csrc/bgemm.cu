@@ -20,33 +20,9 @@ __device__ __forceinline__ void store_out(float *out, int64_t ldo, int32_t *acc,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Generic path (any ab, wb in 1..8): one thread per output.  Used for bit widths that have no
-// tiled specialisation; correct for every shape, not tuned.
+// Fallback convolution (any ab, wb in 1..8): one thread per output.  Only used for geometries outside the
+// tiled kernel's index arithmetic (more than 4095 reduction words per plane, very wide kernels); not tuned.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-bgemm_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__restrict__ w, int wb, int64_t Mg, int Ng,
-                     int Kg, int kw, float alpha, float *__restrict__ out, int64_t ldo, int32_t *__restrict__ acc) {
-    const int n = blockIdx.x * 16 + (threadIdx.x & 15);
-    const int64_t m = (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
-    if (n >= Ng || m >= Mg) return;
-    const uint4 *arow = reinterpret_cast<const uint4 *>(a + m * ab * (int64_t)kw);
-    const uint4 *wrow = reinterpret_cast<const uint4 *>(w + (int64_t)n * wb * kw);
-    const int kq = kw / 4;
-    int32_t s = 0;
-    for (int i = 0; i < ab; ++i) {
-        for (int j = 0; j < wb; ++j) {
-            int32_t x = 0;
-            for (int q = 0; q < kq; ++q) {
-                uint4 av = arow[i * kq + q], wv = wrow[j * kq + q];
-                x += __popc(av.x ^ wv.x) + __popc(av.y ^ wv.y) + __popc(av.z ^ wv.z) + __popc(av.w ^ wv.w);
-            }
-            s += x << (i + j);
-        }
-    }
-    const int32_t AB = ((1 << ab) - 1) * ((1 << wb) - 1);
-    store_out(out, ldo, acc, m, n, Ng, Kg * AB - 2 * s, alpha);
-}
-
 __global__ void __launch_bounds__(256)
 bconv_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__restrict__ w, int wb, ConvGeom g,
                      float alpha, float *__restrict__ out, int32_t *__restrict__ acc) {
@@ -91,22 +67,16 @@ extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed,
         return QNN_E_ALIGN;
     const int64_t AB = (int64_t)((1 << ab) - 1) * ((1 << wb) - 1);
     if ((int64_t)Kg * AB >= ((int64_t)1 << 31)) return QNN_E_RANGE;
-    if (Mg > ((int64_t)1 << 31) - 1 || qnn_ceil_div(Mg, 16) > 65535 * (int64_t)16) return QNN_E_RANGE;
+    if (Mg > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int kw = (int)qnn_row_words_i(Kg);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    if (ab <= 4 && wb <= 4) {
-        qnn_tiled::Params p = {};
-        p.a = a_planes; p.w = w; p.tapsum = nullptr;
-        p.Mg = Mg; p.Ng = Ng;
-        p.a_pitch = kw; p.w_pitch = kw; p.kwords = kw;
-        p.n_elems = Kg; p.alpha = alpha; p.out = out; p.ldo = ldo; p.acc = acc;
-        return qnn_tiled::dispatch_tiled<false>(ab, wb, p, st);
-    }
-    dim3 grid((unsigned)qnn_ceil_div(Ng, 16), (unsigned)qnn_ceil_div(Mg, 16));
-    if (grid.y > 65535) return QNN_E_RANGE;
-    bgemm_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, Mg, Ng, Kg, kw, alpha, out, ldo, acc);
-    return qnn_launch_status();
+    qnn_tiled::Params p = {};
+    p.a = a_planes; p.w = w; p.tapsum = nullptr;
+    p.Mg = Mg; p.Ng = Ng;
+    p.a_pitch = kw; p.w_pitch = kw; p.kwords = kw;
+    p.n_elems = Kg; p.alpha = alpha; p.out = out; p.ldo = ldo; p.acc = acc;
+    return qnn_tiled::dispatch_tiled(false, ab, wb, p, st);
 }
 
 extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
@@ -142,7 +112,7 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
         return qnn_dense::dispatch_dense1(ab, wb, d, st);
     }
     // the tiled kernel divides by cw and S with a 20-bit multiply-shift: exact while kwords*cw and taps*S < 2^20
-    if (ab <= 4 && wb <= 4 && (int64_t)R * S * g.cw * g.cw < (1 << 20) && (int64_t)R * S * S < (1 << 20) &&
+    if ((int64_t)R * S * g.cw * g.cw < (1 << 20) && (int64_t)R * S * S < (1 << 20) &&
         (int64_t)R * S * g.cw < 4096) {
         qnn_tiled::Params p = {};
         p.a = a_planes; p.w = w;
@@ -154,7 +124,7 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
         p.n_elems = R * S * C; p.alpha = alpha; p.out = out; p.ldo = Cout; p.acc = acc;
         p.H = H; p.W = W; p.C = C; p.R = R; p.S = S; p.stride = stride; p.pad = pad; p.Ho = g.Ho; p.Wo = g.Wo;
         p.cw = g.cw; p.piece = (g.cw % 4 == 0) ? 4 : ((g.cw % 2 == 0) ? 2 : 1);
-        return qnn_tiled::dispatch_tiled<true>(ab, wb, p, st);
+        return qnn_tiled::dispatch_tiled(true, ab, wb, p, st);
     }
     dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
     if (grid.y > 65535) return QNN_E_RANGE;

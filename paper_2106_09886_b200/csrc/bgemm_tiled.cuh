@@ -1,4 +1,4 @@
-// Tiled xor+popcount contraction for ab, wb in 1..4 (FC and implicit-im2col convolution).
+// Tiled xor+popcount contraction for ab, wb in 1..8 (FC and implicit-im2col convolution).
 //
 // Persistent CTAs (two per SM) walk over output tiles; the first stage of the next tile is copied
 // while the last stage of the current one is computed and written out.
@@ -24,9 +24,10 @@
 namespace qnn_tiled {
 
 constexpr int kBN = 64, kThreads = 256;
-// default rows per thread: 4 (BM = 64) for ab <= 2, 2 (BM = 32) for ab = 3, 4; ab <= 2 also has a TM = 2
+// default rows per thread: 4 (BM = 64) for ab <= 2, 2 (BM = 32) for ab = 3, 4, 1 (BM = 16) for ab >= 5 (so that
+// TM*ab*8 operand words never exceed 64 registers); ab <= 2 also has a TM = 2
 // instantiation, used when halving the tile fills the SMs' CTA slots more evenly.
-template <int AB> struct TileM { static constexpr int TM = (AB <= 2) ? 4 : 2; };
+template <int AB> struct TileM { static constexpr int TM = (AB <= 2) ? 4 : (AB <= 4 ? 2 : 1); };
 constexpr int kStageChunks = 2;                   // groups of 8 words per stage
 constexpr int kStageWords = 8 * kStageChunks;     // words per (row, plane) per stage
 
@@ -120,8 +121,9 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
     const int tx = tid & 15, ty = tid >> 4;
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
     // staging: unit u = tid + 256*q  ->  row = tid % BM (A) or tid % 64 (W) for every q; the A operand has
-    // at most one unit per thread and stage, the W operand at most two.
-    static_assert(A_UNITS <= kThreads && W_UNITS <= 2 * kThreads, "staging map");
+    // at most one unit per thread and stage, the W operand at most four.
+    constexpr int W_Q = (W_UNITS + kThreads - 1) / kThreads;   // W units per thread and stage (1..4)
+    static_assert(A_UNITS <= kThreads && W_Q <= 4, "staging map");
     const int srow = tid % kBM, wrow = tid % kBN;
     const int ngroups = p.nfull + (p.ntail > 0 ? 1 : 0);
     const bool a_unit = tid < A_UNITS;
@@ -131,7 +133,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
     // Per-tile source bookkeeping of this thread's units.
     struct TileSrc {
         const uint32_t *a;      // FC: start of this thread's (row, plane) words; conv: unused
-        const uint32_t *w[2];   // start of this thread's (feature, plane) words, per unit
+        const uint32_t *w[W_Q]; // start of this thread's (feature, plane) words, per unit
         int64_t pixbase;        // conv: n*H*W of the row's image
         int h0, w0;             // conv: top-left input coordinate of the row's window
         bool a_ok, w_ok;
@@ -155,7 +157,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             t.pixbase = n * p.H * p.W;
         }
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+        for (int q = 0; q < W_Q; ++q) {
             const int u = tid + q * kThreads;
             const int plane = (u % (kBN * WB)) / kBN;
             t.w[q] = p.w + ((int64_t)(t.w_ok ? n0 + wrow : 0) * WB + plane) * p.w_pitch;
@@ -489,20 +491,43 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
             return launch_tiled_tm<AB, WB, CONV, 2>(p, sms, st);
         return launch_tiled_tm<AB, WB, CONV, 4>(p, sms, st);
     } else {
-        return launch_tiled_tm<AB, WB, CONV, 2>(p, sms, st);
+        return launch_tiled_tm<AB, WB, CONV, TileM<AB>::TM>(p, sms, st);
     }
 }
 
-template <bool CONV>
-inline int dispatch_tiled(int ab, int wb, const Params &p, cudaStream_t st) {
-#define QNN_T(A_, W_) \
-    if (ab == A_ && wb == W_) return launch_tiled<A_, W_, CONV>(p, st);
-    QNN_T(1, 1) QNN_T(1, 2) QNN_T(1, 3) QNN_T(1, 4)
-    QNN_T(2, 1) QNN_T(2, 2) QNN_T(2, 3) QNN_T(2, 4)
-    QNN_T(3, 1) QNN_T(3, 2) QNN_T(3, 3) QNN_T(3, 4)
-    QNN_T(4, 1) QNN_T(4, 2) QNN_T(4, 3) QNN_T(4, 4)
+// All weight widths and both operand kinds for one activation width; each activation width is compiled in
+// its own translation unit (tiled_ab<N>.cu) so that the 100+ kernel instantiations build in parallel.
+template <int AB>
+inline int run_tiled_ab(bool conv, int wb, const Params &p, cudaStream_t st) {
+#define QNN_T(W_) \
+    case W_: return conv ? launch_tiled<AB, W_, true>(p, st) : launch_tiled<AB, W_, false>(p, st);
+    switch (wb) {
+        QNN_T(1) QNN_T(2) QNN_T(3) QNN_T(4) QNN_T(5) QNN_T(6) QNN_T(7) QNN_T(8)
+        default: return QNN_E_ARG;
+    }
 #undef QNN_T
-    return QNN_E_ARG;
+}
+int run_tiled_ab1(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab2(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab3(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab4(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab5(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab6(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab7(bool conv, int wb, const Params &p, cudaStream_t st);
+int run_tiled_ab8(bool conv, int wb, const Params &p, cudaStream_t st);
+
+inline int dispatch_tiled(bool conv, int ab, int wb, const Params &p, cudaStream_t st) {
+    switch (ab) {
+        case 1: return run_tiled_ab1(conv, wb, p, st);
+        case 2: return run_tiled_ab2(conv, wb, p, st);
+        case 3: return run_tiled_ab3(conv, wb, p, st);
+        case 4: return run_tiled_ab4(conv, wb, p, st);
+        case 5: return run_tiled_ab5(conv, wb, p, st);
+        case 6: return run_tiled_ab6(conv, wb, p, st);
+        case 7: return run_tiled_ab7(conv, wb, p, st);
+        case 8: return run_tiled_ab8(conv, wb, p, st);
+        default: return QNN_E_ARG;
+    }
 }
 
 }  // namespace qnn_tiled
