@@ -156,6 +156,19 @@ int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float s
                         uint32_t *planes_dev, float *out_dev, void *stream);
 
 /*
+ * The same layer from host memory, cut into chunks of `rows_per_chunk` activation rows that are spread
+ * round-robin over `nstreams` caller-provided streams (cudaStream_t each): chunk i is copied in, encoded,
+ * contracted and copied out on stream i % nstreams, so the two copy directions and the kernels of different
+ * chunks overlap (rows are independent).  Buffers as in qnn_fc_forward_host (each chunk uses its own row
+ * range of them).  The caller orders the streams against earlier and later work; out_host is complete once
+ * every stream has been synchronized.
+ */
+int qnn_fc_forward_host_pipelined(const float *x_host, int64_t Mg, int Kg, int ab, float scale_a, unsigned flags,
+                                  const void *w_packed, int wb, int Ng, float alpha, float *out_host, float *x_dev,
+                                  uint32_t *planes_dev, float *out_dev, int64_t rows_per_chunk, void *const *streams,
+                                  int nstreams);
+
+/*
  * One FC layer for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
  * packaging of qnn_encode_pack + qnn_bgemm, not a step of the method.)
  *

@@ -147,3 +147,33 @@ extern "C" int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int 
         return QNN_E_CUDA;
     return QNN_OK;
 }
+
+extern "C" int qnn_fc_forward_host_pipelined(const float *x_host, int64_t Mg, int Kg, int ab, float scale_a,
+                                             unsigned flags, const void *w_packed, int wb, int Ng, float alpha,
+                                             float *out_host, float *x_dev, uint32_t *planes_dev, float *out_dev,
+                                             int64_t rows_per_chunk, void *const *streams, int nstreams) {
+    if (!x_host || !out_host || !x_dev || !planes_dev || !out_dev || !streams || Mg <= 0 || Kg <= 0 || Ng <= 0)
+        return QNN_E_ARG;
+    if (nstreams < 1 || rows_per_chunk < 1 || !qnn_bits_ok(ab)) return QNN_E_ARG;
+    const int64_t plane_words_per_row = (int64_t)ab * qnn_row_words_i(Kg);
+    int64_t chunk = 0;
+    for (int64_t r0 = 0; r0 < Mg; r0 += rows_per_chunk, ++chunk) {
+        const int64_t rows = (Mg - r0 < rows_per_chunk) ? (Mg - r0) : rows_per_chunk;
+        void *stream = streams[chunk % nstreams];
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        float *xd = x_dev + r0 * Kg;
+        uint32_t *pd = planes_dev + r0 * plane_words_per_row;
+        float *od = out_dev + r0 * Ng;
+        if (cudaMemcpyAsync(xd, x_host + r0 * Kg, (size_t)rows * Kg * sizeof(float), cudaMemcpyHostToDevice, st) !=
+            cudaSuccess)
+            return QNN_E_CUDA;
+        int rc = qnn_encode_pack(xd, rows, Kg, Kg, ab, scale_a, flags, pd, nullptr, stream);
+        if (rc != QNN_OK) return rc;
+        rc = qnn_bgemm(pd, ab, w_packed, wb, rows, Ng, Kg, alpha, od, Ng, nullptr, stream);
+        if (rc != QNN_OK) return rc;
+        if (cudaMemcpyAsync(out_host + r0 * Ng, od, (size_t)rows * Ng * sizeof(float), cudaMemcpyDeviceToHost, st) !=
+            cudaSuccess)
+            return QNN_E_CUDA;
+    }
+    return QNN_OK;
+}

@@ -20,7 +20,7 @@ W_NTC, W_TCN, W_NCT = 0, 1, 2
 EXPORTS = [
     "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
-    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
+    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -54,6 +54,7 @@ def _load() -> C.CDLL:
     lib.qnn_bconv2d.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
+    lib.qnn_fc_forward_host_pipelined.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, i64, C.POINTER(C.c_void_p), i]
     lib.qnn_fc_forward_noalloc.argtypes = [p, i64, i, i64, i, f, u, p, i, i, f, p, i64, p]
     lib.qnn_probe_bitops.argtypes = [i, i, i, p, C.POINTER(C.c_double), p]
     lib.qnn_probe_copy.argtypes = [p, p, sz, p]
@@ -180,6 +181,24 @@ def fc_forward_host(x_host: torch.Tensor, ab: int, scale_a: float, flags: int, w
     _check(lib.qnn_fc_forward_host(_ptr(x_host), Mg, Kg, ab, float(scale_a), flags, _ptr(w_packed), wb, Ng,
                                    float(alpha), _ptr(out_host), _ptr(x_dev), _ptr(planes_dev), _ptr(out_dev),
                                    _stream(stream)), "qnn_fc_forward_host")
+    return out_host
+
+
+def fc_forward_host_pipelined(x_host: torch.Tensor, ab: int, scale_a: float, flags: int, w_packed: torch.Tensor, wb: int,
+                              Ng: int, alpha: float, out_host: torch.Tensor, x_dev: torch.Tensor,
+                              planes_dev: torch.Tensor, out_dev: torch.Tensor, rows_per_chunk: int, streams) -> torch.Tensor:
+    """Row-chunked FC layer from pinned host memory over several torch streams.  The streams are made to wait
+    for the current stream first, and the current stream waits for all of them afterwards."""
+    Mg, Kg = x_host.shape
+    cur = torch.cuda.current_stream()
+    for s in streams:
+        s.wait_stream(cur)
+    arr = (C.c_void_p * len(streams))(*[s.cuda_stream for s in streams])
+    _check(lib.qnn_fc_forward_host_pipelined(_ptr(x_host), Mg, Kg, ab, float(scale_a), flags, _ptr(w_packed), wb, Ng,
+                                             float(alpha), _ptr(out_host), _ptr(x_dev), _ptr(planes_dev), _ptr(out_dev),
+                                             rows_per_chunk, arr, len(streams)), "qnn_fc_forward_host_pipelined")
+    for s in streams:
+        cur.wait_stream(s)
     return out_host
 
 

@@ -139,3 +139,25 @@ def test_fc_forward_host_matches_oracle():
     qnn.fc_forward_host(x_host, 2, sa, 0, packed, 2, 200, alpha, out_host, x_dev, planes, out_dev)
     torch.cuda.synchronize()
     assert_fp32_close(out_host.numpy(), out)
+
+
+def test_fc_forward_host_pipelined_matches_oracle():
+    """Row chunks spread over three streams (ragged last chunk) give the same result as the oracle."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(22)
+    a = np.abs(rng.standard_normal((1000, 700))).astype(np.float32)
+    w = (0.02 * rng.standard_normal((130, 700))).astype(np.float32)
+    sa, sw, alpha = scales_for(a, w, 3, 2)
+    _, _, acc, out = oracle_fc(a, w, False, 3, 2, sa, sw, alpha)
+    packed = qnn.pack_weights(torch.from_numpy(w).to(dev), 130, 1, 700, qnn.W_NTC, 2, sw)
+    x_host = torch.from_numpy(a).pin_memory()
+    out_host = torch.zeros((1000, 130), dtype=torch.float32).pin_memory()
+    x_dev = torch.empty((1000, 700), dtype=torch.float32, device=dev)
+    planes = torch.empty((1000, 3, qnn.row_words(700)), dtype=torch.int32, device=dev)
+    out_dev = torch.empty((1000, 130), dtype=torch.float32, device=dev)
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    qnn.fc_forward_host_pipelined(x_host, 3, sa, 0, packed, 2, 130, alpha, out_host, x_dev, planes, out_dev, 192, streams)
+    torch.cuda.synchronize()
+    assert_fp32_close(out_host.numpy(), out)
