@@ -5,7 +5,13 @@ from pathlib import Path
 import pytest
 
 ROOT = Path(__file__).resolve().parent.parent
-if str(ROOT) not in sys.path:
+# tests/test_oracle_mutations.py runs the pins against a (mutated) copy of oracle/ placed elsewhere
+_ORACLE_ROOT = os.environ.get("QNN_TEST_ORACLE_ROOT")
+if _ORACLE_ROOT:
+    sys.path[:] = [p for p in sys.path if p not in ("", _ORACLE_ROOT, str(ROOT))]
+    sys.path.insert(0, _ORACLE_ROOT)          # ahead of the working directory, which holds the real oracle/
+    sys.path.insert(1, str(ROOT))
+elif str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
 
