@@ -56,11 +56,71 @@ bconv_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__r
     store_out(out, g.Cout, acc, m, co, g.Cout, valid * g.C * AB - 2 * s, alpha);
 }
 
+// Optional fused epilogue: the next layer's encoder applied to the fp32 result.
+struct NextEnc {
+    uint32_t *planes;
+    int bits;
+    float scale;
+    unsigned flags;
+};
+
+int check_next(const NextEnc *ne) {
+    if (!ne) return QNN_OK;
+    if (!ne->planes || !qnn_bits_ok(ne->bits) || (ne->flags & ~QNN_RELU)) return QNN_E_ARG;
+    if (!(ne->scale >= 1e-30f) || !(ne->scale <= 1e30f)) return QNN_E_SCALE;
+    if (!qnn_aligned(ne->planes, 16)) return QNN_E_ALIGN;
+    return QNN_OK;
+}
+
+void fill_next(qnn_tiled::Params &p, const NextEnc *ne, int Ng) {
+    if (!ne) return;
+    p.next_planes = ne->planes;
+    p.next_bits = ne->bits;
+    p.next_kw = (int)qnn_row_words_i(Ng);
+    p.next_inv2s = 1.0f / (2.0f * ne->scale);
+    p.next_half = (float)(1 << (ne->bits - 1));
+    qnn_clamp_bounds(ne->bits, ne->scale, (ne->flags & QNN_RELU) != 0, &p.next_lo, &p.next_hi);
+}
+
+int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
+               float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream);
+int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
+               int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc, const NextEnc *ne, void *stream);
+
 }  // namespace
 
 extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg,
                          float alpha, float *out, int64_t ldo, int32_t *acc, void *stream) {
-    if (!a_planes || !w_packed || (!out && !acc) || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
+    return bgemm_impl(a_planes, ab, w_packed, wb, Mg, Ng, Kg, alpha, out, ldo, acc, nullptr, stream);
+}
+
+extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
+                           int Cout, int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc,
+                           void *stream) {
+    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, alpha, out, acc, nullptr, stream);
+}
+
+extern "C" int qnn_bgemm_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng,
+                                int Kg, float alpha, int next_bits, float next_scale, unsigned next_flags,
+                                uint32_t *next_planes, float *out, int64_t ldo, void *stream) {
+    const NextEnc ne = {next_planes, next_bits, next_scale, next_flags};
+    return bgemm_impl(a_planes, ab, w_packed, wb, Mg, Ng, Kg, alpha, out, ldo, nullptr, &ne, stream);
+}
+
+extern "C" int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W,
+                                  int C, int Cout, int R, int S, int stride, int pad, float alpha, int next_bits,
+                                  float next_scale, unsigned next_flags, uint32_t *next_planes, float *out,
+                                  void *stream) {
+    const NextEnc ne = {next_planes, next_bits, next_scale, next_flags};
+    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, alpha, out, nullptr, &ne, stream);
+}
+
+namespace {
+
+int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
+               float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream) {
+    if (!a_planes || !w_packed || (!out && !acc && !ne) || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
+    if (const int rc = check_next(ne)) return rc;
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb) || (out && ldo < Ng)) return QNN_E_ARG;
     if (!isfinite(alpha)) return QNN_E_SCALE;
     if (!qnn_aligned(a_planes, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(out, 4) || !qnn_aligned(acc, 4))
@@ -76,13 +136,14 @@ extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed,
     p.Mg = Mg; p.Ng = Ng;
     p.a_pitch = kw; p.w_pitch = kw; p.kwords = kw;
     p.n_elems = Kg; p.alpha = alpha; p.out = out; p.ldo = ldo; p.acc = acc;
+    fill_next(p, ne, Ng);
     return qnn_tiled::dispatch_tiled(false, ab, wb, p, st);
 }
 
-extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
-                           int Cout, int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc,
-                           void *stream) {
-    if (!a_planes || !w_packed || (!out && !acc)) return QNN_E_ARG;
+int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
+               int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc, const NextEnc *ne, void *stream) {
+    if (!a_planes || !w_packed || (!out && !acc && !ne)) return QNN_E_ARG;
+    if (const int rc = check_next(ne)) return rc;
     if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || Cout <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0) return QNN_E_ARG;
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb)) return QNN_E_ARG;
     if (!isfinite(alpha)) return QNN_E_SCALE;
@@ -109,7 +170,10 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
         d.Mg = Mg; d.Ng = Cout; d.a_pitch = g.a_pitch; d.w_pitch = g.w_pitch;
         d.alpha = alpha; d.out = out; d.acc = acc;
         d.H = H; d.W = W; d.C = C; d.R = R; d.S = S; d.stride = stride; d.pad = pad; d.Ho = g.Ho; d.Wo = g.Wo;
-        return qnn_dense::dispatch_dense1(ab, wb, d, st);
+        if (ne && !out) return QNN_E_ARG;          // this path encodes from the fp32 result in a second launch
+        const int rc = qnn_dense::dispatch_dense1(ab, wb, d, st);
+        if (rc != QNN_OK || !ne) return rc;
+        return qnn_encode_pack(out, Mg, Cout, Cout, ne->bits, ne->scale, ne->flags, ne->planes, nullptr, stream);
     }
     // the tiled kernel divides by cw and S with a 20-bit multiply-shift: exact while kwords*cw and taps*S < 2^20
     if ((int64_t)R * S * g.cw * g.cw < (1 << 20) && (int64_t)R * S * S < (1 << 20) &&
@@ -124,13 +188,19 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
         p.n_elems = R * S * C; p.alpha = alpha; p.out = out; p.ldo = Cout; p.acc = acc;
         p.H = H; p.W = W; p.C = C; p.R = R; p.S = S; p.stride = stride; p.pad = pad; p.Ho = g.Ho; p.Wo = g.Wo;
         p.cw = g.cw; p.piece = (g.cw % 4 == 0) ? 4 : ((g.cw % 2 == 0) ? 2 : 1);
+        fill_next(p, ne, Cout);
         return qnn_tiled::dispatch_tiled(true, ab, wb, p, st);
     }
     dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
     if (grid.y > 65535) return QNN_E_RANGE;
+    if (ne && !out) return QNN_E_ARG;
     bconv_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, g, alpha, out, acc);
-    return qnn_launch_status();
+    if (cudaGetLastError() != cudaSuccess) return QNN_E_CUDA;
+    if (!ne) return QNN_OK;
+    return qnn_encode_pack(out, Mg, Cout, Cout, ne->bits, ne->scale, ne->flags, ne->planes, nullptr, stream);
 }
+
+}  // namespace
 
 extern "C" int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float scale_a, unsigned flags,
                                    const void *w_packed, int wb, int Ng, float alpha, float *out_host, float *x_dev,

@@ -51,6 +51,10 @@ struct Params {
     // convolution geometry
     int H, W, C, R, S, stride, pad, Ho, Wo, cw, piece;   // piece = words per copy (4, 2 or 1)
     uint32_t cw_magic, s_magic;                           // x / d == (x * magic) >> 20 for the ranges used
+    // fused next-layer encoder (optional): planes of the fp32 result, rows = output rows, k = Ng
+    uint32_t *next_planes;   // [Mg][next_bits][next_kw] or NULL
+    int next_bits, next_kw;
+    float next_inv2s, next_half, next_lo, next_hi;
 };
 
 // Splits kwords into full 8-word groups and a short tail: a remainder of 4..7 words is cheaper as one
@@ -109,7 +113,7 @@ __device__ __forceinline__ void pair8(const uint32_t (&ta)[8], const uint32_t (&
     acc += __popc(fours) * (4 << shift);
 }
 
-template <int AB, int WB, bool CONV, int TM>
+template <int AB, int WB, bool CONV, int TM, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p) {
     constexpr int kBM = 16 * TM;
     constexpr int A_UNITS = kBM * AB * kStageChunks;      // (row, plane, group) units per stage
@@ -344,10 +348,11 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
 #pragma unroll
         for (int r = 0; r < TM; ++r) {
             const int64_t m = m0 + ty + 16 * r;
-            if (m >= p.Mg) continue;
+            const bool row_ok = m < p.Mg;
+            if (!FUSED && !row_ok) continue;      // the fused encoder needs every lane at its ballots
             int n_valid = p.n_elems;
             int corr[4] = {0, 0, 0, 0};
-            if (CONV) {
+            if (CONV && row_ok) {
                 // Taps outside the image were staged as zero words: each contributed popc(w_j) to X_ij, i.e.
                 // AMAX * tapsum[n][tap] to S, and must not be counted in the length.
                 const int wo = (int)(m % p.Wo);
@@ -373,13 +378,49 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 }
                 n_valid = valid_taps * p.C;
             }
+            float fv[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int n = n0 + tx + 16 * c;
-                if (n >= p.Ng) continue;
+                if (!FUSED && n >= p.Ng) continue;
                 const int32_t v = n_valid * PROD - 2 * (acc[r][c] - AMAX * corr[c]);
-                if (p.acc) p.acc[m * p.Ng + n] = v;
-                if (p.out) p.out[m * p.ldo + n] = __fmul_rn(__int2float_rn(v), p.alpha);
+                fv[c] = __fmul_rn(__int2float_rn(v), p.alpha);
+                if (row_ok && n < p.Ng) {
+                    if (p.acc) p.acc[m * p.Ng + n] = v;
+                    if (p.out) p.out[m * p.ldo + n] = fv[c];
+                }
+            }
+            if (FUSED && p.next_planes != nullptr) {
+                // Next layer's encoder on the fp32 result (Alg. 1 forward: scale, then MBitEncoder).  A warp holds
+                // two output rows (lanes 0-15: row ty even, lanes 16-31: row ty odd) x 16 consecutive features
+                // per c, so one ballot per (plane, c) yields half a word for each of the two rows; c = 0,1 form
+                // word n0/32 and c = 2,3 word n0/32 + 1.  Every lane takes part in every ballot.
+                int t[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int n = n0 + tx + 16 * c;
+                    const int code = qnn_code_t(fv[c], p.next_inv2s, p.next_half, p.next_lo, p.next_hi);
+                    t[c] = (row_ok && n < p.Ng) ? code : 0;                 // padding bits are 0
+                }
+                const int lane = tid & 31;
+                const bool upper = lane >= 16;
+                const int word0 = n0 >> 5;
+                for (int i = 0; i < p.next_bits; ++i) {
+                    const uint32_t b0 = __ballot_sync(0xffffffffu, (t[0] >> i) & 1);
+                    const uint32_t b1 = __ballot_sync(0xffffffffu, (t[1] >> i) & 1);
+                    const uint32_t b2 = __ballot_sync(0xffffffffu, (t[2] >> i) & 1);
+                    const uint32_t b3 = __ballot_sync(0xffffffffu, (t[3] >> i) & 1);
+                    if ((lane & 15) == 0 && row_ok) {
+                        const uint32_t w0 = upper ? ((b0 >> 16) | (b1 & 0xffff0000u)) : ((b0 & 0xffffu) | (b1 << 16));
+                        const uint32_t w1 = upper ? ((b2 >> 16) | (b3 & 0xffff0000u)) : ((b2 & 0xffffu) | (b3 << 16));
+                        uint32_t *dst = p.next_planes + (m * p.next_bits + i) * (int64_t)p.next_kw + word0;
+                        *reinterpret_cast<uint2 *>(dst) = make_uint2(w0, w1);
+                        // the last feature tile also clears the padding words of the row
+                        if (n0 + kBN >= p.Ng)
+                            for (int wz = word0 + 2; wz < p.next_kw; wz += 2)
+                                *reinterpret_cast<uint2 *>(dst + (wz - word0)) = make_uint2(0u, 0u);
+                    }
+                }
             }
         }
         tile = next_tile;
@@ -445,12 +486,27 @@ static __global__ void __launch_bounds__(kThreads, 2) probe_csa73_kernel(int ite
 }
 constexpr double kProbeCsa73WordsPerThreadIter = 8.0 * kStageChunks * 4 * 4 * 2 * 2;
 
+template <int AB, int WB, bool CONV, int TM, bool FUSED>
+inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st);
+
+// The epilogue with the next layer's encoder is a separate instantiation for ab <= 4, so that the plain kernels
+// carry none of its code; for ab >= 5 (16-row tiles, where the epilogue matters less) one instantiation serves both.
 template <int AB, int WB, bool CONV, int TM>
 inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
+    if constexpr (AB >= 5) {
+        return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
+    } else {
+        if (p.next_planes != nullptr) return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
+        return launch_tiled_tmf<AB, WB, CONV, TM, false>(p, sms, st);
+    }
+}
+
+template <int AB, int WB, bool CONV, int TM, bool FUSED>
+inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     constexpr int kBM = 16 * TM;
     constexpr size_t smem = 2u * kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u;
     if (smem > 48u * 1024u &&
-        cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV, TM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV, TM, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
         return QNN_E_CUDA;
     Params q = p;
@@ -464,7 +520,7 @@ inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
     // about 5% faster (the hardware's dynamic block placement balances better than the static walk).
     const bool persistent = q.nstages <= 3;
     const int grid = (persistent && q.ntiles > 2 * sms) ? 2 * sms : q.ntiles;
-    bgemm_tiled_kernel<AB, WB, CONV, TM><<<grid, kThreads, smem, st>>>(q);
+    bgemm_tiled_kernel<AB, WB, CONV, TM, FUSED><<<grid, kThreads, smem, st>>>(q);
     return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA;
 }
 
@@ -487,8 +543,8 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
         // operation but give twice as many tiles.  Take them only when that fills the SMs better (small problems).
         const int64_t tn = (p.Ng + kBN - 1) / kBN;
         const int64_t t64 = ((p.Mg + 63) / 64) * tn, t32 = ((p.Mg + 31) / 32) * tn;
-        if (wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
-            return launch_tiled_tm<AB, WB, CONV, 2>(p, sms, st);
+        if (p.next_planes == nullptr && wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
+            return launch_tiled_tmf<AB, WB, CONV, 2, false>(p, sms, st);   // (no fused instantiation of this variant)
         return launch_tiled_tm<AB, WB, CONV, 4>(p, sms, st);
     } else {
         return launch_tiled_tm<AB, WB, CONV, TileM<AB>::TM>(p, sms, st);

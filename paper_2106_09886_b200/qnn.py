@@ -20,6 +20,7 @@ W_NTC, W_TCN, W_NCT = 0, 1, 2
 EXPORTS = [
     "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
+    "qnn_bgemm_encode", "qnn_bconv2d_encode",
     "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -52,6 +53,8 @@ def _load() -> C.CDLL:
     lib.qnn_pack_weights.argtypes = [p, i, i, i, i, i, f, p, p]
     lib.qnn_bgemm.argtypes = [p, i, p, i, i64, i, i, f, p, i64, p, p]
     lib.qnn_bconv2d.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, p]
+    lib.qnn_bgemm_encode.argtypes = [p, i, p, i, i64, i, i, f, i, f, u, p, p, i64, p]
+    lib.qnn_bconv2d_encode.argtypes = [p, i, p, i] + [i] * 9 + [f, i, f, u, p, p, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
     lib.qnn_fc_forward_host_pipelined.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, i64, C.POINTER(C.c_void_p), i]
@@ -164,6 +167,32 @@ def bconv2d(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N:
     _check(lib.qnn_bconv2d(_ptr(a_planes), ab, _ptr(w_packed), wb, N, H, W, Cin, Cout, R, S, stride, pad,
                            float(alpha), _ptr(out), _ptr(acc), _stream(stream)), "qnn_bconv2d")
     return (out, acc) if (want_acc or acc is not None) else out
+
+
+def bgemm_encode(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, Mg: int, Ng: int, Kg: int, alpha: float,
+                 next_bits: int, next_scale: float, next_flags: int = 0, next_planes: torch.Tensor | None = None,
+                 out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """FC layer whose epilogue is the next layer's encoder: returns the next layer's activation planes."""
+    if next_planes is None:
+        next_planes = torch.empty((Mg, next_bits, row_words(Ng)), dtype=torch.int32, device=a_planes.device)
+    _check(lib.qnn_bgemm_encode(_ptr(a_planes), ab, _ptr(w_packed), wb, Mg, Ng, Kg, float(alpha), next_bits,
+                                float(next_scale), next_flags, _ptr(next_planes), _ptr(out),
+                                out.stride(0) if out is not None else Ng, _stream(stream)), "qnn_bgemm_encode")
+    return next_planes
+
+
+def bconv2d_encode(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N: int, H: int, W: int, Cin: int,
+                   Cout: int, R: int, S: int, stride: int, pad: int, alpha: float, next_bits: int, next_scale: float,
+                   next_flags: int = 0, next_planes: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                   stream=None) -> torch.Tensor:
+    """Convolution whose epilogue is the next layer's encoder: returns planes [N*Ho*Wo, next_bits, row_words(Cout)]."""
+    Ho, Wo = conv_out_dim(H, R, stride, pad), conv_out_dim(W, S, stride, pad)
+    if next_planes is None:
+        next_planes = torch.empty((N * Ho * Wo, next_bits, row_words(Cout)), dtype=torch.int32, device=a_planes.device)
+    _check(lib.qnn_bconv2d_encode(_ptr(a_planes), ab, _ptr(w_packed), wb, N, H, W, Cin, Cout, R, S, stride, pad,
+                                  float(alpha), next_bits, float(next_scale), next_flags, _ptr(next_planes), _ptr(out),
+                                  _stream(stream)), "qnn_bconv2d_encode")
+    return next_planes
 
 
 def absmax_f32(x: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:

@@ -100,10 +100,17 @@ def time_stack(net: str, batch: int, reps=3, warmup=2, dev="cuda:0", seed=0, lay
         t_enc = _time_calls(lambda i: qnn.encode_pack(a, s.ab, sa, qnn.RELU, planes=planes), reps, warmup)
         t_conv = _time_calls(lambda i: qnn.bconv2d(planes, s.ab, packed, s.wb, s.N, s.H, s.W, s.C, s.Cout, s.R, s.S,
                                                    s.stride, s.pad, 1e-3, out=out), reps, warmup)
+        # layer chaining: the same convolution writing the next layer's planes instead of fp32
+        nxt = torch.empty((s.Mg, s.ab, qnn.row_words(s.Cout)), dtype=torch.int32, device=dev)
+        fused_out = out if (s.R * s.S * s.C <= 32) else None      # single-word patches encode from the fp32 result
+        t_fused = _time_calls(lambda i: qnn.bconv2d_encode(planes, s.ab, packed, s.wb, s.N, s.H, s.W, s.C, s.Cout, s.R,
+                                                           s.S, s.stride, s.pad, 1e-3, s.ab, sa, qnn.RELU,
+                                                           next_planes=nxt, out=fused_out), reps, warmup)
+        del nxt
         enc_ms, conv_ms = statistics.median(t_enc), statistics.median(t_conv)
         macs = float(s.Mg) * s.Cout * s.Kg
         rows.append({"layer": s.name, "Mg": s.Mg, "Ng": s.Cout, "Kg": s.Kg, "ab": s.ab, "wb": s.wb,
-                     "encode_ms": enc_ms, "conv_ms": conv_ms,
+                     "encode_ms": enc_ms, "conv_ms": conv_ms, "conv_encode_ms": statistics.median(t_fused),
                      "conv_binary_tops": 2 * macs * s.ab * s.wb / (conv_ms * 1e-3) / 1e12,
                      "conv_equiv_int_gops": 2 * macs / (conv_ms * 1e-3) / 1e9,
                      "encode_gbs": (a.numel() * 4 + planes.numel() * 4) / (enc_ms * 1e-3) / 1e9,
@@ -156,11 +163,13 @@ def main():
         layers = [int(v) for v in a.layers.split(",")] if a.layers else None
         r = time_stack(a.net, batch, a.reps, a.warmup, layers=layers)
         if a.table:
-            print(f"{'layer':28s} {'Mg':>8s} {'Ng':>4s} {'Kg':>5s} {'enc ms':>8s} {'conv ms':>8s} {'bTOPS':>7s} {'enc GB/s':>8s}")
+            print(f"{'layer':28s} {'Mg':>8s} {'Ng':>4s} {'Kg':>5s} {'enc ms':>8s} {'conv ms':>8s} {'bTOPS':>7s} {'enc GB/s':>8s} {'conv+enc fused ms':>18s}")
             for L in r["layers"]:
                 print(f"{L['layer']:28s} {L['Mg']:8d} {L['Ng']:4d} {L['Kg']:5d} {L['encode_ms']:8.3f} {L['conv_ms']:8.3f} "
-                      f"{L['conv_binary_tops']:7.1f} {L['encode_gbs']:8.0f}")
-            print(f"total {r['total_ms']:.3f} ms, {r['binary_tops']:.1f} binary TOPS, {r['equiv_int_gops']:.0f} equiv int GOPS")
+                      f"{L['conv_binary_tops']:7.1f} {L['encode_gbs']:8.0f} {L['conv_encode_ms']:18.3f}")
+            print(f"total {r['total_ms']:.3f} ms (encode + conv per layer), {r['binary_tops']:.1f} binary TOPS, "
+                  f"{r['equiv_int_gops']:.0f} equiv int GOPS; chained plane-to-plane (fused encoder, no fp32 between "
+                  f"layers): {sum(L['conv_encode_ms'] for L in r['layers']):.3f} ms")
             return
     else:
         r = time_encode(a.rows, a.k, a.bits, a.reps, a.warmup, a.sets)
