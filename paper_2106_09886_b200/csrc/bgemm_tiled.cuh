@@ -551,39 +551,32 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
     }
 }
 
-// All weight widths and both operand kinds for one activation width; each activation width is compiled in
-// its own translation unit (tiled_ab<N>.cu) so that the 100+ kernel instantiations build in parallel.
-template <int AB>
-inline int run_tiled_ab(bool conv, int wb, const Params &p, cudaStream_t st) {
+// All weight widths for one activation width and operand kind; each (width, kind) is compiled in its own
+// translation unit (tiled_ab<N>_fc.cu / tiled_ab<N>_conv.cu) so that the kernel instantiations build in parallel.
+template <int AB, bool CONV>
+inline int run_tiled_ab(int wb, const Params &p, cudaStream_t st) {
 #define QNN_T(W_) \
-    case W_: return conv ? launch_tiled<AB, W_, true>(p, st) : launch_tiled<AB, W_, false>(p, st);
+    case W_: return launch_tiled<AB, W_, CONV>(p, st);
     switch (wb) {
         QNN_T(1) QNN_T(2) QNN_T(3) QNN_T(4) QNN_T(5) QNN_T(6) QNN_T(7) QNN_T(8)
         default: return QNN_E_ARG;
     }
 #undef QNN_T
 }
-int run_tiled_ab1(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab2(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab3(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab4(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab5(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab6(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab7(bool conv, int wb, const Params &p, cudaStream_t st);
-int run_tiled_ab8(bool conv, int wb, const Params &p, cudaStream_t st);
+#define QNN_DECL(N_) \
+    int run_tiled_ab##N_##_fc(int wb, const Params &p, cudaStream_t st); \
+    int run_tiled_ab##N_##_conv(int wb, const Params &p, cudaStream_t st);
+QNN_DECL(1) QNN_DECL(2) QNN_DECL(3) QNN_DECL(4) QNN_DECL(5) QNN_DECL(6) QNN_DECL(7) QNN_DECL(8)
+#undef QNN_DECL
 
 inline int dispatch_tiled(bool conv, int ab, int wb, const Params &p, cudaStream_t st) {
+#define QNN_CASE(N_) \
+    case N_: return conv ? run_tiled_ab##N_##_conv(wb, p, st) : run_tiled_ab##N_##_fc(wb, p, st);
     switch (ab) {
-        case 1: return run_tiled_ab1(conv, wb, p, st);
-        case 2: return run_tiled_ab2(conv, wb, p, st);
-        case 3: return run_tiled_ab3(conv, wb, p, st);
-        case 4: return run_tiled_ab4(conv, wb, p, st);
-        case 5: return run_tiled_ab5(conv, wb, p, st);
-        case 6: return run_tiled_ab6(conv, wb, p, st);
-        case 7: return run_tiled_ab7(conv, wb, p, st);
-        case 8: return run_tiled_ab8(conv, wb, p, st);
+        QNN_CASE(1) QNN_CASE(2) QNN_CASE(3) QNN_CASE(4) QNN_CASE(5) QNN_CASE(6) QNN_CASE(7) QNN_CASE(8)
         default: return QNN_E_ARG;
     }
+#undef QNN_CASE
 }
 
 }  // namespace qnn_tiled
