@@ -47,7 +47,7 @@ POPC_PER_WORD = 0.5   # popcounts the tiled kernel issues per 32-bit xor word (7
 
 # DRAM read+write of one qnn_bgemm 4096^3 w2a2 launch from the ncu capture summarised in
 # profiles/bgemm_tiled_4096_w2a2.md, valid for the kernel source with this digest only.
-NCU_TRAFFIC = {"bytes": None, "kernel_sha256": None}
+NCU_TRAFFIC = {"bytes": 22787840, "kernel_sha256": "86278b5f1cca1f4216f8206c86dcaf6814e2a15db33e49991d399cc420da205b"}
 
 
 def ncu_traffic_bytes():
@@ -79,7 +79,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -384,7 +384,7 @@ def run_gpu(args):
         qnn.fc_forward_host_pipelined(a_host, AB, sa, 0, packed, WB, Ng, alpha, out_host, a_bufs[b], planes[b],
                                       out_bufs[b], E2E_CHUNK_ROWS, e2e_streams)
 
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(args.steps, 50))
     for i in range(3):
         e2e_step(i)
     barrier()
@@ -461,8 +461,8 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["graft", "reference"], default="graft")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
