@@ -138,24 +138,32 @@ int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, 
 
 /*
  * Layer chaining (Alg. 1 forward: weighted branch sum, scale, then the next layer's MBitEncoder): the
- * contraction of qnn_bgemm / qnn_bconv2d whose epilogue also quantizes, encodes and bit-plane-packs its own
- * fp32 result for the next layer, so that a stack of layers never round-trips through fp32 in memory.
+ * contraction of qnn_bgemm / qnn_bconv2d whose epilogue can also apply a per-feature affine and quantize,
+ * encode and bit-plane-pack its own fp32 result for the next layer, so that a stack of layers never
+ * round-trips through fp32 in memory.
+ *   ch_gamma, ch_beta   optional fp32 [Ng] (device): y = fma(float(acc)*alpha, ch_gamma[n], ch_beta[n]), one
+ *                       rounding; a folded batch normalisation (Section 3.2: when batch normalisation follows,
+ *                       the fixed scaling factor is not used, i.e. pass alpha = 1).  ch_beta may be NULL (0);
+ *                       ch_gamma NULL = no affine.
+ *   next_planes  optional out, uint32 [Mg][next_bits][qnn_row_words(Ng)] (conv: Mg = N*Ho*Wo pixels,
+ *                Ng = Cout), bit-identical to qnn_encode_pack applied to the fp32 result y; NULL = no encoder
+ *                (then next_bits / next_scale / next_flags are ignored)
  *   next_bits, next_scale, next_flags   as bits / scale / flags of qnn_encode_pack (QNN_RELU = the ReLU
  *                                       between the layers); the scale is fixed by the caller beforehand
  *                                       (the paper's range r is a constant or a learned parameter)
- *   next_planes  out, uint32 [Mg][next_bits][qnn_row_words(Ng)] (conv: Mg = N*Ho*Wo pixels, Ng = Cout),
- *                bit-identical to qnn_encode_pack applied to the fp32 result
- *   out          optional fp32 result as in qnn_bgemm / qnn_bconv2d; may be NULL (then nothing but the planes
- *                is written), except for convolutions whose whole patch fits one word (R*S*C <= 32) or whose
- *                geometry is outside the tiled kernel: those encode from `out` in a second launch and need it
- * Other arguments, checks and errors as in qnn_bgemm / qnn_bconv2d.
+ *   out          optional fp32 result y; may be NULL when next_planes is given, except for convolutions whose
+ *                whole patch fits one word (R*S*C <= 32) or whose geometry is outside the tiled kernel:
+ *                those encode from `out` in a second launch and need it (the latter also take no affine)
+ * At least one of ch_gamma / next_planes must be given.  Other arguments, checks and errors as in
+ * qnn_bgemm / qnn_bconv2d.
  */
 int qnn_bgemm_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg,
-                     float alpha, int next_bits, float next_scale, unsigned next_flags, uint32_t *next_planes,
-                     float *out, int64_t ldo, void *stream);
+                     float alpha, const float *ch_gamma, const float *ch_beta, int next_bits, float next_scale,
+                     unsigned next_flags, uint32_t *next_planes, float *out, int64_t ldo, void *stream);
 int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
-                       int Cout, int R, int S, int stride, int pad, float alpha, int next_bits, float next_scale,
-                       unsigned next_flags, uint32_t *next_planes, float *out, void *stream);
+                       int Cout, int R, int S, int stride, int pad, float alpha, const float *ch_gamma,
+                       const float *ch_beta, int next_bits, float next_scale, unsigned next_flags,
+                       uint32_t *next_planes, float *out, void *stream);
 
 /*
  * max_i |x[i]| into *out (device fp32), for workloads whose grid step is derived

@@ -13,6 +13,7 @@ What each function follows in the paper:
 * ``fc`` / ``conv2d`` (and their ``_sampled`` forms) -- Op(EnC(x), EnC(w)) of Eq. 9:
                       the plain integer product that Eq. 8 reproduces exactly.
 * ``scale``        -- the fixed scaling factor of Eq. 9 / Alg. 1 forward pass.
+* ``affine``       -- per-feature affine that replaces the scale when batch normalisation follows (Section 3.2).
 """
 from __future__ import annotations
 
@@ -59,6 +60,7 @@ def _load():
         lib.oracle_conv2d.argtypes = [p, p] + [c.c_int] * 9 + [p]
         lib.oracle_conv2d_sampled.argtypes = [p, p] + [c.c_int] * 9 + [c.c_size_t, p, p, p]
         lib.oracle_scale.argtypes = [p, c.c_size_t, c.c_float, p]
+        lib.oracle_affine.argtypes = [p, c.c_size_t, c.c_size_t, p, p]
         _lib = lib
     return _lib
 
@@ -165,4 +167,18 @@ def scale(acc: np.ndarray, alpha) -> np.ndarray:
     acc = np.ascontiguousarray(acc, dtype=np.int32)
     out = np.empty(acc.shape, dtype=np.float32)
     _check(_load().oracle_scale(_ptr(acc), acc.size, float(np.float32(alpha)), _ptr(out)), "scale")
+    return out
+
+
+def affine(y: np.ndarray, gamma: np.ndarray, beta: np.ndarray | None = None) -> np.ndarray:
+    """y[..., n] -> fma(y, gamma[n], beta[n]) in binary32 (last axis = features); returns a new array."""
+    out = np.ascontiguousarray(y, dtype=np.float32).copy()
+    gamma = np.ascontiguousarray(gamma, dtype=np.float32)
+    Ng = out.shape[-1]
+    assert gamma.shape == (Ng,)
+    if beta is not None:
+        beta = np.ascontiguousarray(beta, dtype=np.float32)
+        assert beta.shape == (Ng,)
+    _check(_load().oracle_affine(_ptr(out), out.size // Ng, Ng, _ptr(gamma), _ptr(beta) if beta is not None else None),
+           "affine")
     return out

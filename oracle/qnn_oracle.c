@@ -224,3 +224,16 @@ int oracle_scale(const int32_t *acc, size_t n, float alpha, float *out) {
     for (ptrdiff_t i = 0; i < (ptrdiff_t)n; ++i) out[i] = (float)acc[i] * alpha;
     return ORACLE_OK;
 }
+
+/*
+ * Per-feature affine after the scale (a folded batch-normalisation; Section 3.2 notes that when batch
+ * normalisation follows, the fixed scaling factor is dropped, i.e. alpha = 1 and the affine carries the scale):
+ * y[m][n] = fma(y[m][n], gamma[n], beta[n]) in binary32, one rounding.  beta may be NULL (0).
+ */
+int oracle_affine(float *y, size_t rows, size_t Ng, const float *gamma, const float *beta) {
+    if (!y || !gamma) return ORACLE_E_ARG;
+#pragma omp parallel for schedule(static)
+    for (ptrdiff_t m = 0; m < (ptrdiff_t)rows; ++m)
+        for (size_t n = 0; n < Ng; ++n) y[(size_t)m * Ng + n] = fmaf(y[(size_t)m * Ng + n], gamma[n], beta ? beta[n] : 0.0f);
+    return ORACLE_OK;
+}

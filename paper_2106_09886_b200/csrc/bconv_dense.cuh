@@ -23,6 +23,7 @@ struct Params {
     int Ng;
     int a_pitch, w_pitch;
     float alpha;
+    const float *ch_gamma, *ch_beta;   // optional per-feature affine after the scale
     float *out;
     int32_t *acc;
     int H, W, C, R, S, stride, pad, Ho, Wo;
@@ -86,6 +87,9 @@ __global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) 
             uint32_t wreg[WB];
 #pragma unroll
             for (int j = 0; j < WB; ++j) wreg[j] = n_ok ? wd_s[j * p.Ng + n] : 0u;
+            const bool affine = p.ch_gamma != nullptr && n_ok;
+            const float gam = affine ? __ldg(p.ch_gamma + n) : 1.0f;
+            const float bet = (affine && p.ch_beta) ? __ldg(p.ch_beta + n) : 0.0f;
             for (int rr = 0; rr < rows_here; ++rr) {
                 int s_acc = 0;
 #pragma unroll
@@ -106,7 +110,11 @@ __global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) 
                     const int32_t v = n_valid * PROD - 2 * (s_acc - AMAX * corr);
                     const int64_t o = (batch * 32 + rr) * (int64_t)p.Ng + n;
                     if (p.acc) p.acc[o] = v;
-                    if (p.out) p.out[o] = __fmul_rn(__int2float_rn(v), p.alpha);
+                    if (p.out) {
+                        float y = __fmul_rn(__int2float_rn(v), p.alpha);
+                        if (affine) y = __fmaf_rn(y, gam, bet);
+                        p.out[o] = y;
+                    }
                 }
             }
         }

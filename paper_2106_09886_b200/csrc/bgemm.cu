@@ -58,15 +58,21 @@ bconv_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__r
 
 // Optional fused epilogue: the next layer's encoder applied to the fp32 result.
 struct NextEnc {
-    uint32_t *planes;
+    uint32_t *planes;      // NULL: no encoder (then only the affine is applied)
     int bits;
     float scale;
     unsigned flags;
+    const float *gamma;    // NULL: no per-feature affine
+    const float *beta;
 };
 
 int check_next(const NextEnc *ne) {
     if (!ne) return QNN_OK;
-    if (!ne->planes || !qnn_bits_ok(ne->bits) || (ne->flags & ~QNN_RELU)) return QNN_E_ARG;
+    if (!ne->planes && !ne->gamma) return QNN_E_ARG;           // nothing to do beyond qnn_bgemm / qnn_bconv2d
+    if (ne->beta && !ne->gamma) return QNN_E_ARG;
+    if (!qnn_aligned(ne->gamma, 4) || !qnn_aligned(ne->beta, 4)) return QNN_E_ALIGN;
+    if (!ne->planes) return QNN_OK;
+    if (!qnn_bits_ok(ne->bits) || (ne->flags & ~QNN_RELU)) return QNN_E_ARG;
     if (!(ne->scale >= 1e-30f) || !(ne->scale <= 1e30f)) return QNN_E_SCALE;
     if (!qnn_aligned(ne->planes, 16)) return QNN_E_ALIGN;
     return QNN_OK;
@@ -74,6 +80,9 @@ int check_next(const NextEnc *ne) {
 
 void fill_next(qnn_tiled::Params &p, const NextEnc *ne, int Ng) {
     if (!ne) return;
+    p.ch_gamma = ne->gamma;
+    p.ch_beta = ne->beta;
+    if (!ne->planes) return;
     p.next_planes = ne->planes;
     p.next_bits = ne->bits;
     p.next_kw = (int)qnn_row_words_i(Ng);
@@ -101,17 +110,18 @@ extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packe
 }
 
 extern "C" int qnn_bgemm_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng,
-                                int Kg, float alpha, int next_bits, float next_scale, unsigned next_flags,
-                                uint32_t *next_planes, float *out, int64_t ldo, void *stream) {
-    const NextEnc ne = {next_planes, next_bits, next_scale, next_flags};
+                                int Kg, float alpha, const float *ch_gamma, const float *ch_beta, int next_bits,
+                                float next_scale, unsigned next_flags, uint32_t *next_planes, float *out, int64_t ldo,
+                                void *stream) {
+    const NextEnc ne = {next_planes, next_bits, next_scale, next_flags, ch_gamma, ch_beta};
     return bgemm_impl(a_planes, ab, w_packed, wb, Mg, Ng, Kg, alpha, out, ldo, nullptr, &ne, stream);
 }
 
 extern "C" int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W,
-                                  int C, int Cout, int R, int S, int stride, int pad, float alpha, int next_bits,
-                                  float next_scale, unsigned next_flags, uint32_t *next_planes, float *out,
-                                  void *stream) {
-    const NextEnc ne = {next_planes, next_bits, next_scale, next_flags};
+                                  int C, int Cout, int R, int S, int stride, int pad, float alpha, const float *ch_gamma,
+                                  const float *ch_beta, int next_bits, float next_scale, unsigned next_flags,
+                                  uint32_t *next_planes, float *out, void *stream) {
+    const NextEnc ne = {next_planes, next_bits, next_scale, next_flags, ch_gamma, ch_beta};
     return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, alpha, out, nullptr, &ne, stream);
 }
 
@@ -119,8 +129,9 @@ namespace {
 
 int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
                float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream) {
-    if (!a_planes || !w_packed || (!out && !acc && !ne) || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
+    if (!a_planes || !w_packed || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
     if (const int rc = check_next(ne)) return rc;
+    if (!out && !acc && !(ne && ne->planes)) return QNN_E_ARG;
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb) || (out && ldo < Ng)) return QNN_E_ARG;
     if (!isfinite(alpha)) return QNN_E_SCALE;
     if (!qnn_aligned(a_planes, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(out, 4) || !qnn_aligned(acc, 4))
@@ -142,8 +153,9 @@ int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
 
 int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
                int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc, const NextEnc *ne, void *stream) {
-    if (!a_planes || !w_packed || (!out && !acc && !ne)) return QNN_E_ARG;
+    if (!a_planes || !w_packed) return QNN_E_ARG;
     if (const int rc = check_next(ne)) return rc;
+    if (!out && !acc && !(ne && ne->planes)) return QNN_E_ARG;
     if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || Cout <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0) return QNN_E_ARG;
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb)) return QNN_E_ARG;
     if (!isfinite(alpha)) return QNN_E_SCALE;
@@ -171,8 +183,9 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
         d.alpha = alpha; d.out = out; d.acc = acc;
         d.H = H; d.W = W; d.C = C; d.R = R; d.S = S; d.stride = stride; d.pad = pad; d.Ho = g.Ho; d.Wo = g.Wo;
         if (ne && !out) return QNN_E_ARG;          // this path encodes from the fp32 result in a second launch
+        if (ne) { d.ch_gamma = ne->gamma; d.ch_beta = ne->beta; }
         const int rc = qnn_dense::dispatch_dense1(ab, wb, d, st);
-        if (rc != QNN_OK || !ne) return rc;
+        if (rc != QNN_OK || !ne || !ne->planes) return rc;
         return qnn_encode_pack(out, Mg, Cout, Cout, ne->bits, ne->scale, ne->flags, ne->planes, nullptr, stream);
     }
     // the tiled kernel divides by cw and S with a 20-bit multiply-shift: exact while kwords*cw and taps*S < 2^20
@@ -193,10 +206,10 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     }
     dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
     if (grid.y > 65535) return QNN_E_RANGE;
-    if (ne && !out) return QNN_E_ARG;
+    if (ne && (!out || ne->gamma)) return QNN_E_ARG;   // the fallback kernel has no affine epilogue
     bconv_generic_kernel<<<grid, 256, 0, st>>>(a_planes, ab, w, wb, g, alpha, out, acc);
     if (cudaGetLastError() != cudaSuccess) return QNN_E_CUDA;
-    if (!ne) return QNN_OK;
+    if (!ne || !ne->planes) return QNN_OK;
     return qnn_encode_pack(out, Mg, Cout, Cout, ne->bits, ne->scale, ne->flags, ne->planes, nullptr, stream);
 }
 

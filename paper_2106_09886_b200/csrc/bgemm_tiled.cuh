@@ -51,6 +51,8 @@ struct Params {
     // convolution geometry
     int H, W, C, R, S, stride, pad, Ho, Wo, cw, piece;   // piece = words per copy (4, 2 or 1)
     uint32_t cw_magic, s_magic;                           // x / d == (x * magic) >> 20 for the ranges used
+    // optional per-feature affine applied after the scale: y = fma(y, ch_gamma[n], ch_beta[n]) (ch_beta may be NULL)
+    const float *ch_gamma, *ch_beta;
     // fused next-layer encoder (optional): planes of the fp32 result, rows = output rows, k = Ng
     uint32_t *next_planes;   // [Mg][next_bits][next_kw] or NULL
     int next_bits, next_kw;
@@ -385,6 +387,8 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 if (!FUSED && n >= p.Ng) continue;
                 const int32_t v = n_valid * PROD - 2 * (acc[r][c] - AMAX * corr[c]);
                 fv[c] = __fmul_rn(__int2float_rn(v), p.alpha);
+                if (FUSED && p.ch_gamma != nullptr && n < p.Ng)
+                    fv[c] = __fmaf_rn(fv[c], __ldg(p.ch_gamma + n), p.ch_beta ? __ldg(p.ch_beta + n) : 0.0f);
                 if (row_ok && n < p.Ng) {
                     if (p.acc) p.acc[m * p.Ng + n] = v;
                     if (p.out) p.out[m * p.ldo + n] = fv[c];
@@ -496,7 +500,7 @@ inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
     if constexpr (AB >= 5) {
         return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
     } else {
-        if (p.next_planes != nullptr) return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
+        if (p.next_planes != nullptr || p.ch_gamma != nullptr) return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
         return launch_tiled_tmf<AB, WB, CONV, TM, false>(p, sms, st);
     }
 }
@@ -543,7 +547,7 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
         // operation but give twice as many tiles.  Take them only when that fills the SMs better (small problems).
         const int64_t tn = (p.Ng + kBN - 1) / kBN;
         const int64_t t64 = ((p.Mg + 63) / 64) * tn, t32 = ((p.Mg + 31) / 32) * tn;
-        if (p.next_planes == nullptr && wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
+        if (p.next_planes == nullptr && p.ch_gamma == nullptr && wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
             return launch_tiled_tmf<AB, WB, CONV, 2, false>(p, sms, st);   // (no fused instantiation of this variant)
         return launch_tiled_tm<AB, WB, CONV, 4>(p, sms, st);
     } else {

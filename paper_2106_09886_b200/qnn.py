@@ -53,8 +53,8 @@ def _load() -> C.CDLL:
     lib.qnn_pack_weights.argtypes = [p, i, i, i, i, i, f, p, p]
     lib.qnn_bgemm.argtypes = [p, i, p, i, i64, i, i, f, p, i64, p, p]
     lib.qnn_bconv2d.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, p]
-    lib.qnn_bgemm_encode.argtypes = [p, i, p, i, i64, i, i, f, i, f, u, p, p, i64, p]
-    lib.qnn_bconv2d_encode.argtypes = [p, i, p, i] + [i] * 9 + [f, i, f, u, p, p, p]
+    lib.qnn_bgemm_encode.argtypes = [p, i, p, i, i64, i, i, f, p, p, i, f, u, p, p, i64, p]
+    lib.qnn_bconv2d_encode.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, i, f, u, p, p, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
     lib.qnn_fc_forward_host_pipelined.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, i64, C.POINTER(C.c_void_p), i]
@@ -171,28 +171,34 @@ def bconv2d(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N:
 
 def bgemm_encode(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, Mg: int, Ng: int, Kg: int, alpha: float,
                  next_bits: int, next_scale: float, next_flags: int = 0, next_planes: torch.Tensor | None = None,
-                 out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
-    """FC layer whose epilogue is the next layer's encoder: returns the next layer's activation planes."""
-    if next_planes is None:
+                 out: torch.Tensor | None = None, ch_gamma: torch.Tensor | None = None,
+                 ch_beta: torch.Tensor | None = None, encode: bool = True, stream=None):
+    """FC layer whose epilogue applies an optional per-feature affine and (encode=True) the next layer's encoder.
+    Returns the next layer's activation planes, or `out` when encode is False."""
+    if encode and next_planes is None:
         next_planes = torch.empty((Mg, next_bits, row_words(Ng)), dtype=torch.int32, device=a_planes.device)
-    _check(lib.qnn_bgemm_encode(_ptr(a_planes), ab, _ptr(w_packed), wb, Mg, Ng, Kg, float(alpha), next_bits,
-                                float(next_scale), next_flags, _ptr(next_planes), _ptr(out),
+    _check(lib.qnn_bgemm_encode(_ptr(a_planes), ab, _ptr(w_packed), wb, Mg, Ng, Kg, float(alpha), _ptr(ch_gamma),
+                                _ptr(ch_beta), next_bits, float(next_scale), next_flags,
+                                _ptr(next_planes) if encode else None, _ptr(out),
                                 out.stride(0) if out is not None else Ng, _stream(stream)), "qnn_bgemm_encode")
-    return next_planes
+    return next_planes if encode else out
 
 
 def bconv2d_encode(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N: int, H: int, W: int, Cin: int,
                    Cout: int, R: int, S: int, stride: int, pad: int, alpha: float, next_bits: int, next_scale: float,
                    next_flags: int = 0, next_planes: torch.Tensor | None = None, out: torch.Tensor | None = None,
-                   stream=None) -> torch.Tensor:
-    """Convolution whose epilogue is the next layer's encoder: returns planes [N*Ho*Wo, next_bits, row_words(Cout)]."""
+                   ch_gamma: torch.Tensor | None = None, ch_beta: torch.Tensor | None = None, encode: bool = True,
+                   stream=None):
+    """Convolution whose epilogue applies an optional per-feature affine and (encode=True) the next layer's
+    encoder: returns planes [N*Ho*Wo, next_bits, row_words(Cout)], or `out` when encode is False."""
     Ho, Wo = conv_out_dim(H, R, stride, pad), conv_out_dim(W, S, stride, pad)
-    if next_planes is None:
+    if encode and next_planes is None:
         next_planes = torch.empty((N * Ho * Wo, next_bits, row_words(Cout)), dtype=torch.int32, device=a_planes.device)
     _check(lib.qnn_bconv2d_encode(_ptr(a_planes), ab, _ptr(w_packed), wb, N, H, W, Cin, Cout, R, S, stride, pad,
-                                  float(alpha), next_bits, float(next_scale), next_flags, _ptr(next_planes), _ptr(out),
-                                  _stream(stream)), "qnn_bconv2d_encode")
-    return next_planes
+                                  float(alpha), _ptr(ch_gamma), _ptr(ch_beta), next_bits, float(next_scale), next_flags,
+                                  _ptr(next_planes) if encode else None, _ptr(out), _stream(stream)),
+           "qnn_bconv2d_encode")
+    return next_planes if encode else out
 
 
 def absmax_f32(x: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:

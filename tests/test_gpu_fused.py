@@ -111,11 +111,68 @@ def test_fused_argument_errors():
     nxt = torch.zeros((8, 2, 4), dtype=torch.int32, device=dev)
     p = lambda t: ctypes.c_void_p(t.data_ptr())
     f = qnn.lib.qnn_bgemm_encode
-    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, 2, 1.0, 0, None, None, 8, None) == qnn.E_ARG
-    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, 9, 1.0, 0, p(nxt), None, 8, None) == qnn.E_ARG
-    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, 2, 0.0, 0, p(nxt), None, 8, None) == qnn.E_SCALE
-    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, 2, 1.0, 4, p(nxt), None, 8, None) == qnn.E_ARG
+    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, None, None, 2, 1.0, 0, None, None, 8, None) == qnn.E_ARG
+    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, None, None, 9, 1.0, 0, p(nxt), None, 8, None) == qnn.E_ARG
+    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, None, None, 2, 0.0, 0, p(nxt), None, 8, None) == qnn.E_SCALE
+    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, None, None, 2, 1.0, 4, p(nxt), None, 8, None) == qnn.E_ARG
+    g = torch.ones(8, dtype=torch.float32, device=dev)
+    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, None, p(g), 2, 1.0, 0, p(nxt), None, 8, None) == qnn.E_ARG   # beta without gamma
+    assert f(p(planes), 2, p(packed), 2, 8, 8, 64, 1.0, p(g), None, 2, 1.0, 0, None, None, 8, None) == qnn.E_ARG     # affine only needs out
     # single-word patches encode from the fp32 result and therefore need `out`
     a3 = qnn.encode_pack(torch.zeros((16, 3), dtype=torch.float32, device=dev), 2, 1.0)
     w3 = qnn.pack_weights(torch.ones((4, 9, 3), dtype=torch.float32, device=dev), 4, 9, 3, qnn.W_NTC, 2, 1.0)
-    assert qnn.lib.qnn_bconv2d_encode(p(a3), 2, p(w3), 2, 1, 4, 4, 3, 4, 3, 3, 1, 1, 1.0, 2, 1.0, 0, p(nxt), None, None) == qnn.E_ARG
+    assert qnn.lib.qnn_bconv2d_encode(p(a3), 2, p(w3), 2, 1, 4, 4, 3, 4, 3, 3, 1, 1, 1.0, None, None, 2, 1.0, 0, p(nxt), None, None) == qnn.E_ARG
+
+
+@pytest.mark.parametrize("with_beta", [True, False])
+def test_bgemm_affine_then_encode(with_beta):
+    """Folded batch-norm: alpha = 1, y = fma(acc, gamma[n], beta[n]); fp32 result and next planes both checked."""
+    torch, qnn, dev = _env()
+    rng = np.random.default_rng(5)
+    Mg, Ng, Kg, ab, wb, nb = 150, 100, 500, 3, 2, 3
+    a = rng.standard_normal((Mg, Kg)).astype(np.float32)
+    w = rng.standard_normal((Ng, Kg)).astype(np.float32)
+    sa, sw, _ = scales_for(a, w, ab, wb)
+    _, _, acc, _ = oracle_fc(a, w, False, ab, wb, sa, sw, np.float32(1))
+    gamma = (rng.standard_normal(Ng) * 1e-3).astype(np.float32)
+    beta = rng.standard_normal(Ng).astype(np.float32) if with_beta else None
+    y = oracle.affine(oracle.scale(acc, np.float32(1)), gamma, beta)
+    ns = wl.per_tensor_scale(np.maximum(y, 0), nb)
+    want = oracle.pack_planes(oracle.quantize(y, nb, ns, True), nb)
+    planes = qnn.encode_pack(torch.from_numpy(a).to(dev), ab, sa)
+    packed = qnn.pack_weights(torch.from_numpy(w).to(dev), Ng, 1, Kg, qnn.W_NTC, wb, sw)
+    g_d = torch.from_numpy(gamma).to(dev)
+    b_d = torch.from_numpy(beta).to(dev) if with_beta else None
+    out_d = torch.empty((Mg, Ng), dtype=torch.float32, device=dev)
+    nxt = qnn.bgemm_encode(planes, ab, packed, wb, Mg, Ng, Kg, 1.0, nb, ns, qnn.RELU, out=out_d, ch_gamma=g_d, ch_beta=b_d)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_d.cpu().numpy(), y)
+    assert np.array_equal(nxt.cpu().numpy().view(np.uint32), want)
+    # affine only (no encoder)
+    out2 = torch.empty((Mg, Ng), dtype=torch.float32, device=dev)
+    qnn.bgemm_encode(planes, ab, packed, wb, Mg, Ng, Kg, 1.0, 0, 0.0, 0, out=out2, ch_gamma=g_d, ch_beta=b_d, encode=False)
+    torch.cuda.synchronize()
+    assert np.array_equal(out2.cpu().numpy(), y)
+
+
+@pytest.mark.parametrize("C,Cout", [(64, 70), (3, 64)])
+def test_bconv2d_affine(C, Cout):
+    torch, qnn, dev = _env()
+    rng = np.random.default_rng(C)
+    a = rng.standard_normal((2, 10, 9, C)).astype(np.float32)
+    w = (0.05 * rng.standard_normal((Cout, 3, 3, C))).astype(np.float32)
+    sa, sw, alpha = scales_for(a, w, 2, 2)
+    _, _, acc, out = oracle_conv(a, w, 2, 2, sa, sw, alpha, 1, 1)
+    gamma = rng.standard_normal(Cout).astype(np.float32)
+    beta = rng.standard_normal(Cout).astype(np.float32)
+    y = oracle.affine(out, gamma, beta)
+    ns = wl.per_tensor_scale(np.maximum(y, 0), 2)
+    want = oracle.pack_planes(oracle.quantize(y.reshape(-1, Cout), 2, ns, True), 2)
+    planes = qnn.encode_pack(torch.from_numpy(a).to(dev).view(-1, C), 2, sa)
+    packed = qnn.pack_weights(torch.from_numpy(w).to(dev), Cout, 9, C, qnn.W_NTC, 2, sw)
+    out_d = torch.empty(out.shape, dtype=torch.float32, device=dev)
+    nxt = qnn.bconv2d_encode(planes, 2, packed, 2, 2, 10, 9, C, Cout, 3, 3, 1, 1, alpha, 2, ns, qnn.RELU, out=out_d,
+                             ch_gamma=torch.from_numpy(gamma).to(dev), ch_beta=torch.from_numpy(beta).to(dev))
+    torch.cuda.synchronize()
+    assert np.array_equal(out_d.cpu().numpy(), y)
+    assert np.array_equal(nxt.cpu().numpy().view(np.uint32), want)

@@ -334,3 +334,26 @@ def test_conv_1x1_is_gemm_and_border_counts_valid_taps():
     ones = np.ones((1, 5, 5, 8), np.int16)
     acc = oracle.conv2d(ones, np.ones((1, 3, 3, 8), np.int16), 1, 1)[0, :, :, 0]
     assert acc[0, 0] == 8 * 4 and acc[0, 2] == 8 * 6 and acc[2, 2] == 8 * 9 and acc[4, 4] == 8 * 4
+
+
+# ----------------------------------------------------------------------------- per-feature affine
+
+def test_affine_exact_cases_and_single_rounding():
+    """Where the fused multiply-add is exact (small integers, power-of-two gains) the result is the integer
+    arithmetic; in general it is the correctly rounded value of y*gamma + beta, i.e. within half an ulp of the
+    float64 value and different from the twice-rounded product-then-sum where those differ."""
+    y = np.arange(-12, 12, dtype=np.float32).reshape(4, 6)
+    g = np.array([1, 2, 0.5, -4, 8, 0.25], dtype=np.float32)
+    b = np.array([0, 1, -3, 5, 0.5, -0.25], dtype=np.float32)
+    assert np.array_equal(oracle.affine(y, g, b), (y.astype(np.float64) * g + b).astype(np.float32))
+    assert np.array_equal(oracle.affine(y, g), (y.astype(np.float64) * g).astype(np.float32))
+    rng = np.random.default_rng(9)
+    y = rng.standard_normal((50, 33)).astype(np.float32) * 100
+    g = rng.standard_normal(33).astype(np.float32)
+    b = rng.standard_normal(33).astype(np.float32)
+    got = oracle.affine(y, g, b)
+    exact = y.astype(np.float64) * g.astype(np.float64) + b.astype(np.float64)
+    assert np.array_equal(got, exact.astype(np.float32))            # float64 holds the exact product: one rounding
+    twice = (y * g).astype(np.float32) + b
+    assert np.any(got != twice.astype(np.float32))                   # a plain multiply then add would differ somewhere
+    assert got.shape == y.shape and np.array_equal(y, y.copy())
