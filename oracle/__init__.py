@@ -60,6 +60,7 @@ def _load():
         lib.oracle_conv2d.argtypes = [p, p] + [c.c_int] * 9 + [p]
         lib.oracle_conv2d_sampled.argtypes = [p, p] + [c.c_int] * 9 + [c.c_size_t, p, p, p]
         lib.oracle_scale.argtypes = [p, c.c_size_t, c.c_float, p]
+        lib.oracle_conv2d_general.argtypes = [p, p] + [c.c_int] * 12 + [p]
         lib.oracle_affine.argtypes = [p, c.c_size_t, c.c_size_t, p, p]
         _lib = lib
     return _lib
@@ -182,3 +183,25 @@ def affine(y: np.ndarray, gamma: np.ndarray, beta: np.ndarray | None = None) -> 
     _check(_load().oracle_affine(_ptr(out), out.size // Ng, Ng, _ptr(gamma), _ptr(beta) if beta is not None else None),
            "affine")
     return out
+
+
+def conv_general_out_dim(size: int, k: int, stride: int, pad: int, dil: int, transposed: bool, out_pad: int = 0) -> int:
+    if not transposed:
+        return (size + 2 * pad - dil * (k - 1) - 1) // stride + 1
+    return (size - 1) * stride - 2 * pad + dil * (k - 1) + 1 + out_pad
+
+
+def conv2d_general(qa: np.ndarray, qw: np.ndarray, stride: int, pad: int, dil: int = 1, transposed: bool = False,
+                   out_pad: int = 0) -> np.ndarray:
+    """Dilated or transposed convolution of codes: qa [N,H,W,C], qw [Cout,R,S,C] -> int32 [N,Ho,Wo,Cout]."""
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    N, H, W, C = qa.shape
+    Cout, R, S, C2 = qw.shape
+    assert C == C2
+    Ho = conv_general_out_dim(H, R, stride, pad, dil, transposed, out_pad)
+    Wo = conv_general_out_dim(W, S, stride, pad, dil, transposed, out_pad)
+    acc = np.empty((N, Ho, Wo, Cout), dtype=np.int32)
+    _check(_load().oracle_conv2d_general(_ptr(qa), _ptr(qw), N, H, W, C, Cout, R, S, stride, pad, dil, int(transposed),
+                                         out_pad, _ptr(acc)), "conv2d_general")
+    return acc

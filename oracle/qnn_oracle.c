@@ -32,6 +32,7 @@
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -236,4 +237,78 @@ int oracle_affine(float *y, size_t rows, size_t Ng, const float *gamma, const fl
     for (ptrdiff_t m = 0; m < (ptrdiff_t)rows; ++m)
         for (size_t n = 0; n < Ng; ++n) y[(size_t)m * Ng + n] = fmaf(y[(size_t)m * Ng + n], gamma[n], beta ? beta[n] : 0.0f);
     return ORACLE_OK;
+}
+
+/*
+ * Convolution with dilation, and transposed convolution ("deconvolution", Section 3.2), on codes.
+ * Forward:     acc[n,ho,wo,co] = sum_{r,s,c} qa[n, ho*stride - pad + r*dil, wo*stride - pad + s*dil, c] * qw[co,r,s,c]
+ * Transposed:  every input pixel (hi, wi) adds qa[n,hi,wi,c]*qw[co,r,s,c] to output (hi*stride - pad + r*dil,
+ *              wi*stride - pad + s*dil); Ho = (H-1)*stride - 2*pad + dil*(R-1) + 1 + out_pad, Wo likewise.
+ * Positions outside the tensors contribute nothing (the encoded tensor is surrounded by, and for the transposed
+ * form interleaved with, true zeros).  The transposed form is written as the scatter it is defined by.
+ */
+int oracle_conv2d_general(const int16_t *qa, const int16_t *qw, int N, int H, int W, int C, int Cout, int R, int S,
+                          int stride, int pad, int dil, int transposed, int out_pad, int32_t *acc) {
+    if (!qa || !qw || !acc || stride < 1 || pad < 0 || dil < 1 || out_pad < 0) return ORACLE_E_ARG;
+    int Ho, Wo;
+    if (!transposed) {
+        Ho = (H + 2 * pad - dil * (R - 1) - 1) / stride + 1;
+        Wo = (W + 2 * pad - dil * (S - 1) - 1) / stride + 1;
+    } else {
+        Ho = (H - 1) * stride - 2 * pad + dil * (R - 1) + 1 + out_pad;
+        Wo = (W - 1) * stride - 2 * pad + dil * (S - 1) + 1 + out_pad;
+    }
+    if (Ho < 1 || Wo < 1) return ORACLE_E_ARG;
+    const size_t total = (size_t)N * Ho * Wo * Cout;
+    int64_t *wide = (int64_t *)calloc(total, sizeof(int64_t));
+    if (!wide) return ORACLE_E_ARG;
+    if (!transposed) {
+#pragma omp parallel for schedule(static)
+        for (ptrdiff_t m = 0; m < (ptrdiff_t)N * Ho * Wo; ++m) {
+            int n = (int)(m / ((ptrdiff_t)Ho * Wo)), ho = (int)((m / Wo) % Ho), wo = (int)(m % Wo);
+            for (int co = 0; co < Cout; ++co) {
+                int64_t sum = 0;
+                for (int r = 0; r < R; ++r) {
+                    int hi = ho * stride - pad + r * dil;
+                    if (hi < 0 || hi >= H) continue;
+                    for (int t = 0; t < S; ++t) {
+                        int wi = wo * stride - pad + t * dil;
+                        if (wi < 0 || wi >= W) continue;
+                        const int16_t *a = qa + (((size_t)n * H + hi) * W + wi) * C;
+                        const int16_t *w = qw + (((size_t)co * R + r) * S + t) * C;
+                        for (int c = 0; c < C; ++c) sum += (int64_t)a[c] * (int64_t)w[c];
+                    }
+                }
+                wide[(size_t)m * Cout + co] = sum;
+            }
+        }
+    } else {
+#pragma omp parallel for schedule(static)
+        for (ptrdiff_t n = 0; n < N; ++n)           /* images are independent; the scatter inside one is serial */
+            for (int hi = 0; hi < H; ++hi)
+                for (int wi = 0; wi < W; ++wi) {
+                    const int16_t *a = qa + (((size_t)n * H + hi) * W + wi) * C;
+                    for (int r = 0; r < R; ++r) {
+                        int ho = hi * stride - pad + r * dil;
+                        if (ho < 0 || ho >= Ho) continue;
+                        for (int t = 0; t < S; ++t) {
+                            int wo = wi * stride - pad + t * dil;
+                            if (wo < 0 || wo >= Wo) continue;
+                            for (int co = 0; co < Cout; ++co) {
+                                const int16_t *w = qw + (((size_t)co * R + r) * S + t) * C;
+                                int64_t sum = 0;
+                                for (int c = 0; c < C; ++c) sum += (int64_t)a[c] * (int64_t)w[c];
+                                wide[(((size_t)n * Ho + ho) * Wo + wo) * Cout + co] += sum;
+                            }
+                        }
+                    }
+                }
+    }
+    int bad = 0;
+    for (size_t i = 0; i < total; ++i) {
+        if (wide[i] > INT32_MAX || wide[i] < INT32_MIN) bad = 1;
+        acc[i] = (int32_t)wide[i];
+    }
+    free(wide);
+    return bad ? ORACLE_E_RANGE : ORACLE_OK;
 }

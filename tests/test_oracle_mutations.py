@@ -28,6 +28,9 @@ MUTATIONS = {
     "conv_tap_transposed": ("const int16_t *w = qw + (((size_t)co * R + r) * S + t) * C;", "const int16_t *w = qw + (((size_t)co * S + t) * R + r) * C;"),
     "conv_border_not_skipped": ("if (wi < 0 || wi >= W) continue;", "if (wi < 0) wi = 0; if (wi >= W) wi = W - 1;"),
     "conv_out_dim": ("return (in + 2 * pad - k) / stride + 1;", "return (in + 2 * pad - k + stride - 1) / stride + 1;"),
+    "dilation_ignored": ("int hi = ho * stride - pad + r * dil;\n                    if (hi < 0 || hi >= H) continue;", "int hi = ho * stride - pad + r;\n                    if (hi < 0 || hi >= H) continue;"),
+    "transposed_scatter_stride": ("int ho = hi * stride - pad + r * dil;", "int ho = hi - pad + r * dil;"),
+    "affine_twice_rounded": ("fmaf(y[(size_t)m * Ng + n], gamma[n], beta ? beta[n] : 0.0f);", "y[(size_t)m * Ng + n] * gamma[n] + (beta ? beta[n] : 0.0f);"),
     "scale_in_double": ("out[i] = (float)acc[i] * alpha;", "out[i] = (float)((double)acc[i] * (double)alpha * (1.0 + 1e-6));"),
 }
 

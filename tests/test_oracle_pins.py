@@ -357,3 +357,27 @@ def test_affine_exact_cases_and_single_rounding():
     twice = (y * g).astype(np.float32) + b
     assert np.any(got != twice.astype(np.float32))                   # a plain multiply then add would differ somewhere
     assert got.shape == y.shape and np.array_equal(y, y.copy())
+
+
+# ----------------------------------------------------------------------------- dilated / transposed convolution
+
+@pytest.mark.parametrize("N,H,W,C,Cout,R,S,stride,pad,dil,transposed,out_pad", [
+    (2, 9, 8, 5, 3, 3, 3, 1, 2, 2, False, 0), (1, 11, 11, 4, 6, 3, 3, 2, 1, 3, False, 0), (1, 7, 7, 3, 2, 3, 3, 1, 1, 1, False, 0),
+    (2, 5, 6, 4, 3, 3, 3, 2, 1, 1, True, 1), (1, 4, 4, 7, 5, 4, 4, 2, 1, 1, True, 0), (1, 6, 5, 3, 4, 3, 2, 3, 0, 1, True, 2),
+    (1, 5, 5, 2, 3, 3, 3, 2, 2, 2, True, 0), (2, 3, 3, 6, 2, 1, 1, 2, 0, 1, True, 1)])
+def test_general_conv_matches_torch(N, H, W, C, Cout, R, S, stride, pad, dil, transposed, out_pad):
+    import torch
+    rng = np.random.default_rng(H * 31 + C + stride)
+    qa = (2 * rng.integers(0, 8, size=(N, H, W, C)) - 7).astype(np.int16)
+    qw = (2 * rng.integers(0, 4, size=(Cout, R, S, C)) - 3).astype(np.int16)
+    acc = oracle.conv2d_general(qa, qw, stride, pad, dil, transposed, out_pad)
+    x = torch.from_numpy(qa.astype(np.float64)).permute(0, 3, 1, 2)
+    if not transposed:
+        wt = torch.from_numpy(qw.astype(np.float64)).permute(0, 3, 1, 2)                 # [Cout, C, R, S]
+        ref = torch.nn.functional.conv2d(x, wt, stride=stride, padding=pad, dilation=dil)
+        if dil == 1:
+            assert np.array_equal(acc, oracle.conv2d(qa, qw, stride, pad))
+    else:
+        wt = torch.from_numpy(qw.astype(np.float64)).permute(3, 0, 1, 2)                 # [C, Cout, R, S]
+        ref = torch.nn.functional.conv_transpose2d(x, wt, stride=stride, padding=pad, output_padding=out_pad, dilation=dil)
+    assert np.array_equal(acc.astype(np.float64), ref.permute(0, 2, 3, 1).numpy())
