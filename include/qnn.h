@@ -137,6 +137,22 @@ int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, 
                 void *stream);
 
 /*
+ * Dilated and transposed convolution on the same contraction (Section 3.2 names deconvolution layers next to
+ * convolution layers).  Arguments as qnn_bconv2d, plus
+ *   dilation    >= 1: tap (r, s) reads input (ho*stride - pad + r*dilation, wo*stride - pad + s*dilation)
+ *   transposed  != 0: transposed convolution ("deconvolution"): every input pixel (hi, wi) contributes through tap
+ *               (r, s) to output (hi*stride - pad + r*dilation, wi*stride - pad + s*dilation);
+ *               Ho = (H-1)*stride - 2*pad + dilation*(R-1) + 1 + out_pad, Wo likewise; w_packed holds the weights
+ *               as [Cout][R][S][Cin] of that scatter (no flipping is applied)
+ *   out_pad     extra rows/columns of a transposed convolution's output (0 otherwise; < max(stride, dilation))
+ * Forward: Ho = (H + 2*pad - dilation*(R-1) - 1)/stride + 1.  Positions outside the input (and, for the transposed
+ * form, the zeros between its pixels) contribute nothing.  QNN_E_RANGE for geometries outside the tiled kernel.
+ */
+int qnn_bconv2d_general(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
+                        int Cout, int R, int S, int stride, int pad, int dilation, int transposed, int out_pad,
+                        float alpha, float *out, int32_t *acc, void *stream);
+
+/*
  * Layer chaining (Alg. 1 forward: weighted branch sum, scale, then the next layer's MBitEncoder): the
  * contraction of qnn_bgemm / qnn_bconv2d whose epilogue can also apply a per-feature affine and quantize,
  * encode and bit-plane-pack its own fp32 result for the next layer, so that a stack of layers never

@@ -94,7 +94,8 @@ void fill_next(qnn_tiled::Params &p, const NextEnc *ne, int Ng) {
 int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
                float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream);
 int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
-               int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc, const NextEnc *ne, void *stream);
+               int R, int S, int stride, int pad, int dil, int transposed, int out_pad, float alpha, float *out,
+               int32_t *acc, const NextEnc *ne, void *stream);
 
 }  // namespace
 
@@ -106,7 +107,15 @@ extern "C" int qnn_bgemm(const uint32_t *a_planes, int ab, const void *w_packed,
 extern "C" int qnn_bconv2d(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C,
                            int Cout, int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc,
                            void *stream) {
-    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, alpha, out, acc, nullptr, stream);
+    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, 1, 0, 0, alpha, out, acc, nullptr,
+                      stream);
+}
+
+extern "C" int qnn_bconv2d_general(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W,
+                                   int C, int Cout, int R, int S, int stride, int pad, int dilation, int transposed,
+                                   int out_pad, float alpha, float *out, int32_t *acc, void *stream) {
+    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, dilation, transposed ? 1 : 0, out_pad,
+                      alpha, out, acc, nullptr, stream);
 }
 
 extern "C" int qnn_bgemm_encode(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng,
@@ -122,7 +131,8 @@ extern "C" int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *
                                   const float *ch_beta, int next_bits, float next_scale, unsigned next_flags,
                                   uint32_t *next_planes, float *out, void *stream) {
     const NextEnc ne = {next_planes, next_bits, next_scale, next_flags, ch_gamma, ch_beta};
-    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, alpha, out, nullptr, &ne, stream);
+    return bconv_impl(a_planes, ab, w_packed, wb, N, H, W, C, Cout, R, S, stride, pad, 1, 0, 0, alpha, out, nullptr, &ne,
+                      stream);
 }
 
 namespace {
@@ -148,24 +158,37 @@ int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     p.a_pitch = kw; p.w_pitch = kw; p.kwords = kw;
     p.n_elems = Kg; p.alpha = alpha; p.out = out; p.ldo = ldo; p.acc = acc;
     fill_next(p, ne, Ng);
-    return qnn_tiled::dispatch_tiled(false, ab, wb, p, st);
+    return qnn_tiled::dispatch_tiled(0, ab, wb, p, st);
 }
 
 int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
-               int R, int S, int stride, int pad, float alpha, float *out, int32_t *acc, const NextEnc *ne, void *stream) {
+               int R, int S, int stride, int pad, int dil, int transposed, int out_pad, float alpha, float *out,
+               int32_t *acc, const NextEnc *ne, void *stream) {
     if (!a_planes || !w_packed) return QNN_E_ARG;
     if (const int rc = check_next(ne)) return rc;
     if (!out && !acc && !(ne && ne->planes)) return QNN_E_ARG;
     if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || Cout <= 0 || R <= 0 || S <= 0 || stride <= 0 || pad < 0) return QNN_E_ARG;
+    if (dil < 1 || out_pad < 0 || (!transposed && out_pad != 0) || (transposed && out_pad >= stride && out_pad >= dil))
+        return QNN_E_ARG;
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb)) return QNN_E_ARG;
     if (!isfinite(alpha)) return QNN_E_SCALE;
     if (!qnn_aligned(a_planes, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(out, 4) || !qnn_aligned(acc, 4))
         return QNN_E_ALIGN;
     ConvGeom g;
     g.N = N; g.H = H; g.W = W; g.C = C; g.Cout = Cout; g.R = R; g.S = S; g.stride = stride; g.pad = pad;
-    g.Ho = (H + 2 * pad - R) / stride + 1;
-    g.Wo = (W + 2 * pad - S) / stride + 1;
-    if (H + 2 * pad < R || W + 2 * pad < S || g.Ho <= 0 || g.Wo <= 0) return QNN_E_ARG;
+    const int64_t ext_r = (int64_t)dil * (R - 1) + 1, ext_s = (int64_t)dil * (S - 1) + 1;   // extent of the dilated kernel
+    int64_t ho64, wo64;
+    if (!transposed) {
+        if (H + 2 * (int64_t)pad < ext_r || W + 2 * (int64_t)pad < ext_s) return QNN_E_ARG;
+        ho64 = (H + 2 * (int64_t)pad - ext_r) / stride + 1;
+        wo64 = (W + 2 * (int64_t)pad - ext_s) / stride + 1;
+    } else {
+        ho64 = ((int64_t)H - 1) * stride - 2 * (int64_t)pad + ext_r + out_pad;
+        wo64 = ((int64_t)W - 1) * stride - 2 * (int64_t)pad + ext_s + out_pad;
+    }
+    if (ho64 <= 0 || wo64 <= 0 || ho64 > 0x7fffffff || wo64 > 0x7fffffff) return QNN_E_ARG;
+    g.Ho = (int)ho64;
+    g.Wo = (int)wo64;
     g.cw = (C + 31) / 32;
     g.a_pitch = (int)qnn_row_words_i(C);
     g.w_pitch = (int)qnn_w_row_words_i(R * S, C);
@@ -175,7 +198,7 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    if (qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout)) {
+    if (dil == 1 && !transposed && qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout)) {
         qnn_dense::Params d = {};
         d.a = a_planes; d.w = w;
         d.tapsum = reinterpret_cast<const int32_t *>(w + (int64_t)Cout * wb * g.w_pitch);
@@ -201,9 +224,11 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
         p.n_elems = R * S * C; p.alpha = alpha; p.out = out; p.ldo = Cout; p.acc = acc;
         p.H = H; p.W = W; p.C = C; p.R = R; p.S = S; p.stride = stride; p.pad = pad; p.Ho = g.Ho; p.Wo = g.Wo;
         p.cw = g.cw; p.piece = (g.cw % 4 == 0) ? 4 : ((g.cw % 2 == 0) ? 2 : 1);
+        p.dil = dil; p.transposed = transposed;
         fill_next(p, ne, Cout);
-        return qnn_tiled::dispatch_tiled(true, ab, wb, p, st);
+        return qnn_tiled::dispatch_tiled((dil != 1 || transposed) ? 2 : 1, ab, wb, p, st);
     }
+    if (dil != 1 || transposed) return QNN_E_RANGE;      // the fallback kernel knows plain convolutions only
     dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));
     if (grid.y > 65535) return QNN_E_RANGE;
     if (ne && (!out || ne->gamma)) return QNN_E_ARG;   // the fallback kernel has no affine epilogue

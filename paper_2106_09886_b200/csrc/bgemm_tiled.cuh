@@ -50,6 +50,7 @@ struct Params {
     int32_t *acc;
     // convolution geometry
     int H, W, C, R, S, stride, pad, Ho, Wo, cw, piece;   // piece = words per copy (4, 2 or 1)
+    int dil, transposed;                                  // KIND 2 only: dilation (>= 1), transposed flag
     uint32_t cw_magic, s_magic;                           // x / d == (x * magic) >> 20 for the ranges used
     // optional per-feature affine applied after the scale: y = fma(y, ch_gamma[n], ch_beta[n]) (ch_beta may be NULL)
     const float *ch_gamma, *ch_beta;
@@ -85,6 +86,19 @@ __device__ __forceinline__ uint32_t lop3_carry_from_sum(uint32_t u, uint32_t v, 
     return d;
 }
 
+// Input coordinate read by tap index r of an output whose base coordinate is `base`, along one axis.
+// Forward convolution: base = o*stride - pad, coordinate base + r*dil.  Transposed convolution: base = o + pad,
+// the tap contributes only where (base - r*dil) is a non-negative multiple of the stride, coordinate = quotient.
+__device__ __forceinline__ bool tap_coord(const Params &p, int base, int r, int limit, int &pos) {
+    if (!p.transposed) {
+        pos = base + r * p.dil;
+        return pos >= 0 && pos < limit;
+    }
+    const int t = base - r * p.dil;
+    pos = (t >= 0) ? t / p.stride : 0;
+    return t >= 0 && pos * p.stride == t && pos < limit;
+}
+
 __device__ __forceinline__ void cp_async(uint32_t dst_smem, const void *src, int bytes_total, bool valid) {
     // 16-, 8- or 4-byte asynchronous copy; an invalid source is replaced by zeros (src-size 0)
     const int n = valid ? bytes_total : 0;
@@ -115,8 +129,11 @@ __device__ __forceinline__ void pair8(const uint32_t (&ta)[8], const uint32_t (&
     acc += __popc(fours) * (4 << shift);
 }
 
-template <int AB, int WB, bool CONV, int TM, bool FUSED>
+// KIND: 0 = fully-connected operand, 1 = convolution gather, 2 = dilated / transposed convolution gather (its
+// own instantiation: carrying that index arithmetic in the plain convolution cost it up to 15%).
+template <int AB, int WB, int KIND, int TM, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p) {
+    constexpr bool CONV = KIND != 0, GENERAL = KIND == 2;
     constexpr int kBM = 16 * TM;
     constexpr int A_UNITS = kBM * AB * kStageChunks;      // (row, plane, group) units per stage
     constexpr int W_UNITS = kBN * WB * kStageChunks;
@@ -158,8 +175,8 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             const int wo = (int)(mm % p.Wo);
             const int ho = (int)((mm / p.Wo) % p.Ho);
             const int64_t n = mm / ((int64_t)p.Wo * p.Ho);
-            t.h0 = ho * p.stride - p.pad;
-            t.w0 = wo * p.stride - p.pad;
+            t.h0 = (GENERAL && p.transposed) ? ho + p.pad : ho * p.stride - p.pad;
+            t.w0 = (GENERAL && p.transposed) ? wo + p.pad : wo * p.stride - p.pad;
             t.pixbase = n * p.H * p.W;
         }
 #pragma unroll
@@ -197,8 +214,12 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                         const int tap = (int)(((uint32_t)kw * p.cw_magic) >> 20);
                         const int cword = kw - tap * p.cw;
                         const int r = (int)(((uint32_t)tap * p.s_magic) >> 20), s = tap - r * p.S;
-                        const int hi = t.h0 + r, wi = t.w0 + s;
-                        const bool ok = t.a_ok && kw < p.kwords && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                        int hi = t.h0 + r, wi = t.w0 + s;
+                        bool ok = t.a_ok && kw < p.kwords && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                        if (GENERAL) {
+                            const bool okh = tap_coord(p, t.h0, r, p.H, hi), okw = tap_coord(p, t.w0, s, p.W, wi);
+                            ok = t.a_ok && kw < p.kwords && okh && okw;
+                        }
                         const uint32_t *src =
                             p.a + ((t.pixbase + (int64_t)hi * p.W + wi) * AB + a_plane) * p.a_pitch + cword;
                         const uint32_t dst = a_smem + a_dst0 + (uint32_t)((off >> 2) * AB * kBM * 16) + (uint32_t)(off & 3) * 4u;
@@ -359,15 +380,18 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 // AMAX * tapsum[n][tap] to S, and must not be counted in the length.
                 const int wo = (int)(m % p.Wo);
                 const int ho = (int)((m / p.Wo) % p.Ho);
-                const int hh = ho * p.stride - p.pad, ww = wo * p.stride - p.pad;
+                const int hh = (GENERAL && p.transposed) ? ho + p.pad : ho * p.stride - p.pad;
+                const int ww = (GENERAL && p.transposed) ? wo + p.pad : wo * p.stride - p.pad;
                 int valid_taps = p.R * p.S;
-                const bool interior = hh >= 0 && ww >= 0 && hh + p.R <= p.H && ww + p.S <= p.W;
+                const bool interior = !GENERAL && hh >= 0 && ww >= 0 && hh + p.R <= p.H && ww + p.S <= p.W;
                 if (!interior) {
                     valid_taps = 0;
                     for (int rr = 0; rr < p.R; ++rr)
                         for (int ss = 0; ss < p.S; ++ss) {
-                            const int hi = hh + rr, wi = ww + ss;
-                            if (hi >= 0 && hi < p.H && wi >= 0 && wi < p.W) {
+                            int hi = hh + rr, wi = ww + ss;
+                            bool inside = hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                            if (GENERAL) inside = tap_coord(p, hh, rr, p.H, hi) && tap_coord(p, ww, ss, p.W, wi);
+                            if (inside) {
                                 ++valid_taps;
                             } else {
 #pragma unroll
@@ -490,14 +514,17 @@ static __global__ void __launch_bounds__(kThreads, 2) probe_csa73_kernel(int ite
 }
 constexpr double kProbeCsa73WordsPerThreadIter = 8.0 * kStageChunks * 4 * 4 * 2 * 2;
 
-template <int AB, int WB, bool CONV, int TM, bool FUSED>
+template <int AB, int WB, int KIND, int TM, bool FUSED>
 inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st);
 
 // The epilogue with the next layer's encoder is a separate instantiation for ab <= 4, so that the plain kernels
 // carry none of its code; for ab >= 5 (16-row tiles, where the epilogue matters less) one instantiation serves both.
-template <int AB, int WB, bool CONV, int TM>
+template <int AB, int WB, int KIND, int TM>
 inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
-    if constexpr (AB >= 5) {
+    constexpr int CONV = KIND;
+    if constexpr (KIND == 2) {
+        return launch_tiled_tmf<AB, WB, KIND, TM, false>(p, sms, st);      // no chaining epilogue for this kind
+    } else if constexpr (AB >= 5) {
         return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
     } else {
         if (p.next_planes != nullptr || p.ch_gamma != nullptr) return launch_tiled_tmf<AB, WB, CONV, TM, true>(p, sms, st);
@@ -505,7 +532,7 @@ inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
     }
 }
 
-template <int AB, int WB, bool CONV, int TM, bool FUSED>
+template <int AB, int WB, int CONV, int TM, bool FUSED>
 inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     constexpr int kBM = 16 * TM;
     constexpr size_t smem = 2u * kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u;
@@ -536,7 +563,7 @@ inline double wave_efficiency(int64_t tiles, int64_t sms) {
     return (double)tiles / (double)(rounds * sms);
 }
 
-template <int AB, int WB, bool CONV>
+template <int AB, int WB, int CONV>
 inline int launch_tiled(const Params &p, cudaStream_t st) {
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -547,8 +574,10 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
         // operation but give twice as many tiles.  Take them only when that fills the SMs better (small problems).
         const int64_t tn = (p.Ng + kBN - 1) / kBN;
         const int64_t t64 = ((p.Mg + 63) / 64) * tn, t32 = ((p.Mg + 31) / 32) * tn;
-        if (p.next_planes == nullptr && p.ch_gamma == nullptr && wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
-            return launch_tiled_tmf<AB, WB, CONV, 2, false>(p, sms, st);   // (no fused instantiation of this variant)
+        if constexpr (CONV != 2) {
+            if (p.next_planes == nullptr && p.ch_gamma == nullptr && wave_efficiency(t32, sms) * 0.95 > wave_efficiency(t64, sms))
+                return launch_tiled_tmf<AB, WB, CONV, 2, false>(p, sms, st);   // (no fused instantiation of this variant)
+        }
         return launch_tiled_tm<AB, WB, CONV, 4>(p, sms, st);
     } else {
         return launch_tiled_tm<AB, WB, CONV, TileM<AB>::TM>(p, sms, st);
@@ -556,8 +585,8 @@ inline int launch_tiled(const Params &p, cudaStream_t st) {
 }
 
 // All weight widths for one activation width and operand kind; each (width, kind) is compiled in its own
-// translation unit (tiled_ab<N>_fc.cu / tiled_ab<N>_conv.cu) so that the kernel instantiations build in parallel.
-template <int AB, bool CONV>
+// translation unit (tiled_ab<N>_fc.cu / _conv.cu / _gconv.cu) so that the kernel instantiations build in parallel.
+template <int AB, int CONV>
 inline int run_tiled_ab(int wb, const Params &p, cudaStream_t st) {
 #define QNN_T(W_) \
     case W_: return launch_tiled<AB, W_, CONV>(p, st);
@@ -569,13 +598,16 @@ inline int run_tiled_ab(int wb, const Params &p, cudaStream_t st) {
 }
 #define QNN_DECL(N_) \
     int run_tiled_ab##N_##_fc(int wb, const Params &p, cudaStream_t st); \
-    int run_tiled_ab##N_##_conv(int wb, const Params &p, cudaStream_t st);
+    int run_tiled_ab##N_##_conv(int wb, const Params &p, cudaStream_t st); \
+    int run_tiled_ab##N_##_gconv(int wb, const Params &p, cudaStream_t st);
 QNN_DECL(1) QNN_DECL(2) QNN_DECL(3) QNN_DECL(4) QNN_DECL(5) QNN_DECL(6) QNN_DECL(7) QNN_DECL(8)
 #undef QNN_DECL
 
-inline int dispatch_tiled(bool conv, int ab, int wb, const Params &p, cudaStream_t st) {
+// kind: 0 = fully-connected, 1 = convolution, 2 = dilated / transposed convolution
+inline int dispatch_tiled(int kind, int ab, int wb, const Params &p, cudaStream_t st) {
 #define QNN_CASE(N_) \
-    case N_: return conv ? run_tiled_ab##N_##_conv(wb, p, st) : run_tiled_ab##N_##_fc(wb, p, st);
+    case N_: return kind == 2 ? run_tiled_ab##N_##_gconv(wb, p, st) \
+                  : kind == 1 ? run_tiled_ab##N_##_conv(wb, p, st) : run_tiled_ab##N_##_fc(wb, p, st);
     switch (ab) {
         QNN_CASE(1) QNN_CASE(2) QNN_CASE(3) QNN_CASE(4) QNN_CASE(5) QNN_CASE(6) QNN_CASE(7) QNN_CASE(8)
         default: return QNN_E_ARG;

@@ -2,5 +2,5 @@
 #include "bgemm_tiled.cuh"
 
 namespace qnn_tiled {
-int run_tiled_ab1_conv(int wb, const Params &p, cudaStream_t st) { return run_tiled_ab<1, true>(wb, p, st); }
+int run_tiled_ab1_conv(int wb, const Params &p, cudaStream_t st) { return run_tiled_ab<1, 1>(wb, p, st); }
 }  // namespace qnn_tiled

@@ -2,5 +2,5 @@
 #include "bgemm_tiled.cuh"
 
 namespace qnn_tiled {
-int run_tiled_ab3_fc(int wb, const Params &p, cudaStream_t st) { return run_tiled_ab<3, false>(wb, p, st); }
+int run_tiled_ab3_fc(int wb, const Params &p, cudaStream_t st) { return run_tiled_ab<3, 0>(wb, p, st); }
 }  // namespace qnn_tiled

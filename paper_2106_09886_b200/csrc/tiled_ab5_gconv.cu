@@ -1,0 +1,6 @@
+// Instantiations of the tiled contraction for 5-bit activations, dilated / transposed convolution operand (all weight widths).
+#include "bgemm_tiled.cuh"
+
+namespace qnn_tiled {
+int run_tiled_ab5_gconv(int wb, const Params &p, cudaStream_t st) { return run_tiled_ab<5, 2>(wb, p, st); }
+}  // namespace qnn_tiled

@@ -20,7 +20,7 @@ W_NTC, W_TCN, W_NCT = 0, 1, 2
 EXPORTS = [
     "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
-    "qnn_bgemm_encode", "qnn_bconv2d_encode",
+    "qnn_bgemm_encode", "qnn_bconv2d_encode", "qnn_bconv2d_general",
     "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -53,6 +53,7 @@ def _load() -> C.CDLL:
     lib.qnn_pack_weights.argtypes = [p, i, i, i, i, i, f, p, p]
     lib.qnn_bgemm.argtypes = [p, i, p, i, i64, i, i, f, p, i64, p, p]
     lib.qnn_bconv2d.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, p]
+    lib.qnn_bconv2d_general.argtypes = [p, i, p, i] + [i] * 12 + [f, p, p, p]
     lib.qnn_bgemm_encode.argtypes = [p, i, p, i, i64, i, i, f, p, p, i, f, u, p, p, i64, p]
     lib.qnn_bconv2d_encode.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, i, f, u, p, p, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
@@ -166,6 +167,30 @@ def bconv2d(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N:
         acc = torch.empty((N, Ho, Wo, Cout), dtype=torch.int32, device=a_planes.device)
     _check(lib.qnn_bconv2d(_ptr(a_planes), ab, _ptr(w_packed), wb, N, H, W, Cin, Cout, R, S, stride, pad,
                            float(alpha), _ptr(out), _ptr(acc), _stream(stream)), "qnn_bconv2d")
+    return (out, acc) if (want_acc or acc is not None) else out
+
+
+def conv_general_out_dim(size: int, k: int, stride: int, pad: int, dilation: int = 1, transposed: bool = False,
+                         out_pad: int = 0) -> int:
+    if not transposed:
+        return (size + 2 * pad - dilation * (k - 1) - 1) // stride + 1
+    return (size - 1) * stride - 2 * pad + dilation * (k - 1) + 1 + out_pad
+
+
+def bconv2d_general(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, N: int, H: int, W: int, Cin: int,
+                    Cout: int, R: int, S: int, stride: int, pad: int, dilation: int, transposed: bool, out_pad: int,
+                    alpha: float, out: torch.Tensor | None = None, acc: torch.Tensor | None = None,
+                    want_acc: bool = False, stream=None):
+    """Dilated or transposed convolution; out [N, Ho, Wo, Cout] with the output size of the chosen form."""
+    Ho = conv_general_out_dim(H, R, stride, pad, dilation, transposed, out_pad)
+    Wo = conv_general_out_dim(W, S, stride, pad, dilation, transposed, out_pad)
+    if out is None:
+        out = torch.empty((N, Ho, Wo, Cout), dtype=torch.float32, device=a_planes.device)
+    if acc is None and want_acc:
+        acc = torch.empty((N, Ho, Wo, Cout), dtype=torch.int32, device=a_planes.device)
+    _check(lib.qnn_bconv2d_general(_ptr(a_planes), ab, _ptr(w_packed), wb, N, H, W, Cin, Cout, R, S, stride, pad,
+                                   dilation, int(transposed), out_pad, float(alpha), _ptr(out), _ptr(acc),
+                                   _stream(stream)), "qnn_bconv2d_general")
     return (out, acc) if (want_acc or acc is not None) else out
 
 
