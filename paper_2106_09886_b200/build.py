@@ -4,6 +4,7 @@
 """
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
@@ -14,6 +15,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 INCLUDE = PKG.parent / "include"
 LIB = PKG / "libqnn.so"
+STAMP = PKG / "libqnn.so.digest"
 
 COMPILE_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -27,12 +29,18 @@ def sources() -> list[Path]:
     return sorted(CSRC.glob("*.cu"))
 
 
+def _digest() -> str:
+    """Content digest of everything the library is built from (file times do not survive copies of the tree)."""
+    h = hashlib.sha256()
+    h.update(" ".join(COMPILE_FLAGS + LINK_FLAGS).encode())
+    for path in sources() + sorted(CSRC.glob("*.cuh")) + sorted(INCLUDE.glob("*.h")):
+        h.update(path.name.encode())
+        h.update(path.read_bytes())
+    return h.hexdigest()
+
+
 def needs_build() -> bool:
-    if not LIB.exists():
-        return True
-    t = LIB.stat().st_mtime
-    deps = sources() + sorted(CSRC.glob("*.cuh")) + sorted(INCLUDE.glob("*.h")) + [Path(__file__)]
-    return any(p.stat().st_mtime > t for p in deps)
+    return not LIB.exists() or not STAMP.exists() or STAMP.read_text().strip() != _digest()
 
 
 def _compile(nvcc: str, src: Path, obj: Path, verbose: bool) -> str:
@@ -62,6 +70,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
     subprocess.check_call([nvcc, *LINK_FLAGS, "-o", str(tmp), *map(str, objs)])
     os.replace(tmp, LIB)
+    STAMP.write_text(_digest() + "\n")
     return LIB
 
 
