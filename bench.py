@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the {-1,+1} bit-plane decomposed quantized layer on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--report FILE]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-cpu-baseline]
 
 One step = one pass of the whole hot path over one batch of synthetic input:
 qnn_encode_pack (fp32 activations -> bit planes) followed by qnn_bgemm (all plane pairs,
@@ -47,7 +47,7 @@ POPC_PER_WORD = 0.5   # popcounts the tiled kernel issues per 32-bit xor word (7
 
 # DRAM read+write of one qnn_bgemm 4096^3 w2a2 launch from the ncu capture summarised in
 # profiles/bgemm_tiled_4096_w2a2.md, valid for the kernel source with this digest only.
-NCU_TRAFFIC = {"bytes": 22787840, "kernel_sha256": "86278b5f1cca1f4216f8206c86dcaf6814e2a15db33e49991d399cc420da205b"}
+NCU_TRAFFIC = {"bytes": 22488576, "kernel_sha256": "2bd69f3e19783a228f44af9cc4a99c9ec0e66f5d75c1badbcd4689e0c4648963"}
 
 
 def ncu_traffic_bytes():
