@@ -161,3 +161,30 @@ def test_fc_forward_host_pipelined_matches_oracle():
     qnn.fc_forward_host_pipelined(x_host, 3, sa, 0, packed, 2, 130, alpha, out_host, x_dev, planes, out_dev, 192, streams)
     torch.cuda.synchronize()
     assert_fp32_close(out_host.numpy(), out)
+
+
+def test_bgemm_output_beyond_2g_elements():
+    """More than 2^31 outputs (8.8 GB of fp32): exercises the 64-bit output indexing.  The oracle evaluates sampled
+    entries, among them the very last rows."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    if torch.cuda.get_device_properties(dev).total_memory < 40 * 2 ** 30:
+        pytest.skip("needs about 10 GB of device memory")
+    Mg, Ng, Kg, ab, wb = 2_200_000, 1000, 32, 2, 2
+    assert Mg * Ng > 2 ** 31
+    rng = np.random.default_rng(31)
+    a = rng.standard_normal((Mg, Kg), dtype=np.float32)
+    w = rng.standard_normal((Ng, Kg), dtype=np.float32)
+    sa, sw, alpha = scales_for(a, w, ab, wb)
+    qa, qw = oracle_fc_codes(a, w, False, ab, wb, sa, sw)
+    planes = qnn.encode_pack(torch.from_numpy(a).to(dev), ab, sa)
+    packed = qnn.pack_weights(torch.from_numpy(w).to(dev), Ng, 1, Kg, qnn.W_NTC, wb, sw)
+    out = qnn.bgemm(planes, ab, packed, wb, Mg, Ng, Kg, alpha)
+    rows = np.concatenate([rng.integers(0, Mg, size=200000), np.full(1000, Mg - 1), np.full(1000, 2 ** 31 // Ng + 1)])
+    cols = np.concatenate([rng.integers(0, Ng, size=200000), np.arange(1000), np.arange(1000)])
+    idx = torch.from_numpy(rows.astype(np.int64) * Ng + cols.astype(np.int64)).to(dev)
+    got = out.view(-1)[idx].cpu().numpy()
+    del out
+    want = oracle.scale(oracle.fc_sampled(qa, qw, rows, cols), alpha)
+    assert_fp32_close(got, want)
