@@ -85,7 +85,12 @@ def time_stack(net: str, batch: int, reps=3, warmup=2, dev="cuda:0", seed=0, lay
     """Every quantized convolution of a ResNet-18- or VGG-16-shaped stack, each on its own synthetic
     input of the right shape (post-ReLU half-normal), timed as qnn_encode_pack + qnn_bconv2d."""
     from . import workloads as wl
-    shapes = wl.resnet18_shapes(batch) if net == "resnet18" else wl.vgg16_shapes(batch)
+    if net == "resnet18":
+        shapes = wl.resnet18_shapes(batch)
+    elif net in ("resnet18_p1", "resnet18_p2"):
+        shapes = wl.resnet18_mixed_shapes(int(net[-1]), batch)     # Table 4's mixed precisions
+    else:
+        shapes = wl.vgg16_shapes(batch)
     g = torch.Generator(device=dev).manual_seed(seed)
     rows = []
     for li, s in enumerate(shapes):
@@ -145,7 +150,7 @@ def main():
     for name, default in (("rows", 4096), ("k", 4096), ("bits", 2)):
         e.add_argument(f"--{name}", type=int, default=default)
     k = sub.add_parser("stack")
-    k.add_argument("--net", choices=["resnet18", "vgg16"], default="resnet18")
+    k.add_argument("--net", choices=["resnet18", "resnet18_p1", "resnet18_p2", "vgg16"], default="resnet18")
     k.add_argument("--batch", type=int, default=0)
     k.add_argument("--layers", type=str, default="")
     k.add_argument("--table", action="store_true")
@@ -159,7 +164,7 @@ def main():
     elif a.case == "conv":
         r = time_conv(a.N, a.H, a.W, a.C, a.Cout, a.R, a.S, a.stride, a.pad, a.ab, a.wb, a.reps, a.warmup, a.sets)
     elif a.case == "stack":
-        batch = a.batch or (256 if a.net == "resnet18" else 64)
+        batch = a.batch or (64 if a.net == "vgg16" else 256)
         layers = [int(v) for v in a.layers.split(",")] if a.layers else None
         r = time_stack(a.net, batch, a.reps, a.warmup, layers=layers)
         if a.table:

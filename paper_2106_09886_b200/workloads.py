@@ -140,6 +140,41 @@ def resnet18_shapes(batch: int = 256, ab: int = 3, wb: int = 3) -> list[ConvShap
     return L
 
 
+# Per-stage bit widths of the paper's mixed-precision ResNet-18 (Table 4): (activation bits M, weight bits K)
+# for Conv2_x .. Conv5_x; the stem (Conv1) and the FC layer stay outside the library (their widths only enter
+# the compression ratio).
+RESNET18_MIXED = {
+    1: {"stem_wb": 8, "stages": [(8, 8), (8, 7), (8, 7), (8, 6)], "fc_wb": 8, "compression": 5.0},
+    2: {"stem_wb": 8, "stages": [(4, 5), (4, 3), (4, 2), (4, 2)], "fc_wb": 6, "compression": 14.1},
+}
+
+
+def resnet18_mixed_shapes(precision: int, batch: int = 256) -> list[ConvShape]:
+    """The ResNet-18-shaped stack with the per-stage (activation, weight) widths of Table 4, Precision#1 or #2."""
+    stages = RESNET18_MIXED[precision]["stages"]
+    out = []
+    for s in resnet18_shapes(batch):
+        stage = int(s.name[1]) - 1                      # names start with s<stage>
+        ab, wb = stages[stage]
+        out.append(ConvShape(s.name + f"_a{ab}w{wb}", s.N, s.H, s.W, s.C, s.Cout, s.R, s.S, s.stride, s.pad, ab, wb,
+                             branch=s.branch))
+    return out
+
+
+def resnet18_weight_bits(precision: int) -> tuple[int, int]:
+    """(bits of all weights at the table's widths, bits at fp32) for the whole ResNet-18: 7x7 stem, the 19
+    quantized convolutions, and the 512x1000 FC layer (biases and normalisation parameters not counted)."""
+    cfg = RESNET18_MIXED[precision]
+    stem, fc = 7 * 7 * 3 * 64, 512 * 1000
+    q = stem * cfg["stem_wb"] + fc * cfg["fc_wb"]
+    n = stem + fc
+    for s in resnet18_mixed_shapes(precision, batch=1):
+        params = s.Cout * s.R * s.S * s.C
+        q += params * s.wb
+        n += params
+    return q, 32 * n
+
+
 def vgg16_shapes(batch: int = 64, ab: int = 4, wb: int = 4) -> list[ConvShape]:
     """13 3x3 stride-1 pad-1 convolutions of a VGG-16-shaped stack at 224x224x3, 2x2 max-pool after each block."""
     cfg = [(64, 2), (128, 2), (256, 3), (512, 3), (512, 3)]

@@ -106,3 +106,26 @@ def test_workloads_are_seeded_and_shaped():
     v = wl.vgg16_shapes()
     assert len(v) == 13 and sum(s.int_macs for s in v) // 10 ** 9 == 982
     assert v[0].Kg == 27 and v[0].Mg == 3211264
+
+
+def test_mixed_precision_resnet18_reproduces_table4_compression():
+    """Table 4: per-stage widths of Precision#1 / #2 give 5.0x / 14.1x weight compression with one bit per
+    element per plane; the packed blobs of the quantized convolutions hold those plane bits, each (feature, plane)
+    row rounded up to 16 bytes, plus the per-tap sums."""
+    from paper_2106_09886_b200 import workloads as wl
+    for precision, want in ((1, 5.0), (2, 14.1)):
+        q, full = wl.resnet18_weight_bits(precision)
+        assert abs(full / q - want) < 0.06, (precision, full / q)
+        assert wl.RESNET18_MIXED[precision]["compression"] == want
+    from paper_2106_09886_b200 import build
+    build.build()
+    from paper_2106_09886_b200 import qnn
+    tot_ideal = tot_rows = 0
+    for s in wl.resnet18_mixed_shapes(2, batch=1):
+        ideal = s.Cout * s.R * s.S * s.C * s.wb // 8
+        row = (s.R * s.S * s.C // 32 + 3) // 4 * 4 * 4                     # bytes of one (feature, plane) row
+        got = qnn.weights_bytes(s.Cout, s.R * s.S, s.C, s.wb)
+        assert got == s.Cout * s.wb * row + (s.Cout * s.R * s.S * 4 + 15) // 16 * 16
+        tot_ideal += ideal
+        tot_rows += s.Cout * s.wb * row
+    assert tot_ideal <= tot_rows <= 1.01 * tot_ideal      # row padding costs under 1% over the whole network

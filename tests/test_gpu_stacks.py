@@ -132,3 +132,9 @@ def test_resnet18_stack_chained_batch2():
 
 def test_vgg16_stack_chained_batch2():
     chain(wl.vgg16_shapes(batch=2), 5, first_signed=True)
+
+
+@pytest.mark.parametrize("precision", [1, 2])
+def test_resnet18_mixed_precision_chained_batch2(precision):
+    """Table 4's mixed precisions (8x8, 8x7, 8x6 / 4x5, 4x3, 4x2 bits per stage), whole stack chained at batch 2."""
+    chain(reorder_branches(wl.resnet18_mixed_shapes(precision, batch=2)), 40 + precision, first_signed=False)
