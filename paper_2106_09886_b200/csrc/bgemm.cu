@@ -226,7 +226,11 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
         p.cw = g.cw; p.piece = (g.cw % 4 == 0) ? 4 : ((g.cw % 2 == 0) ? 2 : 1);
         p.dil = dil; p.transposed = transposed;
         fill_next(p, ne, Cout);
-        return qnn_tiled::dispatch_tiled((dil != 1 || transposed) ? 2 : 1, ab, wb, p, st);
+        int kind = (dil != 1 || transposed) ? 2 : 1;
+        // nine taps and at most 4 channel words: 9-word groups leave no reduction tail (9% faster at C = 64, 128);
+        // for more channels the tail is negligible and the 16-byte copies of the 8-word path win
+        if (kind == 1 && R * S == 9 && g.cw <= 4 && ab <= 4 && wb <= 4) kind = 3;
+        return qnn_tiled::dispatch_tiled(kind, ab, wb, p, st);
     }
     if (dil != 1 || transposed) return QNN_E_RANGE;      // the fallback kernel knows plain convolutions only
     dim3 grid((unsigned)qnn_ceil_div(Cout, 16), (unsigned)qnn_ceil_div(Mg, 16));

@@ -129,17 +129,39 @@ __device__ __forceinline__ void pair8(const uint32_t (&ta)[8], const uint32_t (&
     acc += __popc(fours) * (4 << shift);
 }
 
-// KIND: 0 = fully-connected operand, 1 = convolution gather, 2 = dilated / transposed convolution gather (its
+// Nine re-coded words [x0, x1, x0^x1^x2, x3, x4, x3^x4^x5, x6, x7, x6^x7^x8] of one (output, plane pair):
+// three 3:2 counters, a fourth on their sums and one on their carries: 12 xors/logic ops + 4 three-input
+// ops, 4 popcounts (ones, two words of weight 2, fours).  Used where the reduction is a multiple of 9 words
+// (3x3 convolutions, one group = one channel word of all nine taps), which then has no tail.
+__device__ __forceinline__ void pair9(const uint32_t (&ta)[9], const uint32_t (&tw)[9], const int shift, int &acc) {
+    const uint32_t u1 = ta[0] ^ tw[0], v1 = ta[1] ^ tw[1], s1 = ta[2] ^ tw[2];
+    const uint32_t c1 = lop3_carry_from_sum(u1, v1, s1);
+    const uint32_t u2 = ta[3] ^ tw[3], v2 = ta[4] ^ tw[4], s2 = ta[5] ^ tw[5];
+    const uint32_t c2 = lop3_carry_from_sum(u2, v2, s2);
+    const uint32_t u3 = ta[6] ^ tw[6], v3 = ta[7] ^ tw[7], s3 = ta[8] ^ tw[8];
+    const uint32_t c3 = lop3_carry_from_sum(u3, v3, s3);
+    const uint32_t ones = lop3_xor3(s1, s2, s3), c4 = lop3_maj(s1, s2, s3);
+    const uint32_t twos = lop3_xor3(c1, c2, c3), fours = lop3_maj(c1, c2, c3);
+    acc += __popc(ones) * (1 << shift);
+    acc += __popc(twos) * (2 << shift);
+    acc += __popc(c4) * (2 << shift);
+    acc += __popc(fours) * (4 << shift);
+}
+
+// KIND: 0 = fully-connected operand, 1 = convolution gather, 3 = 3x3 convolution gather with 9-word groups, 2 = dilated / transposed convolution gather (its
 // own instantiation: carrying that index arithmetic in the plain convolution cost it up to 15%).
 template <int AB, int WB, int KIND, int TM, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p) {
-    constexpr bool CONV = KIND != 0, GENERAL = KIND == 2;
+    constexpr bool CONV = KIND != 0, GENERAL = KIND == 2, G9 = KIND == 3;
     constexpr int kBM = 16 * TM;
     constexpr int A_UNITS = kBM * AB * kStageChunks;      // (row, plane, group) units per stage
     constexpr int W_UNITS = kBN * WB * kStageChunks;
     constexpr int A_VEC = kStageChunks * 2 * AB * kBM;    // uint4 per stage, A region
     constexpr int W_VEC = kStageChunks * 2 * WB * kBN;
-    extern __shared__ uint4 smem[];                       // [2 buffers][A_VEC + W_VEC]
+    // G9 keeps the ninth word of every group in a separate uint32 region [group slot][plane][row] per operand
+    constexpr int A_EXT = kStageChunks * AB * kBM, W_EXT = kStageChunks * WB * kBN;          // words
+    constexpr int BUF_VEC = A_VEC + W_VEC + (G9 ? (A_EXT + W_EXT + 3) / 4 : 0);             // uint4 per buffer
+    extern __shared__ uint4 smem[];                       // [2 buffers][BUF_VEC]
     const int tid = threadIdx.x;
     const int tx = tid & 15, ty = tid >> 4;
     const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
@@ -190,8 +212,44 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
 
     // Copies stage `stage` of the tile described by `t` into buffer `buf` (asynchronously; one commit group).
     auto issue_stage = [&](const TileSrc &t, int stage, int buf) {
-        const uint32_t a_smem = smem_base + (uint32_t)buf * (A_VEC + W_VEC) * 16u;
+        const uint32_t a_smem = smem_base + (uint32_t)buf * BUF_VEC * 16u;
         const uint32_t w_smem = a_smem + A_VEC * 16u;
+        if constexpr (G9) {
+            // group gi = channel word gi of all nine taps: nine 4-byte copies per (row, plane) unit
+            const uint32_t a_ext = a_smem + (uint32_t)(A_VEC + W_VEC) * 16u, w_ext = a_ext + (uint32_t)A_EXT * 4u;
+            if (a_unit) {
+                const int gi = stage * kStageChunks + a_ch;
+                if (gi < p.nfull) {
+#pragma unroll
+                    for (int tap = 0; tap < 9; ++tap) {
+                        const int r = (int)(((uint32_t)tap * p.s_magic) >> 20), sx = tap - r * p.S;
+                        const int hi = t.h0 + r, wi = t.w0 + sx;
+                        const bool ok = t.a_ok && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
+                        const uint32_t *src = p.a + ((t.pixbase + (int64_t)hi * p.W + wi) * AB + a_plane) * p.a_pitch + gi;
+                        const uint32_t dst = tap < 8 ? a_smem + a_dst0 + (uint32_t)((tap >> 2) * AB * kBM * 16 + (tap & 3) * 4)
+                                                     : a_ext + (uint32_t)(((a_ch * AB + a_plane) * kBM + srow) * 4);
+                        cp_async(dst, ok ? (const void *)src : (const void *)p.a, 4, ok);
+                    }
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < W_Q; ++q) {
+                const int u = tid + q * kThreads;
+                if ((W_UNITS % kThreads) != 0 && u >= W_UNITS) break;
+                const int rp = u % (kBN * WB), ch = u / (kBN * WB);
+                const int plane = rp / kBN;
+                const int gi = stage * kStageChunks + ch;
+                if (gi >= p.nfull) continue;
+#pragma unroll
+                for (int tap = 0; tap < 9; ++tap) {
+                    const uint32_t dst = tap < 8 ? w_smem + (uint32_t)((((ch * 2 + (tap >> 2)) * WB + plane) * kBN + wrow) * 16 + (tap & 3) * 4)
+                                                 : w_ext + (uint32_t)(((ch * WB + plane) * kBN + wrow) * 4);
+                    cp_async(dst, t.w_ok ? (const void *)(t.w[q] + tap * p.cw + gi) : (const void *)p.w, 4, t.w_ok);
+                }
+            }
+            cp_async_commit();
+            return;
+        }
         if (a_unit) {
             const int gi = stage * kStageChunks + a_ch;
             if (gi < ngroups) {
@@ -252,7 +310,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
 
     // re-code the full groups this thread copied: [x0..x7] -> [x0, x1, x0^x1^x2, x3, x4, x3^x4^x5, x0^..^x6, x7]
     auto recode_stage = [&](int stage, int buf) {
-        uint4 *a_s = smem + (size_t)buf * (A_VEC + W_VEC);
+        uint4 *a_s = smem + (size_t)buf * BUF_VEC;
         uint4 *w_s = a_s + A_VEC;
         auto recode = [](uint4 *lo, uint4 *hi) {
             uint4 x = *lo, y = *hi;
@@ -262,6 +320,31 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             *lo = make_uint4(x.x, x.y, t2, x.w);
             *hi = make_uint4(y.x, t5, t6, y.w);
         };
+        if constexpr (G9) {
+            // [x0..x8] -> [x0, x1, x0^x1^x2, x3, x4, x3^x4^x5, x6, x7, x6^x7^x8]
+            uint32_t *a_e = reinterpret_cast<uint32_t *>(a_s + A_VEC + W_VEC), *w_e = a_e + A_EXT;
+            auto recode9 = [](uint4 *lo, uint4 *hi, uint32_t *ext) {
+                uint4 x = *lo, y = *hi;
+                const uint32_t x8 = *ext;
+                *lo = make_uint4(x.x, x.y, lop3_xor3(x.x, x.y, x.z), x.w);
+                *hi = make_uint4(y.x, lop3_xor3(x.w, y.x, y.y), y.z, y.w);
+                *ext = lop3_xor3(y.z, y.w, x8);
+            };
+            if (a_unit && stage * kStageChunks + a_ch < p.nfull)
+                recode9(a_s + ((a_ch * 2 + 0) * AB + a_plane) * kBM + srow, a_s + ((a_ch * 2 + 1) * AB + a_plane) * kBM + srow,
+                        a_e + (a_ch * AB + a_plane) * kBM + srow);
+#pragma unroll
+            for (int q = 0; q < W_Q; ++q) {
+                const int u = tid + q * kThreads;
+                if ((W_UNITS % kThreads) != 0 && u >= W_UNITS) break;
+                const int rp = u % (kBN * WB), ch = u / (kBN * WB);
+                const int plane = rp / kBN;
+                if (stage * kStageChunks + ch >= p.nfull) continue;
+                recode9(w_s + ((ch * 2 + 0) * WB + plane) * kBN + wrow, w_s + ((ch * 2 + 1) * WB + plane) * kBN + wrow,
+                        w_e + (ch * WB + plane) * kBN + wrow);
+            }
+            return;
+        }
         if (a_unit && stage * kStageChunks + a_ch < p.nfull)
             recode(a_s + ((a_ch * 2 + 0) * AB + a_plane) * kBM + srow, a_s + ((a_ch * 2 + 1) * AB + a_plane) * kBM + srow);
 #pragma unroll
@@ -301,40 +384,49 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 issue_stage(cur, 0, buf ^ 1);                                    // overlaps the epilogue too
             }
 
-            const uint4 *a_s = smem + (size_t)buf * (A_VEC + W_VEC);
+            const uint4 *a_s = smem + (size_t)buf * BUF_VEC;
             const uint4 *w_s = a_s + A_VEC;
             int nch = p.nfull - stage * kStageChunks;
             nch = nch > kStageChunks ? kStageChunks : nch;
+            constexpr int GW = G9 ? 9 : 8;                                   // words per group
+            const uint32_t *a_e = reinterpret_cast<const uint32_t *>(a_s + A_VEC + W_VEC);   // G9: ninth words
+            const uint32_t *w_e = a_e + A_EXT;
 #pragma unroll 1
             for (int ch = 0; ch < nch; ++ch) {
-                uint32_t ta[TM][AB][8];
+                uint32_t ta[TM][AB][GW];
 #pragma unroll
                 for (int r = 0; r < TM; ++r)
 #pragma unroll
-                    for (int i = 0; i < AB; ++i)
+                    for (int i = 0; i < AB; ++i) {
 #pragma unroll
                         for (int g = 0; g < 2; ++g) {
                             const uint4 v = a_s[((ch * 2 + g) * AB + i) * kBM + ty + 16 * r];
                             ta[r][i][4 * g + 0] = v.x; ta[r][i][4 * g + 1] = v.y;
                             ta[r][i][4 * g + 2] = v.z; ta[r][i][4 * g + 3] = v.w;
                         }
+                        if constexpr (G9) ta[r][i][GW - 1] = a_e[(ch * AB + i) * kBM + ty + 16 * r];
+                    }
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int j = 0; j < WB; ++j) {
-                        uint32_t tw[8];
+                        uint32_t tw[GW];
 #pragma unroll
                         for (int g = 0; g < 2; ++g) {
                             const uint4 v = w_s[((ch * 2 + g) * WB + j) * kBN + tx + 16 * c];
                             tw[4 * g + 0] = v.x; tw[4 * g + 1] = v.y; tw[4 * g + 2] = v.z; tw[4 * g + 3] = v.w;
                         }
+                        if constexpr (G9) tw[GW - 1] = w_e[(ch * WB + j) * kBN + tx + 16 * c];
 #pragma unroll
                         for (int r = 0; r < TM; ++r)
 #pragma unroll
-                            for (int i = 0; i < AB; ++i) pair8(ta[r][i], tw, i + j, acc[r][c]);
+                            for (int i = 0; i < AB; ++i) {
+                                if constexpr (G9) pair9(ta[r][i], tw, i + j, acc[r][c]);
+                                else pair8(ta[r][i], tw, i + j, acc[r][c]);
+                            }
                     }
             }
-            if (p.ntail > 0 && stage == p.nstages - 1) {
+            if (!G9 && p.ntail > 0 && stage == p.nstages - 1) {
                 const int ch = p.nfull % kStageChunks;
                 // tail: up to 3 raw words, one popcount each (words past kwords are zero in both operands)
                 uint32_t ta[TM][AB][3];
@@ -535,7 +627,8 @@ inline int launch_tiled_tm(const Params &p, int sms, cudaStream_t st) {
 template <int AB, int WB, int CONV, int TM, bool FUSED>
 inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     constexpr int kBM = 16 * TM;
-    constexpr size_t smem = 2u * kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u;
+    constexpr size_t ext = (CONV == 3) ? ((size_t)kStageChunks * (AB * kBM + WB * kBN) + 3u) / 4u * 16u : 0u;   // ninth words
+    constexpr size_t smem = 2u * (kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u + ext);
     if (smem > 48u * 1024u &&
         cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV, TM, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
@@ -545,7 +638,13 @@ inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     if (tiles_m * tiles_n > 0x7fffffff) return QNN_E_RANGE;
     q.tiles_m = (int)tiles_m;
     q.ntiles = (int)(tiles_m * tiles_n);
-    set_k_split(q);
+    if (CONV == 3) {               // one 9-word group per channel word, no tail
+        q.nfull = q.cw;
+        q.ntail = 0;
+        q.nstages = (q.cw + kStageChunks - 1) / kStageChunks;
+    } else {
+        set_k_split(q);
+    }
     // Short reductions: two persistent CTAs per SM walk the tiles and prefetch across tile boundaries, which
     // hides the first-stage latency that would otherwise dominate.  Long reductions: one CTA per tile measured
     // about 5% faster (the hardware's dynamic block placement balances better than the static walk).
@@ -600,11 +699,25 @@ inline int run_tiled_ab(int wb, const Params &p, cudaStream_t st) {
     int run_tiled_ab##N_##_fc(int wb, const Params &p, cudaStream_t st); \
     int run_tiled_ab##N_##_conv(int wb, const Params &p, cudaStream_t st); \
     int run_tiled_ab##N_##_gconv(int wb, const Params &p, cudaStream_t st);
+// 3x3 convolutions with 9-word groups (kind 3) exist for ab, wb <= 4
+int run_tiled_conv3x3_ab1(int wb, const Params &p, cudaStream_t st);
+int run_tiled_conv3x3_ab2(int wb, const Params &p, cudaStream_t st);
+int run_tiled_conv3x3_ab3(int wb, const Params &p, cudaStream_t st);
+int run_tiled_conv3x3_ab4(int wb, const Params &p, cudaStream_t st);
 QNN_DECL(1) QNN_DECL(2) QNN_DECL(3) QNN_DECL(4) QNN_DECL(5) QNN_DECL(6) QNN_DECL(7) QNN_DECL(8)
 #undef QNN_DECL
 
-// kind: 0 = fully-connected, 1 = convolution, 2 = dilated / transposed convolution
+// kind: 0 = fully-connected, 1 = convolution, 2 = dilated / transposed convolution, 3 = 3x3 convolution (ab, wb <= 4)
 inline int dispatch_tiled(int kind, int ab, int wb, const Params &p, cudaStream_t st) {
+    if (kind == 3) {
+        switch (ab) {
+            case 1: return run_tiled_conv3x3_ab1(wb, p, st);
+            case 2: return run_tiled_conv3x3_ab2(wb, p, st);
+            case 3: return run_tiled_conv3x3_ab3(wb, p, st);
+            case 4: return run_tiled_conv3x3_ab4(wb, p, st);
+            default: return QNN_E_ARG;
+        }
+    }
 #define QNN_CASE(N_) \
     case N_: return kind == 2 ? run_tiled_ab##N_##_gconv(wb, p, st) \
                   : kind == 1 ? run_tiled_ab##N_##_conv(wb, p, st) : run_tiled_ab##N_##_fc(wb, p, st);
