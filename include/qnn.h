@@ -51,7 +51,7 @@ typedef enum qnn_status {
     QNN_E_RANGE = -3,  /* Kg*A*B does not fit int32, or an index does not fit the kernels' 32-bit tile arithmetic */
     QNN_E_SCALE = -4,  /* scale outside [1e-30, 1e30] (or NaN), or alpha not finite */
     QNN_E_CUDA = -5,   /* the CUDA runtime refused a launch or copy (cudaGetLastError is consumed) */
-    QNN_E_DEVICE = -6  /* a kernel reported an internal error through its status word */
+    QNN_E_DEVICE = -6  /* reserved: a kernel reported an internal error (no current kernel waits on anything that can time out) */
 } qnn_status;
 
 /* flags of qnn_encode_pack */
