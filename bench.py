@@ -304,6 +304,9 @@ def cpu_baseline_leg():
 
 def run_gpu(args):
     import torch
+    from paper_2106_09886_b200 import build as lib_build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        lib_build.build()          # no-op when the library on disk matches the sources
     from paper_2106_09886_b200 import qnn
     from paper_2106_09886_b200 import workloads as wl
 
