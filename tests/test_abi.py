@@ -79,6 +79,15 @@ def test_argument_errors_are_reported_before_any_launch(qnn):
     assert lib.qnn_bconv2d(p, 2, p, 2, 1, 4, 4, 8, 8, 3, 3, 0, 1, 1.0, p, None, None) == qnn.E_ARG   # stride 0
     assert lib.qnn_bconv2d(p, 2, p, 2, 1, 2, 2, 8, 8, 5, 5, 1, 0, 1.0, p, None, None) == qnn.E_ARG   # kernel > image
     assert lib.qnn_bconv2d(p, 8, p, 8, 1, 8, 8, 4096, 8, 3, 3, 1, 1, 1.0, p, None, None) == qnn.E_RANGE
+    # empty problems are refused, not launched
+    assert lib.qnn_encode_pack(p, 0, 64, 64, 2, 1.0, 0, p, None, None) == qnn.E_ARG
+    assert lib.qnn_encode_pack(p, 4, 0, 0, 2, 1.0, 0, p, None, None) == qnn.E_ARG
+    assert lib.qnn_pack_weights(p, 0, 1, 64, 0, 2, 1.0, p, None) == qnn.E_ARG
+    assert lib.qnn_bgemm(p, 2, p, 2, 0, 4, 64, 1.0, p, 4, None, None) == qnn.E_ARG
+    assert lib.qnn_bgemm(p, 2, p, 2, 4, 0, 64, 1.0, p, 4, None, None) == qnn.E_ARG
+    assert lib.qnn_bgemm(p, 2, p, 2, 4, 4, 0, 1.0, p, 4, None, None) == qnn.E_ARG
+    assert lib.qnn_bconv2d(p, 2, p, 2, 0, 4, 4, 8, 8, 3, 3, 1, 1, 1.0, p, None, None) == qnn.E_ARG
+    assert lib.qnn_absmax_f32(p, 0, p, None) == qnn.E_ARG
     assert lib.qnn_absmax_f32(None, 4, p, None) == qnn.E_ARG
     assert lib.qnn_probe_copy(p, p, 24, None) == qnn.E_ARG
 
