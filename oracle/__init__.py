@@ -13,6 +13,7 @@ What each function follows in the paper:
 * ``fc`` / ``conv2d`` (and their ``_sampled`` forms) -- Op(EnC(x), EnC(w)) of Eq. 9:
                       the plain integer product that Eq. 8 reproduces exactly.
 * ``scale``        -- the fixed scaling factor of Eq. 9 / Alg. 1 forward pass.
+* ``mbit_encoder_forward`` / ``mbit_encoder_backward`` -- trigonometric encoder of Eq. 10 and its derivative, Eq. 12.
 * ``affine``       -- per-feature affine that replaces the scale when batch normalisation follows (Section 3.2).
 """
 from __future__ import annotations
@@ -61,6 +62,8 @@ def _load():
         lib.oracle_conv2d_sampled.argtypes = [p, p] + [c.c_int] * 9 + [c.c_size_t, p, p, p]
         lib.oracle_scale.argtypes = [p, c.c_size_t, c.c_float, p]
         lib.oracle_conv2d_general.argtypes = [p, p] + [c.c_int] * 12 + [p]
+        lib.oracle_mbit_encoder_forward.argtypes = [p, c.c_size_t, c.c_int, c.c_float, p]
+        lib.oracle_mbit_encoder_backward.argtypes = [p, p, c.c_size_t, c.c_int, c.c_float, p]
         lib.oracle_affine.argtypes = [p, c.c_size_t, c.c_size_t, p, p]
         _lib = lib
     return _lib
@@ -205,3 +208,22 @@ def conv2d_general(qa: np.ndarray, qw: np.ndarray, stride: int, pad: int, dil: i
     _check(_load().oracle_conv2d_general(_ptr(qa), _ptr(qw), N, H, W, C, Cout, R, S, stride, pad, dil, int(transposed),
                                          out_pad, _ptr(acc)), "conv2d_general")
     return acc
+
+
+def mbit_encoder_forward(x: np.ndarray, bits: int, r: float = 1.0) -> np.ndarray:
+    """Eq. 10: returns c float32 [bits, n] with c[m-1] = phi_M^m(x / r) in {-1, 0, +1}."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    c = np.empty((bits, x.size), dtype=np.float32)
+    _check(_load().oracle_mbit_encoder_forward(_ptr(x), x.size, bits, float(np.float32(r)), _ptr(c)), "mbit_encoder_forward")
+    return c
+
+
+def mbit_encoder_backward(x: np.ndarray, gc: np.ndarray, bits: int, r: float = 1.0) -> np.ndarray:
+    """Eq. 12: gradient with respect to x (float64 [n]) given gradients gc [bits, n] of the encoder outputs."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    gc = np.ascontiguousarray(gc, dtype=np.float32)
+    assert gc.shape == (bits, x.size)
+    gx = np.empty(x.size, dtype=np.float64)
+    _check(_load().oracle_mbit_encoder_backward(_ptr(x), _ptr(gc), x.size, bits, float(np.float32(r)), _ptr(gx)),
+           "mbit_encoder_backward")
+    return gx

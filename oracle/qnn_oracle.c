@@ -312,3 +312,50 @@ int oracle_conv2d_general(const int16_t *qa, const int16_t *qw, int N, int H, in
     free(wide);
     return bad ? ORACLE_E_RANGE : ORACLE_OK;
 }
+
+/*
+ * Trigonometric M-bit encoder (Eq. 10) and its straight-through derivative (Eq. 12), the training-side form of
+ * the encoder.  With xn = x / r and k_m = (2^M - 1) / 2^m:
+ *   phi_M^M(xn) = sign(sin(k_M pi xn)),   phi_M^m(xn) = sign(-sin(k_m pi xn)) for m < M,
+ *   d phi_M^m / d xn = +- k_m pi cos(k_m pi xn) for |xn| <= 1, else 0 (sign + for m = M, - otherwise).
+ * Forward: the sign is a decision, so it is taken in the kernel's precision: y = k_m * xn is one binary32
+ * product (k_m is exactly representable), sin(pi y) is 0 exactly when y is an integer, positive when floor(y)
+ * is even and negative when it is odd -- no library sine is involved, so the decision is reproducible.
+ * c[(m-1)*n + e] receives phi_M^m of element e as -1, 0 or +1.
+ */
+int oracle_mbit_encoder_forward(const float *x, size_t n, int bits, float r, float *c) {
+    if (!x || !c || bits < 1 || bits > 8 || !(r > 0.0f)) return ORACLE_E_ARG;
+    for (int m = 1; m <= bits; ++m) {
+        const float k = (float)((1 << bits) - 1) / (float)(1 << m);
+        for (size_t e = 0; e < n; ++e) {
+            const float xn = x[e] / r;
+            const float y = k * xn;
+            const float fl = floorf(y);
+            float sgn;
+            if (!(y == y) || isinf(y)) sgn = 0.0f;                    /* NaN / infinity: no state */
+            else if (fl == y) sgn = 0.0f;
+            else sgn = (fmodf(fl, 2.0f) == 0.0f) ? 1.0f : -1.0f;       /* sin(pi y) > 0 on (2j, 2j+1) */
+            c[(size_t)(m - 1) * n + e] = (m == bits) ? sgn : -sgn;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* gx[e] = (1/r) * sum_m gc[m-1][e] * d phi_M^m / d xn, evaluated in binary64 (Eq. 12; zero outside [-1, 1]). */
+int oracle_mbit_encoder_backward(const float *x, const float *gc, size_t n, int bits, float r, double *gx) {
+    if (!x || !gc || !gx || bits < 1 || bits > 8 || !(r > 0.0f)) return ORACLE_E_ARG;
+    const double pi = 3.14159265358979323846;
+    for (size_t e = 0; e < n; ++e) {
+        const double xn = (double)(x[e] / r);                          /* the division the kernel performs */
+        double g = 0.0;
+        if (xn >= -1.0 && xn <= 1.0) {
+            for (int m = 1; m <= bits; ++m) {
+                const double k = (double)((1 << bits) - 1) / (double)(1 << m);
+                const double d = k * pi * cos(k * pi * xn);
+                g += (double)gc[(size_t)(m - 1) * n + e] * ((m == bits) ? d : -d);
+            }
+        }
+        gx[e] = g / (double)r;
+    }
+    return ORACLE_OK;
+}

@@ -381,3 +381,53 @@ def test_general_conv_matches_torch(N, H, W, C, Cout, R, S, stride, pad, dil, tr
         wt = torch.from_numpy(qw.astype(np.float64)).permute(3, 0, 1, 2)                 # [C, Cout, R, S]
         ref = torch.nn.functional.conv_transpose2d(x, wt, stride=stride, padding=pad, output_padding=out_pad, dilation=dil)
     assert np.array_equal(acc.astype(np.float64), ref.permute(0, 2, 3, 1).numpy())
+
+
+# ----------------------------------------------------------------------------- trigonometric encoder (training side)
+
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_mbit_encoder_forward_is_sign_of_sine_and_matches_the_lookup_encoder(bits):
+    """Away from the zero crossings the parity rule equals sign(+-sin(k pi x)) evaluated in float64 (Eq. 10), and its
+    bits are the planes of the table quantizer (Table 2 / Eq. 7) for data in [-1, 1]; at crossings it is 0."""
+    rng = np.random.default_rng(50 + bits)
+    A = 2 ** bits - 1
+    x = rng.uniform(-1, 1, size=5000)
+    x = x[np.abs(x * A / 2 - np.round(x * A / 2)) > 1e-3].astype(np.float32)
+    c = oracle.mbit_encoder_forward(x, bits)
+    q = oracle.quantize(x, bits, np.float32(1.0) / np.float32(A)).astype(np.int64)
+    t = (q + A) // 2
+    for m in range(1, bits + 1):
+        arg = A / 2 ** m * math.pi * x.astype(np.float64)
+        want = np.sign(np.sin(arg)) if m == bits else np.sign(-np.sin(arg))
+        assert np.array_equal(c[m - 1], want.astype(np.float32)), (bits, m)
+        assert np.array_equal(c[m - 1], np.where((t >> (m - 1)) & 1, 1.0, -1.0).astype(np.float32))
+    # exact zero crossings give 0: x = 0 for every bit, and x = +-2, 4 for the lowest bit (k_1 * x = A * x / 2 is an integer)
+    cz = oracle.mbit_encoder_forward(np.array([0.0, 2.0, -2.0, 4.0], dtype=np.float32), bits)
+    assert np.all(cz[:, 0] == 0.0) and np.all(cz[0] == 0.0)
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 5, 8])
+def test_mbit_encoder_backward_is_the_derivative_of_the_sine_and_zero_outside(bits):
+    """Eq. 12 is the derivative of the sine inside the sign (a straight-through estimate): compare with a central
+    difference of +-sin(k pi x) in float64, and check the cut-off outside [-1, 1] and the 1/r chain factor."""
+    rng = np.random.default_rng(60 + bits)
+    A = 2 ** bits - 1
+    x = rng.uniform(-0.99, 0.99, size=400).astype(np.float32)
+    for m in range(1, bits + 1):
+        gc = np.zeros((bits, x.size), dtype=np.float32)
+        gc[m - 1] = 1.0
+        got = oracle.mbit_encoder_backward(x, gc, bits)
+        k = A / 2 ** m
+        f = (lambda z: np.sin(k * math.pi * z)) if m == bits else (lambda z: -np.sin(k * math.pi * z))
+        h = 1e-6
+        num = (f(x.astype(np.float64) + h) - f(x.astype(np.float64) - h)) / (2 * h)
+        assert np.allclose(got, num, rtol=1e-5, atol=1e-4 * k)
+    xo = np.array([-1.5, 1.0000001, 2.0, -1.0, 1.0, 0.0], dtype=np.float32)
+    g = oracle.mbit_encoder_backward(xo, np.ones((bits, xo.size), np.float32), bits)
+    assert np.all(g[:3] == 0.0) and g[5] != 0.0
+    # chain rule through the range: encoder(x / r)
+    r = 3.0
+    xr = (x * r).astype(np.float32)
+    g1 = oracle.mbit_encoder_backward(xr, np.ones((bits, x.size), np.float32), bits, r)
+    g0 = oracle.mbit_encoder_backward((xr / np.float32(r)).astype(np.float32), np.ones((bits, x.size), np.float32), bits)
+    assert np.allclose(g1, g0 / r, rtol=1e-12)
