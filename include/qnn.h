@@ -182,6 +182,20 @@ int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *w_packed, i
                        uint32_t *next_planes, float *out, void *stream);
 
 /*
+ * Training-side form of the encoder: the trigonometric M-bit encoder (Eq. 10) and its derivative (Eq. 12).
+ * With xn = x / r and k_m = (2^bits - 1) / 2^m (m = 1..bits):
+ *   forward   c[(m-1)*n + e] = phi^m(xn[e]) = sign(sin(k_m*pi*xn)) for m = bits, sign(-sin(k_m*pi*xn)) otherwise,
+ *             as -1, 0 or +1 (0 exactly at a zero crossing).  The sign is taken from y = k_m*xn (one binary32
+ *             product): 0 if y is an integer, else by the parity of floor(y); no library sine decides it.
+ *             Away from the crossings these are the planes of qnn_encode_pack for data in [-r, r].
+ *   backward  gx[e] = (1/r) * sum_m gc[(m-1)*n + e] * (+-) k_m*pi*cos(k_m*pi*xn[e]) for |xn| <= 1, else 0
+ *             (+ for m = bits, - otherwise): the straight-through estimate of Eq. 12, in binary32.
+ *   x fp32 [n]; c, gc fp32 [bits][n]; gx fp32 [n]; r in [1e-30, 1e30].
+ */
+int qnn_mbit_encoder_forward(const float *x, size_t n, int bits, float r, float *c, void *stream);
+int qnn_mbit_encoder_backward(const float *x, const float *gc, size_t n, int bits, float r, float *gx, void *stream);
+
+/*
  * max_i |x[i]| into *out (device fp32), for workloads whose grid step is derived
  * from the tensor's range.  Not a step of the paper's method (its range r is a
  * fixed or learned constant, Eq. 9 / Eq. 15).  NaNs are ignored.

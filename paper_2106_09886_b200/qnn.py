@@ -20,7 +20,8 @@ W_NTC, W_TCN, W_NCT = 0, 1, 2
 EXPORTS = [
     "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
-    "qnn_bgemm_encode", "qnn_bconv2d_encode", "qnn_bconv2d_general",
+    "qnn_bgemm_encode", "qnn_bconv2d_encode", "qnn_bconv2d_general", "qnn_mbit_encoder_forward",
+    "qnn_mbit_encoder_backward",
     "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -56,6 +57,8 @@ def _load() -> C.CDLL:
     lib.qnn_bconv2d_general.argtypes = [p, i, p, i] + [i] * 12 + [f, p, p, p]
     lib.qnn_bgemm_encode.argtypes = [p, i, p, i, i64, i, i, f, p, p, i, f, u, p, p, i64, p]
     lib.qnn_bconv2d_encode.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, i, f, u, p, p, p]
+    lib.qnn_mbit_encoder_forward.argtypes = [p, sz, i, f, p, p]
+    lib.qnn_mbit_encoder_backward.argtypes = [p, p, sz, i, f, p, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
     lib.qnn_fc_forward_host_pipelined.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, i64, C.POINTER(C.c_void_p), i]
@@ -224,6 +227,28 @@ def bconv2d_encode(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: 
                                   _ptr(next_planes) if encode else None, _ptr(out), _stream(stream)),
            "qnn_bconv2d_encode")
     return next_planes if encode else out
+
+
+def mbit_encoder_forward(x: torch.Tensor, bits: int, r: float = 1.0, c: torch.Tensor | None = None, stream=None):
+    """Eq. 10: c fp32 [bits, n] with c[m-1] = phi^m(x / r) in {-1, 0, +1}."""
+    _dev(x, torch.float32, "x")
+    if c is None:
+        c = torch.empty((bits, x.numel()), dtype=torch.float32, device=x.device)
+    _check(lib.qnn_mbit_encoder_forward(_ptr(x), x.numel(), bits, float(r), _ptr(c), _stream(stream)),
+           "qnn_mbit_encoder_forward")
+    return c
+
+
+def mbit_encoder_backward(x: torch.Tensor, gc: torch.Tensor, bits: int, r: float = 1.0, gx: torch.Tensor | None = None,
+                          stream=None):
+    """Eq. 12: gradient with respect to x given the gradients gc [bits, n] of the encoder outputs."""
+    _dev(x, torch.float32, "x")
+    _dev(gc, torch.float32, "gc")
+    if gx is None:
+        gx = torch.empty(x.numel(), dtype=torch.float32, device=x.device)
+    _check(lib.qnn_mbit_encoder_backward(_ptr(x), _ptr(gc), x.numel(), bits, float(r), _ptr(gx), _stream(stream)),
+           "qnn_mbit_encoder_backward")
+    return gx
 
 
 def absmax_f32(x: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:

@@ -128,6 +128,19 @@ def time_stack(net: str, batch: int, reps=3, warmup=2, dev="cuda:0", seed=0, lay
             "binary_tops": 2 * bin_macs / (tot_ms * 1e-3) / 1e12, "equiv_int_gops": 2 * tot_macs / (tot_ms * 1e-3) / 1e9}
 
 
+def time_mbit(n, bits, reps=5, warmup=3, dev="cuda:0", seed=0):
+    """Trigonometric encoder forward and backward on n elements (streaming kernels; GB/s of their algorithmic bytes)."""
+    g = torch.Generator(device=dev).manual_seed(seed)
+    x = torch.rand(n, device=dev, generator=g) * 2 - 1
+    c = torch.empty((bits, n), dtype=torch.float32, device=dev)
+    gc = torch.randn((bits, n), device=dev, generator=g)
+    gx = torch.empty(n, dtype=torch.float32, device=dev)
+    tf = statistics.median(_time_calls(lambda i: qnn.mbit_encoder_forward(x, bits, 1.0, c=c), reps, warmup))
+    tb = statistics.median(_time_calls(lambda i: qnn.mbit_encoder_backward(x, gc, bits, 1.0, gx=gx), reps, warmup))
+    return {"call": "qnn_mbit_encoder", "n": n, "bits": bits, "forward_ms": tf, "backward_ms": tb,
+            "forward_gbs": n * 4 * (1 + bits) / (tf * 1e-3) / 1e9, "backward_gbs": n * 4 * (2 + bits) / (tb * 1e-3) / 1e9}
+
+
 def _report(call, Mg, Ng, Kg, ab, wb, times):
     ms = statistics.median(times)
     macs = float(Mg) * Ng * Kg
@@ -149,12 +162,15 @@ def main():
     e = sub.add_parser("encode")
     for name, default in (("rows", 4096), ("k", 4096), ("bits", 2)):
         e.add_argument(f"--{name}", type=int, default=default)
+    mb = sub.add_parser("mbit")
+    mb.add_argument("--n", type=int, default=1 << 26)
+    mb.add_argument("--bits", type=int, default=2)
     k = sub.add_parser("stack")
     k.add_argument("--net", choices=["resnet18", "resnet18_p1", "resnet18_p2", "vgg16"], default="resnet18")
     k.add_argument("--batch", type=int, default=0)
     k.add_argument("--layers", type=str, default="")
     k.add_argument("--table", action="store_true")
-    for s in (g, c, e, k):
+    for s in (g, c, e, k, mb):
         s.add_argument("--reps", type=int, default=5)
         s.add_argument("--warmup", type=int, default=3)
         s.add_argument("--sets", type=int, default=3)
@@ -163,6 +179,8 @@ def main():
         r = time_gemm(a.m, a.n, a.k, a.ab, a.wb, a.reps, a.warmup, a.sets)
     elif a.case == "conv":
         r = time_conv(a.N, a.H, a.W, a.C, a.Cout, a.R, a.S, a.stride, a.pad, a.ab, a.wb, a.reps, a.warmup, a.sets)
+    elif a.case == "mbit":
+        r = time_mbit(a.n, a.bits, a.reps, a.warmup)
     elif a.case == "stack":
         batch = a.batch or (64 if a.net == "vgg16" else 256)
         layers = [int(v) for v in a.layers.split(",")] if a.layers else None
