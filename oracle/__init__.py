@@ -64,6 +64,12 @@ def _load():
         lib.oracle_conv2d_general.argtypes = [p, p] + [c.c_int] * 12 + [p]
         lib.oracle_mbit_encoder_forward.argtypes = [p, c.c_size_t, c.c_int, c.c_float, p]
         lib.oracle_mbit_encoder_backward.argtypes = [p, p, c.c_size_t, c.c_int, c.c_float, p]
+        lib.oracle_fc_backward_data.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, c.c_int, c.c_int, c.c_float, p]
+        lib.oracle_fc_backward_weights.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, c.c_int, c.c_int, c.c_float, p]
+        lib.oracle_fc_backward_data_sampled.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_int, c.c_int, c.c_float,
+                                                        c.c_size_t, p, p, p]
+        lib.oracle_fc_backward_weights_sampled.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, c.c_int, c.c_int,
+                                                           c.c_float, c.c_size_t, p, p, p]
         lib.oracle_affine.argtypes = [p, c.c_size_t, c.c_size_t, p, p]
         _lib = lib
     return _lib
@@ -227,3 +233,57 @@ def mbit_encoder_backward(x: np.ndarray, gc: np.ndarray, bits: int, r: float = 1
     _check(_load().oracle_mbit_encoder_backward(_ptr(x), _ptr(gc), x.size, bits, float(np.float32(r)), _ptr(gx)),
            "mbit_encoder_backward")
     return gx
+
+
+def fc_backward_data(g: np.ndarray, qw: np.ndarray, ab: int, wb: int, alpha: float) -> np.ndarray:
+    """Algorithm 1, backward: g [Mg, Ng] = dC/da, qw [Ng, Kg] -> float64 [ab, Mg, Kg], entry m-1 = g_{a^m}."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    (Mg, Ng), (Ng2, Kg) = g.shape, qw.shape
+    assert Ng == Ng2
+    ga = np.empty((ab, Mg, Kg), dtype=np.float64)
+    _check(_load().oracle_fc_backward_data(_ptr(g), _ptr(qw), Mg, Ng, Kg, ab, wb, float(np.float32(alpha)), _ptr(ga)),
+           "fc_backward_data")
+    return ga
+
+
+def fc_backward_weights(g: np.ndarray, qa: np.ndarray, ab: int, wb: int, alpha: float) -> np.ndarray:
+    """Algorithm 1, backward: g [Mg, Ng], qa [Mg, Kg] -> float64 [wb, Ng, Kg], entry j-1 = g_{W^j}."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    (Mg, Ng), (Mg2, Kg) = g.shape, qa.shape
+    assert Mg == Mg2
+    gw = np.empty((wb, Ng, Kg), dtype=np.float64)
+    _check(_load().oracle_fc_backward_weights(_ptr(g), _ptr(qa), Mg, Ng, Kg, ab, wb, float(np.float32(alpha)), _ptr(gw)),
+           "fc_backward_weights")
+    return gw
+
+
+def fc_backward_data_sampled(g, qw, ab: int, wb: int, alpha: float, rows, cols) -> np.ndarray:
+    """g_{a^m} at (row, col) pairs: float64 [ab, count]."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    Ng, Kg = qw.shape
+    assert g.shape[1] == Ng and rows.max() < g.shape[0] and cols.max() < Kg and rows.min() >= 0 and cols.min() >= 0
+    out = np.empty((ab, rows.size), dtype=np.float64)
+    _check(_load().oracle_fc_backward_data_sampled(_ptr(g), _ptr(qw), Ng, Kg, ab, wb, float(np.float32(alpha)), rows.size,
+                                                   _ptr(rows), _ptr(cols), _ptr(out)), "fc_backward_data_sampled")
+    return out
+
+
+def fc_backward_weights_sampled(g, qa, ab: int, wb: int, alpha: float, rows, cols) -> np.ndarray:
+    """g_{W^j} at (n, k) pairs: float64 [wb, count]."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    Mg, Kg = qa.shape
+    Ng = g.shape[1]
+    assert g.shape[0] == Mg and rows.max() < Ng and cols.max() < Kg and rows.min() >= 0 and cols.min() >= 0
+    out = np.empty((wb, rows.size), dtype=np.float64)
+    _check(_load().oracle_fc_backward_weights_sampled(_ptr(g), _ptr(qa), Mg, Ng, Kg, ab, wb, float(np.float32(alpha)),
+                                                      rows.size, _ptr(rows), _ptr(cols), _ptr(out)),
+           "fc_backward_weights_sampled")
+    return out

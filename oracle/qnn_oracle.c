@@ -359,3 +359,111 @@ int oracle_mbit_encoder_backward(const float *x, const float *gc, size_t n, int 
     }
     return ORACLE_OK;
 }
+
+/*
+ * Backward products of one fully-connected layer (Algorithm 1, backward propagation).
+ * Forward (Algorithm 1, forward propagation): a_hat[r][n] = sum_m sum_j 2^(m+j-2) sum_k a^m[r][k] * W^j[n][k] and
+ * a = alpha * a_hat, with a^m, W^j in {-1,+1} the planes of the odd codes qa (ab planes) and qw (wb planes):
+ * q = sum_i 2^(i-1) * plane_i(q).  Given g = dC/da (binary32 input, all arithmetic here in binary64):
+ *   g_hat            = alpha * g
+ *   g_a^m [r][k]     = sum_j 2^(m+j-2) * sum_n g_hat[r][n] * W^j[n][k]        m = 1..ab
+ *   g_W^j [n][k]     = sum_m 2^(m+j-2) * sum_r g_hat[r][n] * a^m[r][k]        j = 1..wb
+ * The loops follow the algorithm's order (planes outside, contraction inside); no regrouping into codes.
+ */
+static double plane_of(int q, int bits, int i) {                      /* i = 1..bits; q odd in [-(2^bits-1), 2^bits-1] */
+    const int t = (q + ((1 << bits) - 1)) / 2;
+    return ((t >> (i - 1)) & 1) ? 1.0 : -1.0;
+}
+
+static int codes_ok(const int16_t *q, size_t n, int bits) {
+    const int A = (1 << bits) - 1;
+    for (size_t i = 0; i < n; ++i)
+        if (q[i] < -A || q[i] > A || ((q[i] & 1) == 0)) return 0;
+    return 1;
+}
+
+/* ga[(m-1)*Mg*Kg + r*Kg + k] = g_a^m[r][k] */
+int oracle_fc_backward_data(const float *g, const int16_t *qw, size_t Mg, size_t Ng, size_t Kg, int ab, int wb,
+                            float alpha, double *ga) {
+    if (!g || !qw || !ga || ab < 1 || ab > 8 || wb < 1 || wb > 8) return ORACLE_E_ARG;
+    if (!codes_ok(qw, Ng * Kg, wb)) return ORACLE_E_ARG;
+    for (int m = 1; m <= ab; ++m) {
+#pragma omp parallel for schedule(static)
+        for (size_t r = 0; r < Mg; ++r)
+            for (size_t k = 0; k < Kg; ++k) {
+                double sum = 0.0;
+                for (int j = 1; j <= wb; ++j) {
+                    double part = 0.0;
+                    for (size_t n = 0; n < Ng; ++n)
+                        part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qw[n * Kg + k], wb, j);
+                    sum += ldexp(part, m + j - 2);
+                }
+                ga[((size_t)(m - 1) * Mg + r) * Kg + k] = sum;
+            }
+    }
+    return ORACLE_OK;
+}
+
+/* gw[(j-1)*Ng*Kg + n*Kg + k] = g_W^j[n][k] */
+int oracle_fc_backward_weights(const float *g, const int16_t *qa, size_t Mg, size_t Ng, size_t Kg, int ab, int wb,
+                               float alpha, double *gw) {
+    if (!g || !qa || !gw || ab < 1 || ab > 8 || wb < 1 || wb > 8) return ORACLE_E_ARG;
+    if (!codes_ok(qa, Mg * Kg, ab)) return ORACLE_E_ARG;
+    for (int j = 1; j <= wb; ++j) {
+#pragma omp parallel for schedule(static)
+        for (size_t n = 0; n < Ng; ++n)
+            for (size_t k = 0; k < Kg; ++k) {
+                double sum = 0.0;
+                for (int m = 1; m <= ab; ++m) {
+                    double part = 0.0;
+                    for (size_t r = 0; r < Mg; ++r)
+                        part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qa[r * Kg + k], ab, m);
+                    sum += ldexp(part, m + j - 2);
+                }
+                gw[((size_t)(j - 1) * Ng + n) * Kg + k] = sum;
+            }
+    }
+    return ORACLE_OK;
+}
+
+/* The same two gradients at `count` sampled positions only (for sizes where the full loops take too long):
+ * out[(p-1)*count + i] = g_a^p[rows[i]][cols[i]]  resp.  g_W^p[rows[i]][cols[i]]. */
+int oracle_fc_backward_data_sampled(const float *g, const int16_t *qw, size_t Ng, size_t Kg, int ab, int wb, float alpha,
+                                    size_t count, const int64_t *rows, const int64_t *cols, double *out) {
+    if (!g || !qw || !out || !rows || !cols || ab < 1 || ab > 8 || wb < 1 || wb > 8) return ORACLE_E_ARG;
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < count; ++i) {
+        const size_t r = (size_t)rows[i], k = (size_t)cols[i];
+        for (int m = 1; m <= ab; ++m) {
+            double sum = 0.0;
+            for (int j = 1; j <= wb; ++j) {
+                double part = 0.0;
+                for (size_t n = 0; n < Ng; ++n)
+                    part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qw[n * Kg + k], wb, j);
+                sum += ldexp(part, m + j - 2);
+            }
+            out[(size_t)(m - 1) * count + i] = sum;
+        }
+    }
+    return ORACLE_OK;
+}
+
+int oracle_fc_backward_weights_sampled(const float *g, const int16_t *qa, size_t Mg, size_t Ng, size_t Kg, int ab, int wb,
+                                       float alpha, size_t count, const int64_t *rows, const int64_t *cols, double *out) {
+    if (!g || !qa || !out || !rows || !cols || ab < 1 || ab > 8 || wb < 1 || wb > 8) return ORACLE_E_ARG;
+#pragma omp parallel for schedule(static)
+    for (size_t i = 0; i < count; ++i) {
+        const size_t n = (size_t)rows[i], k = (size_t)cols[i];
+        for (int j = 1; j <= wb; ++j) {
+            double sum = 0.0;
+            for (int m = 1; m <= ab; ++m) {
+                double part = 0.0;
+                for (size_t r = 0; r < Mg; ++r)
+                    part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qa[r * Kg + k], ab, m);
+                sum += ldexp(part, m + j - 2);
+            }
+            out[(size_t)(j - 1) * count + i] = sum;
+        }
+    }
+    return ORACLE_OK;
+}

@@ -31,6 +31,10 @@ MUTATIONS = {
     "dilation_ignored": ("int hi = ho * stride - pad + r * dil;\n                    if (hi < 0 || hi >= H) continue;", "int hi = ho * stride - pad + r;\n                    if (hi < 0 || hi >= H) continue;"),
     "transposed_scatter_stride": ("int ho = hi * stride - pad + r * dil;", "int ho = hi - pad + r * dil;"),
     "affine_twice_rounded": ("fmaf(y[(size_t)m * Ng + n], gamma[n], beta ? beta[n] : 0.0f);", "y[(size_t)m * Ng + n] * gamma[n] + (beta ? beta[n] : 0.0f);"),
+    "backward_data_weight_index_transposed": ("part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qw[n * Kg + k], wb, j);\n                    sum += ldexp(part, m + j - 2);\n                }\n                ga[", "part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qw[(n * Kg + k) % Kg * Ng + (n * Kg + k) / Kg % Ng], wb, j);\n                    sum += ldexp(part, m + j - 2);\n                }\n                ga["),
+    "backward_plane_weight_off_by_one": ("sum += ldexp(part, m + j - 2);\n                }\n                gw[", "sum += ldexp(part, m + j - 1);\n                }\n                gw["),
+    "backward_drops_alpha": ("part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qa[r * Kg + k], ab, m);\n                    sum += ldexp(part, m + j - 2);\n                }\n                gw[", "part += ((double)g[r * Ng + n]) * plane_of(qa[r * Kg + k], ab, m);\n                    sum += ldexp(part, m + j - 2);\n                }\n                gw["),
+    "backward_plane_sign": ("return ((t >> (i - 1)) & 1) ? 1.0 : -1.0;", "return ((t >> (i - 1)) & 1) ? -1.0 : 1.0;"),
     "scale_in_double": ("out[i] = (float)acc[i] * alpha;", "out[i] = (float)((double)acc[i] * (double)alpha * (1.0 + 1e-6));"),
 }
 

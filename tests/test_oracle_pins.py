@@ -431,3 +431,78 @@ def test_mbit_encoder_backward_is_the_derivative_of_the_sine_and_zero_outside(bi
     g1 = oracle.mbit_encoder_backward(xr, np.ones((bits, x.size), np.float32), bits, r)
     g0 = oracle.mbit_encoder_backward((xr / np.float32(r)).astype(np.float32), np.ones((bits, x.size), np.float32), bits)
     assert np.allclose(g1, g0 / r, rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- backward products (Algorithm 1)
+
+def _planes_pm1(q, bits):
+    """Codes -> float64 [bits, ...] of {-1,+1} planes (plane i-1 = a^i), by Eq. 8's bit decomposition."""
+    t = codes_to_t(q, bits)
+    return np.stack([np.where((t >> i) & 1, 1.0, -1.0) for i in range(bits)])
+
+
+def _backward_case(seed, Mg, Ng, Kg, ab, wb):
+    rng = np.random.default_rng(seed)
+    qa = (2 * rng.integers(0, 2 ** ab, size=(Mg, Kg)) - (2 ** ab - 1)).astype(np.int16)
+    qw = (2 * rng.integers(0, 2 ** wb, size=(Ng, Kg)) - (2 ** wb - 1)).astype(np.int16)
+    g = rng.standard_normal((Mg, Ng)).astype(np.float32)
+    alpha = float(np.float32(0.37 / ((2 ** ab - 1) * (2 ** wb - 1))))
+    return qa, qw, g, alpha
+
+
+@pytest.mark.parametrize("ab,wb", [(1, 1), (2, 2), (3, 1), (2, 4), (8, 8)])
+def test_backward_products_are_the_exact_change_of_the_forward_under_a_plane_flip(ab, wb):
+    """The forward (the pinned integer product) is linear in every plane entry, so flipping one entry of a^m or W^j
+    from -1 to +1 changes C = <g, alpha * a_hat> by exactly twice the oracle's gradient at that entry."""
+    Mg, Ng, Kg = 5, 7, 9
+    qa, qw, g, alpha = _backward_case(100 * ab + wb, Mg, Ng, Kg, ab, wb)
+    ga = oracle.fc_backward_data(g, qw, ab, wb, alpha)
+    gw = oracle.fc_backward_weights(g, qa, ab, wb, alpha)
+    assert ga.shape == (ab, Mg, Kg) and gw.shape == (wb, Ng, Kg)
+
+    def cost(qa_, qw_):
+        return float(np.sum(g.astype(np.float64) * alpha * oracle.fc(qa_, qw_).astype(np.float64)))
+
+    rng = np.random.default_rng(7)
+    pa, pw = _planes_pm1(qa, ab), _planes_pm1(qw, wb)
+    base = cost(qa, qw)
+    for _ in range(40):
+        m, r, k = rng.integers(0, ab), rng.integers(0, Mg), rng.integers(0, Kg)
+        q2 = qa.copy()
+        q2[r, k] -= np.int16(pa[m, r, k] * 2 * 2 ** m)              # flips plane m of that entry
+        assert cost(q2, qw) - base == pytest.approx(-2 * pa[m, r, k] * ga[m, r, k], rel=1e-9, abs=1e-12)
+        j, n, k = rng.integers(0, wb), rng.integers(0, Ng), rng.integers(0, Kg)
+        w2 = qw.copy()
+        w2[n, k] -= np.int16(pw[j, n, k] * 2 * 2 ** j)
+        assert cost(qa, w2) - base == pytest.approx(-2 * pw[j, n, k] * gw[j, n, k], rel=1e-9, abs=1e-12)
+
+
+@pytest.mark.parametrize("ab,wb", [(2, 2), (4, 3)])
+def test_backward_products_special_cases(ab, wb):
+    """A one-hot g picks out one weight row / one activation row scaled by alpha * 2^(m-1); a library matmul on the
+    codes gives the same numbers; the sampled variants agree with the full ones."""
+    Mg, Ng, Kg = 6, 10, 13
+    qa, qw, g, alpha = _backward_case(5, Mg, Ng, Kg, ab, wb)
+    e = np.zeros((Mg, Ng), dtype=np.float32)
+    e[2, 3] = 1.0
+    ga = oracle.fc_backward_data(e, qw, ab, wb, alpha)
+    gw = oracle.fc_backward_weights(e, qa, ab, wb, alpha)
+    for m in range(ab):
+        want = np.zeros((Mg, Kg))
+        want[2] = alpha * 2.0 ** m * qw[3]
+        assert np.allclose(ga[m], want, rtol=1e-14, atol=0)
+    for j in range(wb):
+        want = np.zeros((Ng, Kg))
+        want[3] = alpha * 2.0 ** j * qa[2]
+        assert np.allclose(gw[j], want, rtol=1e-14, atol=0)
+    ga = oracle.fc_backward_data(g, qw, ab, wb, alpha)
+    gw = oracle.fc_backward_weights(g, qa, ab, wb, alpha)
+    G = alpha * g.astype(np.float64)
+    for m in range(ab):
+        assert np.allclose(ga[m], 2.0 ** m * (G @ qw.astype(np.float64)), rtol=1e-12, atol=1e-15)
+    for j in range(wb):
+        assert np.allclose(gw[j], 2.0 ** j * (G.T @ qa.astype(np.float64)), rtol=1e-12, atol=1e-15)
+    rows = np.array([0, 5, 2, 2]); cols = np.array([12, 0, 7, 8])
+    assert np.array_equal(oracle.fc_backward_data_sampled(g, qw, ab, wb, alpha, rows, cols), ga[:, rows, cols])
+    rows = np.array([9, 0, 4, 4])
+    assert np.array_equal(oracle.fc_backward_weights_sampled(g, qa, ab, wb, alpha, rows, cols), gw[:, rows, cols])
