@@ -51,7 +51,7 @@ typedef enum qnn_status {
     QNN_E_RANGE = -3,  /* Kg*A*B does not fit int32, or an index does not fit the kernels' 32-bit tile arithmetic */
     QNN_E_SCALE = -4,  /* scale outside [1e-30, 1e30] (or NaN), or alpha not finite */
     QNN_E_CUDA = -5,   /* the CUDA runtime refused a launch or copy (cudaGetLastError is consumed) */
-    QNN_E_DEVICE = -6  /* reserved: a kernel reported an internal error (no current kernel waits on anything that can time out) */
+    QNN_E_DEVICE = -6  /* a kernel gave up a bounded wait (qnn_tensor_path_status) */
 } qnn_status;
 
 /* flags of qnn_encode_pack */
@@ -194,6 +194,53 @@ int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *w_packed, i
  */
 int qnn_mbit_encoder_forward(const float *x, size_t n, int bits, float r, float *c, void *stream);
 int qnn_mbit_encoder_backward(const float *x, const float *gc, size_t n, int bits, float r, float *gx, void *stream);
+
+/*
+ * Backward products of a fully-connected layer (Algorithm 1, backward propagation).  The forward is
+ * a[r][n] = alpha * sum_k qa[r][k] * qw[n][k] with qa, qw the odd codes whose planes a^m, W^j the layer holds
+ * (qa = sum_m 2^(m-1) a^m, qw = sum_j 2^(j-1) W^j).  Given g = dC/da, fp32 [m][n]:
+ *   qnn_bgemm_backward_data     G [r][kk] = alpha * sum_nn g[r][nn] * qw[nn][kk];  Algorithm 1's per-plane gradient is
+ *                               g_{a^p} = 2^(p-1) * G.  With x given (fp32 [m][k], the values the previous layer fed
+ *                               to its encoder, range r, ab planes) the encoder derivative of Eq. 12 is applied in
+ *                               the same kernel: out[r][kk] = (1/r) * sum_p 2^(p-1) * G[r][kk] * dphi^p/dxn(x[r][kk]/r),
+ *                               i.e. qnn_mbit_encoder_backward fed with gc_p = 2^(p-1) * G.  x = NULL: out = G
+ *                               (ab and r are ignored).
+ *   qnn_bgemm_backward_weights  GW[nn][kk] = alpha * sum_r g[r][nn] * qa[r][kk];  g_{W^j} = 2^(j-1) * GW.
+ * Both are TF32 tensor-core contractions with fp32 accumulation: the codes are exact, each element of g enters with
+ * 11 significant bits, so |error| <= alpha * sum |g| * |q| * (2^-10 + contraction length * 2^-24); a g whose
+ * elements have at most 11 significant bits and whose sums stay below 2^24 in units of its last place is contracted
+ * exactly.
+ *   w_planes  device planes [n][wb][qnn_row_words(k)] (what qnn_encode_pack writes for a [n][k] matrix; the
+ *             canonical-plane view of packed FC weights), a_planes [m][ab][qnn_row_words(k)]; 16-byte aligned
+ *   g         device fp32 [m][n], 16-byte aligned for backward_data (4-byte for backward_weights)
+ *   out / gw  device fp32 [m][k] / [n][k]
+ *   workspace device scratch owned by the caller, 256-byte aligned, at least qnn_bgemm_backward_*_workspace(m, n, k)
+ *             bytes (0 from the query = dimensions out of range); holds the codes (and g) in the operand order the
+ *             tensor cores read.  Every dimension is at most 65535*32.
+ * QNN_E_ARG also for a workspace that is too small.  The kernels bound every wait on an arrival; one that gives up
+ * is reported by qnn_tensor_path_status.
+ */
+size_t qnn_bgemm_backward_data_workspace(size_t m, size_t n, size_t k);
+int qnn_bgemm_backward_data(const float *g, const uint32_t *w_planes, size_t m, size_t n, size_t k, int wb, float alpha,
+                            const float *x, int ab, float r, float *out, void *workspace, size_t workspace_bytes,
+                            void *stream);
+size_t qnn_bgemm_backward_weights_workspace(size_t m, size_t n, size_t k);
+int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_planes, size_t m, size_t n, size_t k, int ab,
+                               float alpha, float *gw, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Planes [rows][bits][qnn_row_words(k)] -> the odd codes q = sum_i 2^(i-1) * plane_i (Eq. 8) as fp32:
+ * out[row*ld + col] (transpose = 0, ld >= k) or out[col*ld + row] (transpose != 0, ld >= rows).
+ */
+int qnn_unpack_codes_f32(const uint32_t *planes, size_t rows, size_t k, int bits, int transpose, float *out, size_t ld,
+                         void *stream);
+
+/*
+ * Synchronises the device and reports whether a tensor-path kernel gave up a bounded wait since the last call:
+ * *status = 0 and QNN_OK, or *status = 1 + the id of the first wait that gave up (0 producer, 1 MMA issuer,
+ * 2 epilogue) and QNN_E_DEVICE; the record is cleared.  Results of a call that reported an error are undefined.
+ */
+int qnn_tensor_path_status(unsigned int *status);
 
 /*
  * max_i |x[i]| into *out (device fp32), for workloads whose grid step is derived

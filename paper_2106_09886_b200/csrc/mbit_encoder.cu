@@ -2,6 +2,7 @@
 // Both are streaming element-wise kernels (bound: HBM; forward reads 4 B and writes 4*bits B per element,
 // backward reads 4 + 4*bits B and writes 4 B).
 #include "qnn_internal.cuh"
+#include "mbit_math.cuh"
 
 namespace {
 
@@ -32,23 +33,6 @@ __device__ __forceinline__ void mbit_forward_elem(float x, float r, float (&cm)[
         const float s = sign_sin_pi(__fmul_rn(k, xn));
         cm[m - 1] = (m == BITS) ? s : -s;
     }
-}
-
-// One element of Eq. 12: gm[m-1] is the incoming gradient of plane m-1.
-template <int BITS>
-__device__ __forceinline__ float mbit_backward_elem(float x, float r, const float (&gm)[BITS]) {
-    const float pi = 3.14159265358979323846f;
-    const float xn = __fdiv_rn(x, r);
-    float g = 0.0f;
-    if (xn >= -1.0f && xn <= 1.0f) {
-#pragma unroll
-        for (int m = 1; m <= BITS; ++m) {
-            const float k = (float)((1 << BITS) - 1) / (float)(1 << m);
-            const float d = __fmul_rn(__fmul_rn(k, pi), cospif(__fmul_rn(k, xn)));   // k*pi*cos(k*pi*xn)
-            g = __fmaf_rn(gm[m - 1], (m == BITS) ? d : -d, g);
-        }
-    }
-    return __fdiv_rn(g, r);
 }
 
 // VEC = 4: n is a multiple of 4 and every pointer is 16-byte aligned, so each thread moves float4s; VEC = 1 otherwise.

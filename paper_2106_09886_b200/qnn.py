@@ -21,7 +21,9 @@ EXPORTS = [
     "qnn_status_string", "qnn_version", "qnn_row_words", "qnn_planes_bytes", "qnn_weights_bytes",
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
     "qnn_bgemm_encode", "qnn_bconv2d_encode", "qnn_bconv2d_general", "qnn_mbit_encoder_forward",
-    "qnn_mbit_encoder_backward",
+    "qnn_mbit_encoder_backward", "qnn_bgemm_backward_data_workspace", "qnn_bgemm_backward_data",
+    "qnn_bgemm_backward_weights_workspace", "qnn_bgemm_backward_weights", "qnn_unpack_codes_f32",
+    "qnn_tensor_path_status",
     "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -59,6 +61,14 @@ def _load() -> C.CDLL:
     lib.qnn_bconv2d_encode.argtypes = [p, i, p, i] + [i] * 9 + [f, p, p, i, f, u, p, p, p]
     lib.qnn_mbit_encoder_forward.argtypes = [p, sz, i, f, p, p]
     lib.qnn_mbit_encoder_backward.argtypes = [p, p, sz, i, f, p, p]
+    lib.qnn_bgemm_backward_data_workspace.restype = sz
+    lib.qnn_bgemm_backward_data_workspace.argtypes = [sz, sz, sz]
+    lib.qnn_bgemm_backward_data.argtypes = [p, p, sz, sz, sz, i, f, p, i, f, p, p, sz, p]
+    lib.qnn_bgemm_backward_weights_workspace.restype = sz
+    lib.qnn_bgemm_backward_weights_workspace.argtypes = [sz, sz, sz]
+    lib.qnn_bgemm_backward_weights.argtypes = [p, p, sz, sz, sz, i, f, p, p, sz, p]
+    lib.qnn_unpack_codes_f32.argtypes = [p, sz, sz, i, i, p, sz, p]
+    lib.qnn_tensor_path_status.argtypes = [C.POINTER(C.c_uint)]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
     lib.qnn_fc_forward_host_pipelined.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, i64, C.POINTER(C.c_void_p), i]
@@ -249,6 +259,56 @@ def mbit_encoder_backward(x: torch.Tensor, gc: torch.Tensor, bits: int, r: float
     _check(lib.qnn_mbit_encoder_backward(_ptr(x), _ptr(gc), x.numel(), bits, float(r), _ptr(gx), _stream(stream)),
            "qnn_mbit_encoder_backward")
     return gx
+
+
+def _workspace(nbytes: int, device, workspace):
+    if workspace is None:
+        workspace = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=device)
+    return workspace
+
+
+def bgemm_backward_data(g: torch.Tensor, w_planes: torch.Tensor, k: int, wb: int, alpha: float,
+                        x: torch.Tensor | None = None, ab: int = 1, r: float = 1.0, out: torch.Tensor | None = None,
+                        workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Algorithm 1 backward, activation side: g fp32 [m, n], w_planes [n, wb, row_words(k)] -> fp32 [m, k]
+    (G, or the gradient through the encoder when x is given)."""
+    _dev(g, torch.float32, "g")
+    m, n = g.shape
+    if out is None:
+        out = torch.empty((m, k), dtype=torch.float32, device=g.device)
+    ws = _workspace(lib.qnn_bgemm_backward_data_workspace(m, n, k), g.device, workspace)
+    _check(lib.qnn_bgemm_backward_data(_ptr(g), _ptr(w_planes), m, n, k, wb, float(alpha), _ptr(x), ab, float(r),
+                                       _ptr(out), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "qnn_bgemm_backward_data")
+    return out
+
+
+def bgemm_backward_weights(g: torch.Tensor, a_planes: torch.Tensor, k: int, ab: int, alpha: float,
+                           gw: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Algorithm 1 backward, weight side: g fp32 [m, n], a_planes [m, ab, row_words(k)] -> GW fp32 [n, k]."""
+    _dev(g, torch.float32, "g")
+    m, n = g.shape
+    if gw is None:
+        gw = torch.empty((n, k), dtype=torch.float32, device=g.device)
+    ws = _workspace(lib.qnn_bgemm_backward_weights_workspace(m, n, k), g.device, workspace)
+    _check(lib.qnn_bgemm_backward_weights(_ptr(g), _ptr(a_planes), m, n, k, ab, float(alpha), _ptr(gw), _ptr(ws),
+                                          ws.numel() * ws.element_size(), _stream(stream)), "qnn_bgemm_backward_weights")
+    return gw
+
+
+def unpack_codes_f32(planes: torch.Tensor, rows: int, k: int, bits: int, transpose: bool = False, stream=None) -> torch.Tensor:
+    """Planes [rows, bits, row_words(k)] -> odd codes as fp32 [rows, k] (or [k, rows] when transpose)."""
+    out = torch.empty((k, rows) if transpose else (rows, k), dtype=torch.float32, device=planes.device)
+    _check(lib.qnn_unpack_codes_f32(_ptr(planes), rows, k, bits, int(transpose), _ptr(out), rows if transpose else k,
+                                    _stream(stream)), "qnn_unpack_codes_f32")
+    return out
+
+
+def tensor_path_status() -> int:
+    """Synchronises; 0, or raises QnnError(QNN_E_DEVICE) when a tensor-path kernel gave up a bounded wait."""
+    st = C.c_uint(0)
+    _check(lib.qnn_tensor_path_status(C.byref(st)), "qnn_tensor_path_status")
+    return st.value
 
 
 def absmax_f32(x: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
