@@ -118,7 +118,8 @@ __host__ __device__ constexpr uint32_t idesc_tf32() {
 constexpr int BM = 128;                 // rows of C per CTA = lanes of tensor memory
 constexpr int BK = 32;                  // fp32 elements per stage row = 128 bytes = one swizzle span
 constexpr int UMMA_K = 8;               // K of one TF32 instruction (32 bytes)
-constexpr int GEMM_THREADS = 192;       // warp 0: TMA producer, warp 1: MMA issuer + tensor-memory owner, warps 2-5: epilogue
+constexpr int EPI_WARPS = 8;            // two warps per quarter of the tensor-memory lanes, alternating 32-column chunks
+constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;   // warp 0: TMA producer, warp 1: MMA issuer + tensor-memory owner
 
 struct GemmParams {
     int M, N, K;                        // C[M][N] = alpha * sum_k A[M][K] * B[N][K]
@@ -131,7 +132,7 @@ struct GemmParams {
     int vec_x;
     int bits;
     float r;
-    int tiles_n;
+    int tiles_n, tiles;
 };
 
 template <int BN, int STAGES>
@@ -140,25 +141,26 @@ struct GemmSmem {
     static constexpr int B_BYTES = BN * BK * 4;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-    static constexpr int TOTAL = BAR_OFFSET + (2 * STAGES + 1) * 8 + 16 + 1024;   // + slack for the 1024-byte alignment
+    static constexpr int TOTAL = BAR_OFFSET + (2 * STAGES + 4) * 8 + 16 + 1024;   // + slack for the 1024-byte alignment
 };
 
+// Persistent: CTA b works on tiles b, b + gridDim.x, ...  The accumulator is double-buffered in tensor memory
+// (2 x BN columns), so the epilogue of one tile runs under the main loop of the next.
 template <int BN, int STAGES>
-__global__ void __launch_bounds__(GEMM_THREADS) tf32_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                                const __grid_constant__ CUtensorMap map_b,
-                                                                const GemmParams p) {
+__global__ void __launch_bounds__(GEMM_THREADS, 1) tf32_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                   const __grid_constant__ CUtensorMap map_b,
+                                                                   const GemmParams p) {
     using L = GemmSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET);
     uint64_t *empty = full + STAGES;
-    uint64_t *acc_bar = empty + STAGES;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_bar + 1);
+    uint64_t *acc_full = empty + STAGES;          // [2]: the MMAs of a tile have retired
+    uint64_t *acc_empty = acc_full + 2;           // [2]: the epilogue has read the buffer out
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile_m = blockIdx.x / p.tiles_n, tile_n = blockIdx.x % p.tiles_n;
-    const int m0 = tile_m * BM, n0 = tile_n * BN;
     const int nkb = (p.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
@@ -166,12 +168,15 @@ __global__ void __launch_bounds__(GEMM_THREADS) tf32_gemm_kernel(const __grid_co
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(acc_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], EPI_WARPS);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(tmem_slot, BN);
+    if (warp == 1) tmem_alloc(tmem_slot, 2 * BN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -179,49 +184,63 @@ __global__ void __launch_bounds__(GEMM_THREADS) tf32_gemm_kernel(const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            int issued = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-                if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0)) break;
-                mbar_expect_tx(&full[s], L::STAGE_BYTES);
-                tma_load_2d(smem + s * L::STAGE_BYTES, &map_a, &full[s], kb * BK, m0);
-                tma_load_2d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], kb * BK, n0);
-                issued = kb + 1;
+            long long it = 0;                                 // stage uses so far, over all tiles
+            for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x) {
+                const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = (int)(it % STAGES);
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0)) break;
+                    mbar_expect_tx(&full[s], L::STAGE_BYTES);
+                    tma_load_2d(smem + s * L::STAGE_BYTES, &map_a, &full[s], kb * BK, m0);
+                    tma_load_2d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], kb * BK, n0);
+                }
             }
             if (*abort_flag) {   // let the copies still in flight land before the CTA's shared memory goes away
-                for (int kb = issued > STAGES ? issued - STAGES : 0; kb < issued; ++kb)
-                    for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try_wait(&full[kb % STAGES], (uint32_t)(kb / STAGES) & 1u); ++it) {}
+                for (long long j = it > STAGES ? it - STAGES : 0; j < it; ++j)
+                    for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(&full[j % STAGES], (uint32_t)(j / STAGES) & 1u); ++w) {}
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_tf32<BN>();
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-                if (!mbar_wait(&full[s], ph, abort_flag, 1)) break;
+            long long it = 0;
+            int local = 0;
+            for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++local) {
+                const int buf = local & 1;
+                if (!mbar_wait(&acc_empty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag, 3)) break;
                 tc_fence_after();
-                const uint64_t a_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES));
-                const uint64_t b_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES + L::A_BYTES));
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = (int)(it % STAGES);
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(&full[s], ph, abort_flag, 1)) break;
+                    tc_fence_after();
+                    const uint64_t a_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES));
+                    const uint64_t b_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES + L::A_BYTES));
 #pragma unroll
-                for (int j = 0; j < BK / UMMA_K; ++j)   // 32 bytes along K per step = 2 descriptor address units
-                    tc_mma_tf32(tmem_base, a_desc + 2 * j, b_desc + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
-                tc_commit(&empty[s]);
+                    for (int j = 0; j < BK / UMMA_K; ++j)   // 32 bytes along K per step = 2 descriptor address units
+                        tc_mma_tf32(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                    tc_commit(&empty[s]);
+                }
+                tc_commit(&acc_full[buf]);
             }
-            tc_commit(acc_bar);
         }
     } else {
-        const bool ok = mbar_wait(acc_bar, 0, abort_flag, 2);
-        tc_fence_after();
-        if (ok) {
-            const int q = warp & 3;                        // a warp reaches the 32 lanes [32*(warp%4), +32) only
+        const int q = warp & 3;                            // a warp reaches the 32 lanes [32*(warp%4), +32) only
+        const int half = (warp - 2) >> 2;                  // which of the two warps of this quarter
+        int local = 0;
+        for (int tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++local) {
+            const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+            const int buf = local & 1;
+            if (!mbar_wait(&acc_full[buf], (uint32_t)(local >> 1) & 1u, abort_flag, 2)) break;
+            tc_fence_after();
             const int row = m0 + q * 32 + lane;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = half * 32; c0 < BN; c0 += 64) {
                 if (n0 + c0 >= p.N) break;                 // uniform over the warp
                 float v[32];
-                tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+                tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
                 if (row < p.M) {
                     float *crow = p.C + (long long)row * p.ldc + n0 + c0;
                     const float *xrow = p.x ? p.x + (long long)row * p.ldx + n0 + c0 : nullptr;
@@ -253,52 +272,64 @@ __global__ void __launch_bounds__(GEMM_THREADS) tf32_gemm_kernel(const __grid_co
                     }
                 }
             }
+            // the buffer is free once every epilogue warp has its values in registers
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&acc_empty[buf])) : "memory");
         }
-        tc_fence_before();
     }
+    tc_fence_before();
     __syncthreads();
     if (warp == 1) {
-        // the accumulator's last MMA must have retired before its columns are given back
-        for (uint32_t it = 0; it < WAIT_LIMIT && !mbar_try_wait(acc_bar, 0); ++it) {}
+        // every MMA that was issued has retired once the last committed tile's barrier has completed its phase
+        const int mine = p.tiles > (int)blockIdx.x ? (p.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+        if (mine > 0) {
+            const int last = mine - 1;
+            for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(&acc_full[last & 1], (uint32_t)(last >> 1) & 1u); ++w) {}
+        }
         tc_fence_after();
-        tmem_dealloc(tmem_base, BN);
+        tmem_dealloc(tmem_base, 2 * BN);
     }
 }
 
 // ------------------------------------------------------------------------------------------------ staging kernels
 
-// Bit planes [rows][bits][kw] -> odd codes q = 2t - (2^bits - 1) as fp32.  TRANSPOSE = false: out[row][col];
-// TRANSPOSE = true: out[col][row].  A block covers 32 rows x 32 columns (one plane word per row); the 32 threads
-// of a warp run along the contiguous index of the output.
+// Bit planes [rows][bits][kw] -> odd codes q = 2t - (2^bits - 1) as fp32.  TRANSPOSE = false: out[row][col], a
+// block covers 32 rows x 256 columns (warp w owns plane word w of eight).  TRANSPOSE = true: out[col][row], a block
+// covers 256 rows x 32 columns (one plane word per row), so that each output row receives 1 KiB in one piece.
+// The 32 threads of a warp run along the contiguous index of the output: every store instruction writes one line.
 template <bool TRANSPOSE>
 __global__ void __launch_bounds__(256) unpack_codes_kernel(const uint32_t *__restrict__ planes, long long rows, long long k,
                                                           int bits, long long kw, float *__restrict__ out, long long ld) {
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const long long r0 = (long long)blockIdx.y * 32, wcol = blockIdx.x;
     const float amax = (float)((1 << bits) - 1);
     if (TRANSPOSE) {
-        const long long row = r0 + tx;
+        const long long row = (long long)blockIdx.y * 256 + threadIdx.x, wcol = blockIdx.x;
+        if (row >= rows) return;
         uint32_t w[8];
 #pragma unroll
-        for (int b = 0; b < 8; ++b) w[b] = (b < bits && row < rows) ? planes[(row * bits + b) * kw + wcol] : 0u;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int c = ty + 8 * i;
+        for (int b = 0; b < 8; ++b) w[b] = b < bits ? __ldg(planes + (row * bits + b) * kw + wcol) : 0u;
+#pragma unroll 8
+        for (int c = 0; c < 32; ++c) {
             const long long col = wcol * 32 + c;
             int t = 0;
 #pragma unroll
             for (int b = 0; b < 8; ++b) t |= (int)((w[b] >> c) & 1u) << b;
-            if (row < rows && col < k) out[col * ld + row] = (float)(2 * t) - amax;
+            if (col < k) __stcs(out + col * ld + row, (float)(2 * t) - amax);
         }
     } else {
+        const long long r0 = (long long)blockIdx.y * 32, wcol = (long long)blockIdx.x * 8 + ty;
         const long long col = wcol * 32 + tx;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const long long row = r0 + ty + 8 * i;
-            if (row >= rows) continue;
+        if (wcol * 32 >= k) return;
+#pragma unroll 4
+        for (int i = 0; i < 32; ++i) {
+            const long long row = r0 + i;
+            if (row >= rows) break;
             int t = 0;
-            for (int b = 0; b < bits; ++b) t |= (int)((planes[(row * bits + b) * kw + wcol] >> tx) & 1u) << b;
-            if (col < k) out[row * ld + col] = (float)(2 * t) - amax;
+#pragma unroll
+            for (int b = 0; b < 8; ++b)
+                if (b < bits) t |= (int)((__ldg(planes + (row * bits + b) * kw + wcol) >> tx) & 1u) << b;
+            if (col < k) __stcs(out + row * ld + col, (float)(2 * t) - amax);
         }
     }
 }
@@ -364,37 +395,61 @@ bool make_map(CUtensorMap *map, const float *base, long long rows, long long col
 
 long long pad32(long long v) { return (v + 31) / 32 * 32; }
 
-constexpr int GEMM_BN = 128, GEMM_STAGES = 3;
-
-// C[M][N] = alpha * A[M][K] * B[N][K]^T (optionally times the encoder derivative at x).
-int run_gemm(const float *A, long long lda, const float *B, long long ldb, GemmParams p, cudaStream_t st) {
-    using L = GemmSmem<GEMM_BN, GEMM_STAGES>;
-    if (p.M <= 0 || p.N <= 0 || p.K <= 0) return QNN_E_ARG;
-    if (!qnn_aligned(A, 16) || !qnn_aligned(B, 16) || lda % 4 || ldb % 4) return QNN_E_ALIGN;
-    CUtensorMap map_a, map_b;
-    if (!make_map(&map_a, A, p.M, p.K, lda, BM) || !make_map(&map_b, B, p.N, p.K, ldb, GEMM_BN)) return QNN_E_CUDA;
-    static bool attr_set = false;   // per process; the attribute is per device and function, set again if it fails
+template <int BN, int STAGES>
+int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, GemmParams p, int sms, cudaStream_t st) {
+    using L = GemmSmem<BN, STAGES>;
+    static bool attr_set = false;   // per process; set again on the next call if it failed
     if (!attr_set) {
-        if (cudaFuncSetAttribute(tf32_gemm_kernel<GEMM_BN, GEMM_STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 L::TOTAL) != cudaSuccess)
+        if (cudaFuncSetAttribute(tf32_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) !=
+            cudaSuccess)
             return QNN_E_CUDA;
         attr_set = true;
     }
-    const long long tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + GEMM_BN - 1) / GEMM_BN;
+    const long long tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return QNN_E_ARG;
     p.tiles_n = (int)tiles_n;
+    p.tiles = (int)(tiles_m * tiles_n);
+    const int grid = p.tiles < sms ? p.tiles : sms;
+    tf32_gemm_kernel<BN, STAGES><<<grid, GEMM_THREADS, L::TOTAL, st>>>(map_a, map_b, p);
+    return qnn_launch_status();
+}
+
+int sm_count() {
+    static int sms = 0;
+    if (!sms) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            sms = 0;
+    }
+    return sms;
+}
+
+// C[M][N] = alpha * A[M][K] * B[N][K]^T (optionally times the encoder derivative at x).  128 x 256 tiles when they
+// give every SM a tile (they read each A tile from shared memory half as often per flop as 128 x 128 ones, which a
+// single CTA per SM cannot feed fast enough), 128 x 128 tiles otherwise.
+int run_gemm(const float *A, long long lda, const float *B, long long ldb, GemmParams p, cudaStream_t st) {
+    if (p.M <= 0 || p.N <= 0 || p.K <= 0) return QNN_E_ARG;
+    if (!qnn_aligned(A, 16) || !qnn_aligned(B, 16) || lda % 4 || ldb % 4) return QNN_E_ALIGN;
+    const int sms = sm_count();
+    if (sms <= 0) return QNN_E_CUDA;
+    const bool wide = ((long long)(p.M + BM - 1) / BM) * ((p.N + 255) / 256) >= sms;
+    CUtensorMap map_a, map_b;
+    if (!make_map(&map_a, A, p.M, p.K, lda, BM) || !make_map(&map_b, B, p.N, p.K, ldb, wide ? 256 : 128)) return QNN_E_CUDA;
     p.vec_c = qnn_aligned(p.C, 16) && p.ldc % 4 == 0;
     p.vec_x = p.x && qnn_aligned(p.x, 16) && p.ldx % 4 == 0;
-    tf32_gemm_kernel<GEMM_BN, GEMM_STAGES><<<(unsigned)(tiles_m * tiles_n), GEMM_THREADS, L::TOTAL, st>>>(map_a, map_b, p);
-    return qnn_launch_status();
+    return wide ? launch_gemm<256, 4>(map_a, map_b, p, sms, st) : launch_gemm<128, 6>(map_a, map_b, p, sms, st);
 }
 
 int unpack_codes(const uint32_t *planes, long long rows, long long k, int bits, bool transpose, float *out, long long ld,
                  cudaStream_t st) {
     const long long kw = qnn_row_words_i(k);
-    const dim3 grid((unsigned)qnn_ceil_div(k, 32), (unsigned)qnn_ceil_div(rows, 32));
-    if (transpose) unpack_codes_kernel<true><<<grid, 256, 0, st>>>(planes, rows, k, bits, kw, out, ld);
-    else unpack_codes_kernel<false><<<grid, 256, 0, st>>>(planes, rows, k, bits, kw, out, ld);
+    if (transpose) {
+        const dim3 grid((unsigned)qnn_ceil_div(k, 32), (unsigned)qnn_ceil_div(rows, 256));
+        unpack_codes_kernel<true><<<grid, 256, 0, st>>>(planes, rows, k, bits, kw, out, ld);
+    } else {
+        const dim3 grid((unsigned)qnn_ceil_div(k, 256), (unsigned)qnn_ceil_div(rows, 32));
+        unpack_codes_kernel<false><<<grid, 256, 0, st>>>(planes, rows, k, bits, kw, out, ld);
+    }
     return qnn_launch_status();
 }
 

@@ -141,6 +141,31 @@ def time_mbit(n, bits, reps=5, warmup=3, dev="cuda:0", seed=0):
             "forward_gbs": n * 4 * (1 + bits) / (tf * 1e-3) / 1e9, "backward_gbs": n * 4 * (2 + bits) / (tb * 1e-3) / 1e9}
 
 
+def time_backward(m, n, k, ab, wb, reps=5, warmup=3, dev="cuda:0", seed=0):
+    """Backward products of one FC layer (TF32 tensor-core contractions): whole calls, and the staging part alone."""
+    g = torch.Generator(device=dev).manual_seed(seed)
+    grad = torch.randn((m, n), device=dev, generator=g)
+    x = (torch.rand((m, k), device=dev, generator=g) * 2 - 1)
+    a_planes = qnn.encode_pack(x, ab, 1.0 / (2 ** ab - 1))
+    w_planes = qnn.encode_pack(torch.randn((n, k), device=dev, generator=g).clamp_(-1, 1), wb, 1.0 / (2 ** wb - 1))
+    alpha = 1.0 / ((2 ** ab - 1) * (2 ** wb - 1))
+    out = torch.empty((m, k), dtype=torch.float32, device=dev)
+    gw = torch.empty((n, k), dtype=torch.float32, device=dev)
+    wsd = torch.empty(qnn.lib.qnn_bgemm_backward_data_workspace(m, n, k) + 256, dtype=torch.uint8, device=dev)
+    wsw = torch.empty(qnn.lib.qnn_bgemm_backward_weights_workspace(m, n, k) + 256, dtype=torch.uint8, device=dev)
+    med = lambda f: statistics.median(_time_calls(f, reps, warmup))
+    td = med(lambda i: qnn.bgemm_backward_data(grad, w_planes, k, wb, alpha, out=out, workspace=wsd))
+    te = med(lambda i: qnn.bgemm_backward_data(grad, w_planes, k, wb, alpha, x=x, ab=ab, r=1.0, out=out, workspace=wsd))
+    tw = med(lambda i: qnn.bgemm_backward_weights(grad, a_planes, k, ab, alpha, gw=gw, workspace=wsw))
+    tu = med(lambda i: qnn.unpack_codes_f32(w_planes, n, k, wb, transpose=True))
+    status = qnn.tensor_path_status()
+    fl = 2.0 * m * n * k
+    return {"call": "qnn_bgemm_backward", "m": m, "n": n, "k": k, "ab": ab, "wb": wb, "status": status,
+            "data_ms": td, "data_encoder_ms": te, "weights_ms": tw, "unpack_t_ms": tu,
+            "data_tflops": fl / (td * 1e-3) / 1e12, "data_encoder_tflops": fl / (te * 1e-3) / 1e12,
+            "weights_tflops": fl / (tw * 1e-3) / 1e12}
+
+
 def _report(call, Mg, Ng, Kg, ab, wb, times):
     ms = statistics.median(times)
     macs = float(Mg) * Ng * Kg
@@ -165,12 +190,18 @@ def main():
     mb = sub.add_parser("mbit")
     mb.add_argument("--n", type=int, default=1 << 26)
     mb.add_argument("--bits", type=int, default=2)
+    bw = sub.add_parser("backward")
+    bw.add_argument("--m", type=int, default=4096)
+    bw.add_argument("--n", type=int, default=4096)
+    bw.add_argument("--k", type=int, default=4096)
+    bw.add_argument("--ab", type=int, default=2)
+    bw.add_argument("--wb", type=int, default=2)
     k = sub.add_parser("stack")
     k.add_argument("--net", choices=["resnet18", "resnet18_p1", "resnet18_p2", "vgg16"], default="resnet18")
     k.add_argument("--batch", type=int, default=0)
     k.add_argument("--layers", type=str, default="")
     k.add_argument("--table", action="store_true")
-    for s in (g, c, e, k, mb):
+    for s in (g, c, e, k, mb, bw):
         s.add_argument("--reps", type=int, default=5)
         s.add_argument("--warmup", type=int, default=3)
         s.add_argument("--sets", type=int, default=3)
@@ -179,6 +210,8 @@ def main():
         r = time_gemm(a.m, a.n, a.k, a.ab, a.wb, a.reps, a.warmup, a.sets)
     elif a.case == "conv":
         r = time_conv(a.N, a.H, a.W, a.C, a.Cout, a.R, a.S, a.stride, a.pad, a.ab, a.wb, a.reps, a.warmup, a.sets)
+    elif a.case == "backward":
+        r = time_backward(a.m, a.n, a.k, a.ab, a.wb, a.reps, a.warmup)
     elif a.case == "mbit":
         r = time_mbit(a.n, a.bits, a.reps, a.warmup)
     elif a.case == "stack":
