@@ -126,21 +126,41 @@ struct GemmParams {
     float alpha;
     float *C;
     long long ldc;
-    int vec_c;                          // 1: C rows may be written as float4
     const float *x;                     // optional [M][N] (leading dimension ldx): fuse Eq. 12 with `bits` planes and range r
     long long ldx;
-    int vec_x;
     int bits;
     float r;
+    MbitPlaneConsts enc;                // constants of Eq. 12 for `bits` planes
     int tiles_n, tiles;
 };
+
+// One column of a 32 x 32 chunk (this lane's), rows_here rows: C = Eq. 12 applied to the staged products and x.
+// Four rows are in flight at a time; the element arithmetic has no branch, so their instructions interleave.
+template <int BITS>
+__device__ __forceinline__ void epilogue_encoder(float *cptr, long long ldc, const float *xptr, long long ldx,
+                                                 const float *stage_col, int rows_here, float r, const MbitPlaneConsts &c) {
+    int rr = 0;
+#pragma unroll 1
+    for (; rr + 4 <= rows_here; rr += 4) {
+        float xv[4], o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) xv[e] = __ldcs(xptr + (long long)(rr + e) * ldx);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e] = mbit_backward_shared<BITS>(xv[e], r, stage_col[(rr + e) * 33], c);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) cptr[(long long)(rr + e) * ldc] = o[e];
+    }
+    for (; rr < rows_here; ++rr)
+        cptr[(long long)rr * ldc] = mbit_backward_shared<BITS>(__ldcs(xptr + (long long)rr * ldx), r, stage_col[rr * 33], c);
+}
 
 template <int BN, int STAGES>
 struct GemmSmem {
     static constexpr int A_BYTES = BM * BK * 4;
     static constexpr int B_BYTES = BN * BK * 4;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int EPI_OFFSET = STAGES * STAGE_BYTES;                       // per epilogue warp a 32 x 33 fp32 tile
+    static constexpr int BAR_OFFSET = EPI_OFFSET + EPI_WARPS * 32 * 33 * 4;
     static constexpr int TOTAL = BAR_OFFSET + (2 * STAGES + 4) * 8 + 16 + 1024;   // + slack for the 1024-byte alignment
 };
 
@@ -235,44 +255,41 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tf32_gemm_kernel(const __grid
             const int buf = local & 1;
             if (!mbar_wait(&acc_full[buf], (uint32_t)(local >> 1) & 1u, abort_flag, 2)) break;
             tc_fence_after();
-            const int row = m0 + q * 32 + lane;
+            // Each 32 x 32 chunk goes through the warp's shared tile: tensor memory hands a thread one row, memory
+            // wants a warp on one row, so that every access to C and x is a whole 128-byte line.
+            float *stage = reinterpret_cast<float *>(smem + L::EPI_OFFSET) + (warp - 2) * (32 * 33);
 #pragma unroll 1
             for (int c0 = half * 32; c0 < BN; c0 += 64) {
                 if (n0 + c0 >= p.N) break;                 // uniform over the warp
                 float v[32];
                 tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
-                if (row < p.M) {
-                    float *crow = p.C + (long long)row * p.ldc + n0 + c0;
-                    const float *xrow = p.x ? p.x + (long long)row * p.ldx + n0 + c0 : nullptr;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        const int col = n0 + c0 + i;
-                        const bool whole = col + 3 < p.N;
-                        float o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) o[e] = __fmul_rn(v[i + e], p.alpha);
-                        if (xrow) {
-                            float xv[4] = {0.f, 0.f, 0.f, 0.f};
-                            if (whole && p.vec_x) {
-                                const float4 t = __ldcs(reinterpret_cast<const float4 *>(xrow + i));
-                                xv[0] = t.x; xv[1] = t.y; xv[2] = t.z; xv[3] = t.w;
-                            } else {
-                                for (int e = 0; e < 4; ++e)
-                                    if (col + e < p.N) xv[e] = __ldcs(xrow + i + e);
-                            }
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) o[e] = mbit_backward_shared(xv[e], p.r, o[e], p.bits);
+                for (int i = 0; i < 32; ++i) stage[lane * 33 + i] = __fmul_rn(v[i], p.alpha);
+                __syncwarp();
+                const int col = n0 + c0 + lane;
+                const int rows_here = min(32, p.M - (m0 + q * 32));
+                if (col < p.N) {
+                    float *cptr = p.C + (long long)(m0 + q * 32) * p.ldc + col;
+                    if (p.x) {
+                        const float *xptr = p.x + (long long)(m0 + q * 32) * p.ldx + col;
+                        switch (p.bits) {
+                            case 1: epilogue_encoder<1>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            case 2: epilogue_encoder<2>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            case 3: epilogue_encoder<3>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            case 4: epilogue_encoder<4>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            case 5: epilogue_encoder<5>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            case 6: epilogue_encoder<6>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            case 7: epilogue_encoder<7>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
+                            default: epilogue_encoder<8>(cptr, p.ldc, xptr, p.ldx, stage + lane, rows_here, p.r, p.enc); break;
                         }
-                        if (whole && p.vec_c) {
-                            *reinterpret_cast<float4 *>(crow + i) = make_float4(o[0], o[1], o[2], o[3]);
-                        } else {
-                            for (int e = 0; e < 4; ++e)
-                                if (col + e < p.N) crow[i + e] = o[e];
-                        }
+                    } else {
+#pragma unroll 8
+                        for (int rr = 0; rr < rows_here; ++rr) cptr[(long long)rr * p.ldc] = stage[rr * 33 + lane];
                     }
                 }
+                __syncwarp();
             }
-            // the buffer is free once every epilogue warp has its values in registers
+            // the buffer is free once every epilogue warp has read its part out
             tc_fence_before();
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&acc_empty[buf])) : "memory");
@@ -315,7 +332,7 @@ __global__ void __launch_bounds__(256) unpack_codes_kernel(const uint32_t *__res
             int t = 0;
 #pragma unroll
             for (int b = 0; b < 8; ++b) t |= (int)((w[b] >> c) & 1u) << b;
-            if (col < k) __stcs(out + col * ld + row, (float)(2 * t) - amax);
+            if (col < k) out[col * ld + row] = (float)(2 * t) - amax;   // default policy: the GEMM reads it next, from L2
         }
     } else {
         const long long r0 = (long long)blockIdx.y * 32, wcol = (long long)blockIdx.x * 8 + ty;
@@ -329,7 +346,7 @@ __global__ void __launch_bounds__(256) unpack_codes_kernel(const uint32_t *__res
 #pragma unroll
             for (int b = 0; b < 8; ++b)
                 if (b < bits) t |= (int)((__ldg(planes + (row * bits + b) * kw + wcol) >> tx) & 1u) << b;
-            if (col < k) __stcs(out + row * ld + col, (float)(2 * t) - amax);
+            if (col < k) out[row * ld + col] = (float)(2 * t) - amax;
         }
     }
 }
@@ -435,8 +452,6 @@ int run_gemm(const float *A, long long lda, const float *B, long long ldb, GemmP
     const bool wide = ((long long)(p.M + BM - 1) / BM) * ((p.N + 255) / 256) >= sms;
     CUtensorMap map_a, map_b;
     if (!make_map(&map_a, A, p.M, p.K, lda, BM) || !make_map(&map_b, B, p.N, p.K, ldb, wide ? 256 : 128)) return QNN_E_CUDA;
-    p.vec_c = qnn_aligned(p.C, 16) && p.ldc % 4 == 0;
-    p.vec_x = p.x && qnn_aligned(p.x, 16) && p.ldx % 4 == 0;
     return wide ? launch_gemm<256, 4>(map_a, map_b, p, sms, st) : launch_gemm<128, 6>(map_a, map_b, p, sms, st);
 }
 
@@ -508,6 +523,7 @@ extern "C" int qnn_bgemm_backward_data(const float *g, const uint32_t *w_planes,
     p.alpha = alpha;
     p.C = out; p.ldc = (long long)k;
     p.x = x; p.ldx = (long long)k; p.bits = ab; p.r = r;
+    if (x) p.enc = mbit_plane_consts(ab);
     return run_gemm(a, lda, wqt, ldn, p, st);
 }
 
