@@ -315,24 +315,25 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tf32_gemm_kernel(const __grid
 // block covers 32 rows x 256 columns (warp w owns plane word w of eight).  TRANSPOSE = true: out[col][row], a block
 // covers 256 rows x 32 columns (one plane word per row), so that each output row receives 1 KiB in one piece.
 // The 32 threads of a warp run along the contiguous index of the output: every store instruction writes one line.
-template <bool TRANSPOSE>
+template <bool TRANSPOSE, int BITS>
 __global__ void __launch_bounds__(256) unpack_codes_kernel(const uint32_t *__restrict__ planes, long long rows, long long k,
-                                                          int bits, long long kw, float *__restrict__ out, long long ld) {
+                                                          long long kw, float *__restrict__ out, long long ld) {
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const float amax = (float)((1 << bits) - 1);
+    const float amax = (float)((1 << BITS) - 1);
     if (TRANSPOSE) {
         const long long row = (long long)blockIdx.y * 256 + threadIdx.x, wcol = blockIdx.x;
         if (row >= rows) return;
-        uint32_t w[8];
+        uint32_t w[BITS];
 #pragma unroll
-        for (int b = 0; b < 8; ++b) w[b] = b < bits ? __ldg(planes + (row * bits + b) * kw + wcol) : 0u;
+        for (int b = 0; b < BITS; ++b) w[b] = __ldg(planes + (row * BITS + b) * kw + wcol);
+        const int ncol = (int)min(32ll, k - wcol * 32);
+        float *o = out + wcol * 32 * ld + row;
 #pragma unroll 8
         for (int c = 0; c < 32; ++c) {
-            const long long col = wcol * 32 + c;
             int t = 0;
 #pragma unroll
-            for (int b = 0; b < 8; ++b) t |= (int)((w[b] >> c) & 1u) << b;
-            if (col < k) out[col * ld + row] = (float)(2 * t) - amax;   // default policy: the GEMM reads it next, from L2
+            for (int b = 0; b < BITS; ++b) t |= (int)((w[b] >> c) & 1u) << b;
+            if (c < ncol) o[c * ld] = (float)(2 * t) - amax;   // default cache policy: the GEMM reads it next, from L2
         }
     } else {
         const long long r0 = (long long)blockIdx.y * 32, wcol = (long long)blockIdx.x * 8 + ty;
@@ -344,8 +345,7 @@ __global__ void __launch_bounds__(256) unpack_codes_kernel(const uint32_t *__res
             if (row >= rows) break;
             int t = 0;
 #pragma unroll
-            for (int b = 0; b < 8; ++b)
-                if (b < bits) t |= (int)((__ldg(planes + (row * bits + b) * kw + wcol) >> tx) & 1u) << b;
+            for (int b = 0; b < BITS; ++b) t |= (int)((__ldg(planes + (row * BITS + b) * kw + wcol) >> tx) & 1u) << b;
             if (col < k) out[row * ld + col] = (float)(2 * t) - amax;
         }
     }
@@ -455,16 +455,24 @@ int run_gemm(const float *A, long long lda, const float *B, long long ldb, GemmP
     return wide ? launch_gemm<256, 4>(map_a, map_b, p, sms, st) : launch_gemm<128, 6>(map_a, map_b, p, sms, st);
 }
 
+template <bool TRANSPOSE>
+void launch_unpack(const uint32_t *planes, long long rows, long long k, int bits, long long kw, float *out, long long ld,
+                   cudaStream_t st) {
+    const dim3 grid = TRANSPOSE ? dim3((unsigned)qnn_ceil_div(k, 32), (unsigned)qnn_ceil_div(rows, 256))
+                                : dim3((unsigned)qnn_ceil_div(k, 256), (unsigned)qnn_ceil_div(rows, 32));
+#define UNPACK_CASE(B) case B: unpack_codes_kernel<TRANSPOSE, B><<<grid, 256, 0, st>>>(planes, rows, k, kw, out, ld); break;
+    switch (bits) {
+        UNPACK_CASE(1) UNPACK_CASE(2) UNPACK_CASE(3) UNPACK_CASE(4) UNPACK_CASE(5) UNPACK_CASE(6) UNPACK_CASE(7)
+        default: unpack_codes_kernel<TRANSPOSE, 8><<<grid, 256, 0, st>>>(planes, rows, k, kw, out, ld); break;
+    }
+#undef UNPACK_CASE
+}
+
 int unpack_codes(const uint32_t *planes, long long rows, long long k, int bits, bool transpose, float *out, long long ld,
                  cudaStream_t st) {
     const long long kw = qnn_row_words_i(k);
-    if (transpose) {
-        const dim3 grid((unsigned)qnn_ceil_div(k, 32), (unsigned)qnn_ceil_div(rows, 256));
-        unpack_codes_kernel<true><<<grid, 256, 0, st>>>(planes, rows, k, bits, kw, out, ld);
-    } else {
-        const dim3 grid((unsigned)qnn_ceil_div(k, 256), (unsigned)qnn_ceil_div(rows, 32));
-        unpack_codes_kernel<false><<<grid, 256, 0, st>>>(planes, rows, k, bits, kw, out, ld);
-    }
+    if (transpose) launch_unpack<true>(planes, rows, k, bits, kw, out, ld, st);
+    else launch_unpack<false>(planes, rows, k, bits, kw, out, ld, st);
     return qnn_launch_status();
 }
 
