@@ -141,3 +141,43 @@ def test_backward_argument_checks():
     with pytest.raises(qnn.QnnError):
         qnn.bgemm_backward_weights(g, planes, 8, 9, 1.0)
     assert qnn.lib.qnn_bgemm_backward_data_workspace(0, 1, 1) == 0
+
+
+@pytest.mark.parametrize("m,n,k,ab,wb", [(4096, 4096, 4096, 2, 2), (3000, 4100, 2050, 3, 4)])
+def test_backward_products_full_size_sampled(m, n, k, ab, wb):
+    """The benchmarked size (and a ragged large one) in the launch configuration run_case.py times: 128 x 256 tiles,
+    persistent CTAs.  Sampled outputs against the oracle: exact for integer gradients, within the bound for real ones."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(m + k)
+    qa, qw = _codes(rng, m, k, ab), _codes(rng, n, k, wb)
+    pa, pw = _planes_dev(qa, ab, dev), _planes_dev(qw, wb, dev)
+    count = 300
+    r_d, c_d = rng.integers(0, m, count), rng.integers(0, k, count)
+    r_w, c_w = rng.integers(0, n, count), rng.integers(0, k, count)
+    r_d[:4], c_d[:4] = [0, m - 1, 0, m - 1], [0, k - 1, k - 1, 0]          # tile corners
+    r_w[:4], c_w[:4] = [0, n - 1, 0, n - 1], [0, k - 1, k - 1, 0]
+    for kind in ("integer", "real"):
+        if kind == "integer":
+            g, alpha = rng.integers(-8, 9, size=(m, n)).astype(np.float32), 0.25
+        else:
+            g, alpha = rng.standard_normal((m, n)).astype(np.float32), 0.8 / ((2 ** ab - 1) * (2 ** wb - 1))
+        gd = torch.from_numpy(g).to(dev)
+        G = qnn.bgemm_backward_data(gd, pw, k, wb, alpha).cpu().numpy().astype(np.float64)
+        GW = qnn.bgemm_backward_weights(gd, pa, k, ab, alpha).cpu().numpy().astype(np.float64)
+        assert qnn.tensor_path_status() == 0
+        want_d = oracle.fc_backward_data_sampled(g, qw, ab, wb, alpha, r_d, c_d)[0]
+        want_w = oracle.fc_backward_weights_sampled(g, qa, ab, wb, alpha, r_w, c_w)[0]
+        if kind == "integer":
+            assert np.array_equal(G[r_d, c_d], want_d) and np.array_equal(GW[r_w, c_w], want_w)
+        else:
+            a32 = float(np.float32(alpha))
+            bd = a32 * np.einsum("in,ni->i", np.abs(g[r_d]).astype(np.float64), np.abs(qw[:, c_d]).astype(np.float64)) \
+                * (2.0 ** -10 + n * 2.0 ** -24)
+            bw = a32 * np.einsum("ri,ri->i", np.abs(g[:, r_w]).astype(np.float64), np.abs(qa[:, c_w]).astype(np.float64)) \
+                * (2.0 ** -10 + m * 2.0 ** -24)
+            assert np.all(np.abs(G[r_d, c_d] - want_d) <= bd) and np.all(np.abs(GW[r_w, c_w] - want_w) <= bw)
+            # every element is finite and the matrix has the scale the samples have (nothing left unwritten)
+            assert np.isfinite(G).all() and np.isfinite(GW).all()
+            assert 0.5 < np.std(G) / np.std(want_d) < 2.0 and 0.5 < np.std(GW) / np.std(want_w) < 2.0
