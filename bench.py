@@ -274,6 +274,57 @@ def int8_tensor_comparison(torch, qnn, dev, a_dev, w_host, sa, sw, planes, packe
         return {"what": "int8 tensor-core GEMM comparison", "unavailable": f"{type(exc).__name__}: {exc}"[:200]}
 
 
+def training_side_leg(torch, qnn, dev, planes, packed, mp, mp_kind):
+    """Outside the timed step: the backward products of the same layer (Algorithm 1 backward) as TF32 tensor-core
+    GEMMs and the streaming encoder derivative, with CUDA events, against the measured bf16 peak scaled by the
+    nominal TF32:bf16 ratio and the measured copy peak."""
+    try:
+        wp, _ = qnn.weights_views(packed, N_SQ, 1, N_SQ, WB)
+        wp = wp.contiguous()
+        m = n = k = N_SQ
+        gen = torch.Generator(device=dev).manual_seed(7)
+        grads = [torch.randn((m, n), device=dev, generator=gen) for _ in range(2)]
+        x = torch.rand((m, k), device=dev, generator=gen) * 2 - 1
+        outs = [torch.empty((m, k), dtype=torch.float32, device=dev) for _ in range(2)]
+        gws = [torch.empty((n, k), dtype=torch.float32, device=dev) for _ in range(2)]
+        wsd = torch.empty(qnn.lib.qnn_bgemm_backward_data_workspace(m, n, k), dtype=torch.uint8, device=dev)
+        wsw = torch.empty(qnn.lib.qnn_bgemm_backward_weights_workspace(m, n, k), dtype=torch.uint8, device=dev)
+        alpha = 1.0 / ((2 ** AB - 1) * (2 ** WB - 1))
+
+        def timed(fn, reps=20):
+            for i in range(3):
+                fn(i)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(reps):
+                fn(i)
+            e1.record()
+            e1.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        t_data = timed(lambda i: qnn.bgemm_backward_data(grads[i % 2], wp, k, WB, alpha, out=outs[i % 2], workspace=wsd))
+        t_enc = timed(lambda i: qnn.bgemm_backward_data(grads[i % 2], wp, k, WB, alpha, x=x, ab=AB, r=1.0, out=outs[i % 2],
+                                                        workspace=wsd))
+        t_w = timed(lambda i: qnn.bgemm_backward_weights(grads[i % 2], planes, k, AB, alpha, gw=gws[i % 2], workspace=wsw))
+        gc = torch.randn((AB, m * k), device=dev, generator=gen)
+        gx = torch.empty(m * k, dtype=torch.float32, device=dev)
+        t_mb = timed(lambda i: qnn.mbit_encoder_backward(x.view(-1), gc, AB, 1.0, gx=gx))
+        status = qnn.tensor_path_status()
+        flop = 2.0 * m * n * k
+        peak = mp["bf16_tflops"] * (1.1 / 2.25)
+        return {"what": "Algorithm 1 backward of the benchmarked layer: whole calls (code unpack / transpose + TF32 tcgen05 GEMM), CUDA events",
+                "workload": f"fc {m}x{n}x{k}, w{WB}a{AB}", "dtype": "tf32 x exact codes, fp32 accumulate",
+                "backward_data_ms": t_data, "backward_data_with_encoder_derivative_ms": t_enc, "backward_weights_ms": t_w,
+                "backward_data_tflops": flop / (t_data * 1e-3) / 1e12, "backward_weights_tflops": flop / (t_w * 1e-3) / 1e12,
+                "roofline": {"bound": "tensor", "achieved": flop / (t_data * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                             "frac": flop / (t_data * 1e-3) / 1e12 / peak,
+                             "peak_kind": f"{mp_kind} bf16 burst x 1.1/2.25 (nominal TF32:bf16)"},
+                "mbit_encoder_backward_gbs": m * k * 4.0 * (2 + AB) / (t_mb * 1e-3) / 1e9, "tensor_path_status": status}
+    except Exception as exc:   # reported beside the benchmark, never fails it
+        return {"what": "Algorithm 1 backward", "unavailable": f"{type(exc).__name__}: {exc}"[:200]}
+
+
 def load_measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -453,6 +504,8 @@ def run_gpu(args):
         }
         if comparison is not None:
             line["comparison_int8_tensor"] = comparison
+        if world == 1:
+            line["training_side"] = training_side_leg(torch, qnn, dev, planes[0], packed, mp, mp_kind)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg()
         print(json.dumps(line), flush=True)
