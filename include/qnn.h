@@ -243,6 +243,19 @@ int qnn_unpack_codes_f32(const uint32_t *planes, size_t rows, size_t k, int bits
 int qnn_tensor_path_status(unsigned int *status);
 
 /*
+ * Comparison only, not the paper's method: the product of qnn_bgemm computed as ONE signed 8-bit tensor-core GEMM
+ * on the unpacked odd codes (Eq. 8 read backwards: q = sum_i 2^(i-1) * plane_i), to show what the bit-plane
+ * decomposition competes with on this GPU.  Arguments as qnn_bgemm (a_planes, w_packed of a fully-connected layer
+ * with taps = 1, alpha); acc (optional) receives the int32 accumulators [Mg][Ng], out (optional) float(acc) * alpha;
+ * at least one of them is given.  Both are bit-identical to qnn_bgemm's.  ab, wb <= 7 (QNN_E_RANGE for 8: the code
+ * +-255 does not fit a signed byte), Kg*A*B < 2^31.  workspace: device scratch of at least
+ * qnn_bgemm_int8_tensor_workspace(Mg, Ng, Kg) bytes, 256-byte aligned, owned by the caller (holds the unpacked codes).
+ */
+size_t qnn_bgemm_int8_tensor_workspace(int64_t Mg, int Ng, int Kg);
+int qnn_bgemm_int8_tensor(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg,
+                          float alpha, int32_t *acc, float *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * max_i |x[i]| into *out (device fp32), for workloads whose grid step is derived
  * from the tensor's range.  Not a step of the paper's method (its range r is a
  * fixed or learned constant, Eq. 9 / Eq. 15).  NaNs are ignored.

@@ -14,6 +14,9 @@ static inline int64_t qnn_row_words_i(int64_t k) { return qnn_ceil_div(qnn_ceil_
 static inline int64_t qnn_w_row_words_i(int taps, int c_in) {
     return qnn_ceil_div((int64_t)taps * qnn_ceil_div(c_in, 32), 4) * 4;
 }
+// Defined in backward.cu: device word shared by all tensor-path kernels (see qnn_tensor_path_status).
+unsigned int *qnn_tc_error_word();
+
 static inline int qnn_launch_status() { return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA; }
 
 // Unsigned code t in [0, 2^bits - 1] of a real value (odd code q = 2t - (2^bits - 1)).

@@ -23,7 +23,7 @@ EXPORTS = [
     "qnn_bgemm_encode", "qnn_bconv2d_encode", "qnn_bconv2d_general", "qnn_mbit_encoder_forward",
     "qnn_mbit_encoder_backward", "qnn_bgemm_backward_data_workspace", "qnn_bgemm_backward_data",
     "qnn_bgemm_backward_weights_workspace", "qnn_bgemm_backward_weights", "qnn_unpack_codes_f32",
-    "qnn_tensor_path_status",
+    "qnn_tensor_path_status", "qnn_bgemm_int8_tensor_workspace", "qnn_bgemm_int8_tensor",
     "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -69,6 +69,9 @@ def _load() -> C.CDLL:
     lib.qnn_bgemm_backward_weights.argtypes = [p, p, sz, sz, sz, i, f, p, p, sz, p]
     lib.qnn_unpack_codes_f32.argtypes = [p, sz, sz, i, i, p, sz, p]
     lib.qnn_tensor_path_status.argtypes = [C.POINTER(C.c_uint)]
+    lib.qnn_bgemm_int8_tensor_workspace.restype = sz
+    lib.qnn_bgemm_int8_tensor_workspace.argtypes = [i64, i, i]
+    lib.qnn_bgemm_int8_tensor.argtypes = [p, i, p, i, i64, i, i, f, p, p, p, sz, p]
     lib.qnn_absmax_f32.argtypes = [p, sz, p, p]
     lib.qnn_fc_forward_host.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, p]
     lib.qnn_fc_forward_host_pipelined.argtypes = [p, i64, i, i, f, u, p, i, i, f, p, p, p, p, i64, C.POINTER(C.c_void_p), i]
@@ -302,6 +305,21 @@ def unpack_codes_f32(planes: torch.Tensor, rows: int, k: int, bits: int, transpo
     _check(lib.qnn_unpack_codes_f32(_ptr(planes), rows, k, bits, int(transpose), _ptr(out), rows if transpose else k,
                                     _stream(stream)), "qnn_unpack_codes_f32")
     return out
+
+
+def bgemm_int8_tensor(a_planes: torch.Tensor, ab: int, w_packed: torch.Tensor, wb: int, Mg: int, Ng: int, Kg: int,
+                      alpha: float, want_acc: bool = True, out: torch.Tensor | None = None, acc: torch.Tensor | None = None,
+                      workspace: torch.Tensor | None = None, stream=None):
+    """Comparison path: the product of bgemm as one int8 tensor-core GEMM on the unpacked codes -> (out fp32, acc int32)."""
+    dev = a_planes.device
+    if out is None:
+        out = torch.empty((Mg, Ng), dtype=torch.float32, device=dev)
+    if acc is None and want_acc:
+        acc = torch.empty((Mg, Ng), dtype=torch.int32, device=dev)
+    ws = _workspace(lib.qnn_bgemm_int8_tensor_workspace(Mg, Ng, Kg), dev, workspace)
+    _check(lib.qnn_bgemm_int8_tensor(_ptr(a_planes), ab, _ptr(w_packed), wb, Mg, Ng, Kg, float(alpha), _ptr(acc), _ptr(out),
+                                     _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)), "qnn_bgemm_int8_tensor")
+    return out, acc
 
 
 def tensor_path_status() -> int:
