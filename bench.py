@@ -268,8 +268,28 @@ def int8_tensor_comparison(torch, qnn, dev, a_dev, w_host, sa, sw, planes, packe
             e1.synchronize()
             times.append(e0.elapsed_time(e1))
         ms = statistics.median(times)
+        # the same product through this library's own tcgen05 kind::i8 kernel (unpack of both operands included)
+        ws = torch.empty(qnn.lib.qnn_bgemm_int8_tensor_workspace(Mg, N_SQ, Kg), dtype=torch.uint8, device=dev)
+        out8 = torch.empty((Mg, N_SQ), dtype=torch.float32, device=dev)
+        acc8 = torch.empty((Mg, N_SQ), dtype=torch.int32, device=dev)
+        qnn.bgemm_int8_tensor(planes, AB, packed, WB, Mg, N_SQ, Kg, alpha, out=out8, acc=acc8, workspace=ws)
+        torch.cuda.synchronize()
+        same8 = bool(torch.equal(acc8, acc))
+        own = []
+        for _ in range(13):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            qnn.bgemm_int8_tensor(planes, AB, packed, WB, Mg, N_SQ, Kg, alpha, want_acc=False, out=out8, workspace=ws)
+            e1.record()
+            e1.synchronize()
+            own.append(e0.elapsed_time(e1))
+        ms8 = statistics.median(own[3:])
         return {"what": "int8 tensor-core GEMM on the unpacked odd codes, cuBLASLt via torch._int_mm (library call, comparison only)",
-                "ms": ms, "equiv_int_gops": 2.0 * Mg * N_SQ * Kg / (ms * 1e-3) / 1e9, "int32_result_identical_to_qnn_bgemm": same}
+                "ms": ms, "equiv_int_gops": 2.0 * Mg * N_SQ * Kg / (ms * 1e-3) / 1e9, "int32_result_identical_to_qnn_bgemm": same,
+                "own_tcgen05_i8": {"what": "qnn_bgemm_int8_tensor: planes -> int8 codes (both operands) + tcgen05 kind::i8 GEMM, fp32 output (comparison only)",
+                                   "ms": ms8, "equiv_int_gops": 2.0 * Mg * N_SQ * Kg / (ms8 * 1e-3) / 1e9,
+                                   "int32_result_identical_to_qnn_bgemm": same8,
+                                   "tensor_path_status": qnn.tensor_path_status()}}
     except Exception as exc:   # comparison only: never fail the benchmark over it
         return {"what": "int8 tensor-core GEMM comparison", "unavailable": f"{type(exc).__name__}: {exc}"[:200]}
 
