@@ -141,6 +141,7 @@ struct GemmParams {
     float r;
     MbitPlaneConsts enc;                // constants of Eq. 12 for `bits` planes
     int tiles_n, tiles;
+    int whole_items, items;             // work items: tiles [0, whole_items) whole, the rest split into two halves along N
 };
 
 // One column of a 32 x 32 chunk (this lane's), rows_here rows: C = Eq. 12 applied to the staged products and x.
@@ -163,6 +164,23 @@ __device__ __forceinline__ void epilogue_encoder(float *cptr, long long ldc, con
         cptr[(long long)rr * ldc] = mbit_backward_shared<BITS>(__ldcs(xptr + (long long)rr * ldx), r, stage_col[rr * 33], c);
 }
 
+// Work item w of a launch: whole tiles first; the tiles of a ragged last round (fewer than half as many as there are
+// CTAs) are split into two halves along N so that the round takes about half a tile's time instead of a whole one.
+struct WorkItem {
+    int m0, n0, width;
+};
+template <int BN>
+__device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p) {
+    int tile = w, off = 0, width = BN;
+    if (w >= p.whole_items) {
+        const int r = w - p.whole_items;
+        tile = p.whole_items + (r >> 1);
+        off = (r & 1) * (BN / 2);
+        width = BN / 2;
+    }
+    return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN + off, width};
+}
+
 template <int BN, int STAGES>
 struct GemmSmem {
     static constexpr int A_BYTES = BM * BK_BYTES;
@@ -177,8 +195,9 @@ struct GemmSmem {
 // (2 x BN columns), so the epilogue of one tile runs under the main loop of the next.
 template <int BN, int STAGES, int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                                   const __grid_constant__ CUtensorMap map_b,
-                                                                   const GemmParams p) {
+                                                                 const __grid_constant__ CUtensorMap map_b,
+                                                                 const __grid_constant__ CUtensorMap map_b_half,
+                                                                 const GemmParams p) {
     using L = GemmSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -215,15 +234,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     if (warp == 0) {
         if (lane == 0) {
             long long it = 0;                                 // stage uses so far, over all tiles
-            for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x) {
-                const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+            for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x) {
+                const WorkItem wi = work_item<BN>(w, p);
+                const bool whole = wi.width == BN;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                     if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err)) break;
-                    mbar_expect_tx(&full[s], L::STAGE_BYTES);
-                    tma_load_2d(smem + s * L::STAGE_BYTES, &map_a, &full[s], kb * BK, m0);
-                    tma_load_2d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], kb * BK, n0);
+                    mbar_expect_tx(&full[s], whole ? L::STAGE_BYTES : L::A_BYTES + L::B_BYTES / 2);
+                    tma_load_2d(smem + s * L::STAGE_BYTES, &map_a, &full[s], kb * BK, wi.m0);
+                    tma_load_2d(smem + s * L::STAGE_BYTES + L::A_BYTES, whole ? &map_b : &map_b_half, &full[s], kb * BK, wi.n0);
                 }
             }
             if (*abort_flag) {   // let the copies still in flight land before the CTA's shared memory goes away
@@ -233,10 +253,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_kmajor<BN, KIND>();
             long long it = 0;
             int local = 0;
-            for (int tile = blockIdx.x; tile < p.tiles && !*abort_flag; tile += gridDim.x, ++local) {
+            for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x, ++local) {
+                const uint32_t idesc = work_item<BN>(w, p).width == BN ? idesc_kmajor<BN, KIND>() : idesc_kmajor<BN / 2, KIND>();
                 const int buf = local & 1;
                 if (!mbar_wait(&acc_empty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag, 3, p.err)) break;
                 tc_fence_after();
@@ -260,8 +280,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         const int q = warp & 3;                            // a warp reaches the 32 lanes [32*(warp%4), +32) only
         const int half = (warp - 2) >> 2;                  // which of the two warps of this quarter
         int local = 0;
-        for (int tile = blockIdx.x; tile < p.tiles; tile += gridDim.x, ++local) {
-            const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+        for (int w = blockIdx.x; w < p.items; w += gridDim.x, ++local) {
+            const WorkItem wi = work_item<BN>(w, p);
+            const int m0 = wi.m0, n0 = wi.n0;
             const int buf = local & 1;
             if (!mbar_wait(&acc_full[buf], (uint32_t)(local >> 1) & 1u, abort_flag, 2, p.err)) break;
             tc_fence_after();
@@ -269,7 +290,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             // wants a warp on one row, so that every access to C and x is a whole 128-byte line.
             float *stage = reinterpret_cast<float *>(smem + L::EPI_OFFSET) + (warp - 2) * (32 * 33);
 #pragma unroll 1
-            for (int c0 = half * 32; c0 < BN; c0 += 64) {
+            for (int c0 = half * 32; c0 < wi.width; c0 += 64) {
                 if (n0 + c0 >= p.N) break;                 // uniform over the warp
                 uint32_t v[32];
                 tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
@@ -325,7 +346,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     __syncthreads();
     if (warp == 1) {
         // every MMA that was issued has retired once the last committed tile's barrier has completed its phase
-        const int mine = p.tiles > (int)blockIdx.x ? (p.tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+        const int mine = p.items > (int)blockIdx.x ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
         if (mine > 0) {
             const int last = mine - 1;
             for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(&acc_full[last & 1], (uint32_t)(last >> 1) & 1u); ++w) {}
@@ -372,7 +393,8 @@ bool make_map(CUtensorMap *map, const void *base, long long rows, long long cols
 long long pad32(long long v) { return (v + 31) / 32 * 32; }
 
 template <int BN, int STAGES, int KIND>
-int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, GemmParams p, int sms, cudaStream_t st) {
+int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtensorMap &map_b_half, GemmParams p, int sms,
+                cudaStream_t st) {
     using L = GemmSmem<BN, STAGES>;
     static bool attr_set = false;   // per process; set again on the next call if it failed
     if (!attr_set) {
@@ -386,7 +408,11 @@ int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, GemmParams p
     p.tiles_n = (int)tiles_n;
     p.tiles = (int)(tiles_m * tiles_n);
     const int grid = p.tiles < sms ? p.tiles : sms;
-    tc_gemm_kernel<BN, STAGES, KIND><<<grid, GEMM_THREADS, L::TOTAL, st>>>(map_a, map_b, p);
+    const int rem = p.tiles % grid;
+    const bool split = rem > 0 && 2 * rem <= grid;
+    p.whole_items = split ? p.tiles - rem : p.tiles;
+    p.items = split ? p.tiles + rem : p.tiles;
+    tc_gemm_kernel<BN, STAGES, KIND><<<grid, GEMM_THREADS, L::TOTAL, st>>>(map_a, map_b, map_b_half, p);
     return qnn_launch_status();
 }
 
@@ -411,10 +437,12 @@ int run_gemm(const void *A, long long lda, const void *B, long long ldb, GemmPar
     const int sms = sm_count();
     if (sms <= 0) return QNN_E_CUDA;
     const bool wide = ((long long)(p.M + BM - 1) / BM) * ((p.N + 255) / 256) >= sms;
-    CUtensorMap map_a, map_b;
-    if (!make_map(&map_a, A, p.M, p.K, lda, BM, KIND) || !make_map(&map_b, B, p.N, p.K, ldb, wide ? 256 : 128, KIND))
+    CUtensorMap map_a, map_b, map_b_half;
+    if (!make_map(&map_a, A, p.M, p.K, lda, BM, KIND) || !make_map(&map_b, B, p.N, p.K, ldb, wide ? 256 : 128, KIND) ||
+        !make_map(&map_b_half, B, p.N, p.K, ldb, wide ? 128 : 64, KIND))
         return QNN_E_CUDA;
-    return wide ? launch_gemm<256, 4, KIND>(map_a, map_b, p, sms, st) : launch_gemm<128, 6, KIND>(map_a, map_b, p, sms, st);
+    return wide ? launch_gemm<256, 4, KIND>(map_a, map_b, map_b_half, p, sms, st)
+                : launch_gemm<128, 6, KIND>(map_a, map_b, map_b_half, p, sms, st);
 }
 
 }  // namespace
