@@ -35,6 +35,11 @@ MUTATIONS = {
     "backward_plane_weight_off_by_one": ("sum += ldexp(part, m + j - 2);\n                }\n                gw[", "sum += ldexp(part, m + j - 1);\n                }\n                gw["),
     "backward_drops_alpha": ("part += ((double)alpha * (double)g[r * Ng + n]) * plane_of(qa[r * Kg + k], ab, m);\n                    sum += ldexp(part, m + j - 2);\n                }\n                gw[", "part += ((double)g[r * Ng + n]) * plane_of(qa[r * Kg + k], ab, m);\n                    sum += ldexp(part, m + j - 2);\n                }\n                gw["),
     "backward_plane_sign": ("return ((t >> (i - 1)) & 1) ? 1.0 : -1.0;", "return ((t >> (i - 1)) & 1) ? -1.0 : 1.0;"),
+    "mbit_lower_planes_not_negated": ("c[(size_t)(m - 1) * n + e] = (m == bits) ? sgn : -sgn;", "c[(size_t)(m - 1) * n + e] = sgn;"),
+    "mbit_frequency_uses_2_to_M": ("const float k = (float)((1 << bits) - 1) / (float)(1 << m);", "const float k = (float)(1 << bits) / (float)(1 << m);"),
+    "mbit_derivative_not_windowed": ("if (xn >= -1.0 && xn <= 1.0) {", "if (1) {"),
+    "mbit_derivative_sine": ("const double d = k * pi * cos(k * pi * xn);", "const double d = k * pi * sin(k * pi * xn);"),
+    "mbit_derivative_forgets_r": ("gx[e] = g / (double)r;", "gx[e] = g;"),
     "scale_in_double": ("out[i] = (float)acc[i] * alpha;", "out[i] = (float)((double)acc[i] * (double)alpha * (1.0 + 1e-6));"),
 }
 
