@@ -15,6 +15,7 @@ What each function follows in the paper:
 * ``scale``        -- the fixed scaling factor of Eq. 9 / Alg. 1 forward pass.
 * ``mbit_encoder_forward`` / ``mbit_encoder_backward`` -- trigonometric encoder of Eq. 10 and its derivative, Eq. 12.
 * ``affine``       -- per-feature affine that replaces the scale when batch normalisation follows (Section 3.2).
+* ``eq16_speedup`` -- the paper's analytic speed-up model S_MK (Eq. 16, Section 4.6), plain arithmetic.
 """
 from __future__ import annotations
 
@@ -287,3 +288,16 @@ def fc_backward_weights_sampled(g, qa, ab: int, wb: int, alpha: float, rows, col
                                                       rows.size, _ptr(rows), _ptr(cols), _ptr(out)),
            "fc_backward_weights_sampled")
     return out
+
+
+def eq16_speedup(n: int, m_bits: int, k_bits: int, gamma: float = 1.91, beta: float | None = None, reg_len: int = 64):
+    """Eq. 16 (Section 4.6): modelled speed-up S_MK of an M-bit x K-bit bit-plane dot product of length n over
+    n multiply-accumulates.  The numerator is n MACs, each worth gamma bitwise operations; the denominator charges
+    each of the M*K plane pairs gamma + 2*ceil(n/L) operations (xnor and bit-count per L-element register word)
+    and the M*K - 1 additions that combine the pairs beta each.  The paper takes gamma = 1.91, L = 64 and
+    beta = gamma/2 (the default here when beta is None)."""
+    if beta is None:
+        beta = gamma / 2.0
+    pairs = m_bits * k_bits
+    words = -(-int(n) // int(reg_len))
+    return (n * gamma) / (pairs * (gamma + 2 * words) + (pairs - 1) * beta)

@@ -506,3 +506,34 @@ def test_backward_products_special_cases(ab, wb):
     assert np.array_equal(oracle.fc_backward_data_sampled(g, qw, ab, wb, alpha, rows, cols), ga[:, rows, cols])
     rows = np.array([9, 0, 4, 4])
     assert np.array_equal(oracle.fc_backward_weights_sampled(g, qa, ab, wb, alpha, rows, cols), gw[:, rows, cols])
+
+
+# ---- Eq. 16 (Section 4.6): the analytic speed-up model -------------------------------------------------------------
+
+def test_eq16_reproduces_the_printed_two_bit_speedup(golden_dir):
+    rows = [ln.split() for ln in (golden_dir / "eq16_speedup.txt").read_text().splitlines()
+            if ln.strip() and not ln.startswith("#")]
+    assert rows
+    for n, m, k, gamma, L, printed, allowance in rows:
+        s = oracle.eq16_speedup(int(n), int(m), int(k), gamma=float(gamma), reg_len=int(L))
+        assert abs(s - float(printed)) <= float(allowance)
+        assert abs(oracle.eq16_speedup(int(n), int(m), int(k), gamma=float(gamma), beta=0.0, reg_len=int(L))
+                   - float(printed)) > float(allowance)          # the beta term is visible at this precision
+
+
+def test_eq16_limits_and_shape():
+    g, L = 1.91, 64
+    # long vectors: the gamma and beta terms vanish against 2*ceil(n/L) per pair -> gamma*L/(2*M*K)
+    for m, k in ((1, 1), (2, 2), (3, 5), (8, 8)):
+        s = oracle.eq16_speedup(1 << 30, m, k, g, None, L)
+        assert math.isclose(s, g * L / (2 * m * k), rel_tol=1e-5)
+        # the model only sees the number of plane pairs M*K
+        assert oracle.eq16_speedup(8192, m, k) == oracle.eq16_speedup(8192, k, m)
+    assert oracle.eq16_speedup(8192, 2, 6) == oracle.eq16_speedup(8192, 3, 4)
+    # more pairs never help; one pair of one word: n*gamma / (gamma + 2)
+    vals = [oracle.eq16_speedup(8192, b, b) for b in range(1, 9)]
+    assert all(a > b for a, b in zip(vals, vals[1:]))
+    assert math.isclose(oracle.eq16_speedup(64, 1, 1, g, 0.0, L), 64 * g / (g + 2))
+    # a dropped beta term or a floor instead of the ceiling would move these
+    assert math.isclose(oracle.eq16_speedup(65, 1, 1, g, None, L), 65 * g / (g + 4))
+    assert math.isclose(oracle.eq16_speedup(128, 2, 1, 2.0, 3.0, 64), 128 * 2.0 / (2 * (2.0 + 4) + 3.0))
