@@ -1,26 +1,73 @@
 // qnn_encode_pack, qnn_pack_weights, qnn_absmax_f32: real tensors -> bit planes.
 //
-// Both packers are bandwidth-bound streaming kernels.  A warp owns 128 consecutive
-// elements of one row: lane L reads elements 32*j + L (j = 0..3, four coalesced
-// 128-byte requests), quantizes them, and one __ballot_sync per plane and j turns
-// the warp's 32 decisions into one canonical word (lane L -> bit L).  Lane i then
-// holds the four words of plane i and stores them as one 16-byte vector.
+// Activations (qnn_encode_pack) take one of two kernels:
+//  * encode_pack_lanes_kernel (source 16-byte aligned, ldx a multiple of 4: the usual case): a lane owns a
+//    whole output word, i.e. 32 consecutive elements; see the comment above the kernel.
+//  * encode_pack_kernel (any alignment): a warp owns 128 consecutive elements of one row, lane L reads
+//    elements 32*j + L (four coalesced 128-byte requests) and one __ballot_sync per plane and j turns the
+//    warp's 32 decisions into one canonical word (lane L -> bit L); lane i stores plane i's four words.
+// The weight packer (offline) uses the ballot scheme as well.
 #include "qnn_internal.cuh"
+#include <string.h>
 
 namespace {
 
 constexpr int kEncThreads = 256;
+
+// The code t of qnn_code_t without a float->int conversion.  Conversions run on the XU pipe, whose rate made
+// them the bottleneck of this kernel (ncu: XU saturated, DRAM at half its rate).  Two rewrites, both exact:
+//  * For x <= 0 the quantizer takes ceil(v) - 1, which equals floor(v) unless v is an integer; for a positive
+//    float v that is floor(pred(v)) with pred(v) the next float below v (bit pattern - 1): an integer v >= 1 loses
+//    less than 1, a non-integer v cannot fall below floor(v), which is itself a float.  The pre-clamp keeps
+//    v >= 2^(b-1) * (2^-10 - 2^-23) > 0, so the pattern never wraps.
+//  * floor(y) for 0 <= y < 2^23 is read from the mantissa of y + 2^23 rounded DOWN (one add on the FMA pipe):
+//    the sum's unit in the last place is 1, so rounding down yields exactly 2^23 + floor(y).
+// enc_code_bits returns that sum's bit pattern, 0x4B000000 + t.
+constexpr uint32_t kEncMagicBits = 0x4B000000u;             // bit pattern of 2^23
+__device__ __forceinline__ uint32_t enc_code_bits(float x, float inv2s, float half, float lo, float hi) {
+    x = fminf(fmaxf(x, lo), hi);          // NaN -> lo
+    const float v = __fmaf_rn(x, inv2s, half);
+    const int vb = __float_as_int(v) - ((x > 0.0f) ? 0 : 1);
+    return (uint32_t)__float_as_int(__fadd_rd(__int_as_float(vb), 8388608.0f));
+}
+__device__ __forceinline__ int enc_code_t(float x, float inv2s, float half, float lo, float hi) {
+    return (int)(enc_code_bits(x, inv2s, half, lo, hi) & 0xffu);
+}
+
+// One- and two-bit codes are decided by comparisons alone.  The quantizer is a non-decreasing step function of x,
+// so t = [x >= t_lo] + [x > 0] + [x >= t_hi] for two bits (the middle step, between codes -1 and +1, is at 0 with
+// 0 itself on the lower side) and t = [x > 0] for one bit; t_lo / t_hi are the smallest floats at which the
+// quantizer's own formula (fused multiply-add, then floor / ceil - 1) reaches the next code, found on the host
+// with the same binary32 arithmetic.  NaN fails every comparison (t = 0, the most negative code); with a fused
+// ReLU every x <= 0 and NaN take the code of 0, i.e. the lowest step counts as passed.
+struct EncThresholds { float t_lo, t_hi; };
+
+template <int BITS, bool RELU>
+__device__ __forceinline__ void enc_ballots_small(float x, const EncThresholds th, uint32_t (&b)[BITS]) {
+    const bool c_mid = x > 0.0f;
+    if (BITS == 1) {
+        b[0] = __ballot_sync(0xffffffffu, c_mid);
+    } else {
+        const bool c_hi = x >= th.t_hi;
+        const bool c_lo = RELU ? true : (x >= th.t_lo);
+        b[BITS - 1] = __ballot_sync(0xffffffffu, c_mid);                   // t >= 2 exactly when x > 0
+        b[0] = __ballot_sync(0xffffffffu, (c_lo != c_mid) != c_hi);        // parity of the steps passed
+    }
+}
 
 // A unit is 128 consecutive elements: four ballots per plane give four canonical words.  For rows
 // longer than 64 elements a unit is a 128-element segment of one row (RPU = 1); for shorter rows
 // (NHWC activations with few channels) a unit spans RPU = 2 (k <= 64) or 4 (k <= 32) whole rows so
 // that the lanes stay busy.  UN units are loaded before the first ballot, so 4*UN independent
 // 128-byte requests per warp are in flight.  Unit indices advance incrementally (no division in the loop).
-template <int BITS, int UN, int RPU, bool FULL>
+// MODE 0: any width, codes from the quantizer's formula; MODE 1 / 2 (BITS <= 2, RPU = 1, no rowsum): codes from
+// comparisons against precomputed thresholds, without / with the fused ReLU.
+template <int BITS, int UN, int RPU, bool FULL, int MODE>
 __global__ void __launch_bounds__(kEncThreads)
 encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, float lo, float hi,
-                   uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum, int groups_per_row, int segs_per_row,
-                   int kw, int64_t first_row_step, int first_grp_step) {
+                   const EncThresholds th, uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum,
+                   int groups_per_row, int segs_per_row, int kw, int64_t first_row_step, int first_grp_step) {
+    static_assert(MODE == 0 || (BITS <= 2 && RPU == 1), "threshold mode");
     const float half = (float)(1 << (BITS - 1));
     constexpr int SPAN = 128 / RPU;                       // elements of one row inside a unit (RPU > 1)
     const int lane = threadIdx.x & 31;
@@ -53,24 +100,38 @@ encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx
             const int seg = grp * UN + q;
             if (RPU == 1 && seg >= segs_per_row) break;                            // warp-uniform
             int t[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int kk = (RPU == 1) ? seg * 128 + 32 * j + lane : (32 * j) % SPAN + lane;
-                const int code = qnn_code_t(v[q][j], inv2s, half, lo, hi);
-                t[j] = (FULL || kk < k) ? code : 0;                                // padding bits are 0
-            }
             uint32_t b[BITS][4];
+            if constexpr (MODE != 0) {
+                // (rows that end inside the unit were loaded as 0.0f; their padding bits are cleared below)
 #pragma unroll
-            for (int i = 0; i < BITS; ++i)
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t bj[BITS];
+                    enc_ballots_small<BITS, MODE == 2>(v[q][j], th, bj);
+                    const int k0 = seg * 128 + 32 * j;                          // warp-uniform
+                    const uint32_t keep = FULL ? 0xffffffffu : (k0 + 32 <= k ? 0xffffffffu : (k0 >= k ? 0u : (0xffffffffu >> (32 - (k - k0)))));
 #pragma unroll
-                for (int j = 0; j < 4; ++j) b[i][j] = __ballot_sync(0xffffffffu, t[j] & (1 << i));
+                    for (int i = 0; i < BITS; ++i) b[i][j] = bj[i] & keep;
+                    t[j] = 0;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int kk = (RPU == 1) ? seg * 128 + 32 * j + lane : (32 * j) % SPAN + lane;
+                    const int code = enc_code_t(v[q][j], inv2s, half, lo, hi);
+                    t[j] = (FULL || kk < k) ? code : 0;                                // padding bits are 0
+                }
+#pragma unroll
+                for (int i = 0; i < BITS; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) b[i][j] = __ballot_sync(0xffffffffu, t[j] & (1 << i));
+            }
             if (RPU == 1) {
-                uint4 mine = make_uint4(b[0][0], b[0][1], b[0][2], b[0][3]);
+                // lane i stores plane i (each lane's address already points at its own plane): one predicated
+                // 16-byte store per plane instead of moving the ballots into the storing lanes' registers
+                uint32_t *dst = planes + (ru * BITS + (lane < BITS ? lane : 0)) * (int64_t)kw + seg * 4;
 #pragma unroll
-                for (int i = 1; i < BITS; ++i)
-                    if (lane == i) mine = make_uint4(b[i][0], b[i][1], b[i][2], b[i][3]);
-                if (lane < BITS)
-                    *reinterpret_cast<uint4 *>(planes + (ru * BITS + lane) * (int64_t)kw + seg * 4) = mine;
+                for (int i = 0; i < BITS; ++i)
+                    if (lane == i) *reinterpret_cast<uint4 *>(dst) = make_uint4(b[i][0], b[i][1], b[i][2], b[i][3]);
                 if (rowsum != nullptr) {
                     int s = t[0] + t[1] + t[2] + t[3];
 #pragma unroll
@@ -108,6 +169,112 @@ encode_pack_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx
         grp += first_grp_step;
         ru += first_row_step;
         if (grp >= groups_per_row) { grp -= groups_per_row; ++ru; }
+    }
+}
+
+
+// ---- per-lane packing kernel (the default whenever x is 16-byte aligned and ldx is a multiple of 4) ----------------
+// A warp-wide ballot costs about four ALU-pipe slots per lane on this GPU, so turning 32 lanes' decisions into a
+// word that way makes the encoder ALU-bound at 3 or more bits.  Here a lane owns one whole output word instead: 32
+// consecutive elements of a row.  A warp takes a unit of 32 words (4 KB of floats): every lane loads eight coalesced
+// float4 (all eight in flight before the first is used), quantizes each to four codes packed into the bytes of one
+// register, and hands that register through a small per-warp slice of shared memory to the lane that owns the word;
+// the owner reads its eight registers of codes back (two 16-byte reads) and moves bit i of each byte into a nibble
+// with one mask and one multiply:
+//   ((c & (0x01010101 << i)) * (0x10204080 >> i)) >> 28 = b3 b2 b1 b0   (partial products land on distinct bits)
+// which a funnel shift appends to plane i's word: 2 ALU operations + 1 multiply per 4 elements and plane.
+// (Copying the floats themselves to shared memory with cp.async was tried first: 16-byte cp.async retires about
+// one lane per clock per SM here, which capped the kernel at 4.2 TB/s.)
+// A unit is R rows x S words with R*S = 32 and S a power of two covering min(kw, 32) words, so that short rows (NHWC
+// activations with few channels) keep all lanes busy.  Plane words of one row segment are stored by consecutive
+// lanes (coalesced).  Padding words and the bits past k are written as 0.
+// Shared-memory slot of word `item` of the unit: 8 registers + 4 words of padding after every fourth item, which
+// makes both the 4-byte writes (lane -> item lane/8 + 4j, register lane%8) and the 16-byte reads conflict-free.
+__device__ __forceinline__ int enc_slot(int item) { return 8 * item + 4 * (item >> 2); }
+constexpr int kLaneSlotWords = 8 * 32 + 4 * 8;
+
+template <int BITS, int LOG2S>
+__global__ void __launch_bounds__(kEncThreads, 4)
+encode_pack_lanes_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, float lo, float hi,
+                         uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum, int kw, int segs, int64_t n_units) {
+    __shared__ __align__(16) uint32_t enc_codes[kEncThreads / 32][kLaneSlotWords];
+    const float half = (float)(1 << (BITS - 1));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t *sc = enc_codes[warp];
+    constexpr int S = 1 << LOG2S, R = 32 >> LOG2S;
+    const int64_t nwarps = (int64_t)gridDim.x * (kEncThreads / 32);
+    const int ca = lane >> 3, cc = lane & 7;                 // load role: word ca + 4j of the unit, 16-byte piece cc
+    // Piece j of this lane is word ca + 4j of the unit: row j / (S/4) of the unit, and within that row's segment
+    // element 128*(j % (S/4)) + 4*lane.  With S fixed at compile time every piece is a constant offset from one base.
+    constexpr int JPR = S / 4;                               // pieces per lane and row
+
+    for (int64_t u = (int64_t)blockIdx.x * (kEncThreads / 32) + warp; u < n_units; u += nwarps) {
+        const int64_t rg = u / segs;                         // warp-uniform
+        const int seg = (int)(u - rg * segs);
+        const float *xl = x + rg * R * ldx + (int64_t)seg * S * 32 + 4 * lane;
+        const int64_t rows_left = rows - rg * R;
+        const int k_left = k - seg * S * 32;                 // elements of the row from this segment on (may be <= 0)
+        float4 f[8];
+        if (rows_left >= R && k_left >= S * 32) {            // the whole unit is inside the tensor
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                f[j] = __ldcs(reinterpret_cast<const float4 *>(xl + (int64_t)(j / JPR) * ldx + 128 * (j % JPR)));
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int r = j / JPR, e = 128 * (j % JPR) + 4 * lane;
+                const float *src = xl + (int64_t)r * ldx + 128 * (j % JPR);
+                f[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (r < rows_left) {
+                    if (e + 4 <= k_left) {
+                        f[j] = __ldcs(reinterpret_cast<const float4 *>(src));
+                    } else if (e < k_left) {                 // the row ends inside this piece
+                        f[j].x = src[0];
+                        if (e + 1 < k_left) f[j].y = src[1];
+                        if (e + 2 < k_left) f[j].z = src[2];
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            // four codes in the bytes of one register; each operand is 2^23's pattern + t, the shifted ones lose
+            // that pattern's bits off the top, the unshifted one's is subtracted
+            const uint32_t t0 = enc_code_bits(f[j].x, inv2s, half, lo, hi), t1 = enc_code_bits(f[j].y, inv2s, half, lo, hi);
+            const uint32_t t2 = enc_code_bits(f[j].z, inv2s, half, lo, hi), t3 = enc_code_bits(f[j].w, inv2s, half, lo, hi);
+            sc[enc_slot(ca + 4 * j) + cc] = t0 + (t1 << 8) + (t2 << 16) + (t3 << 24) - kEncMagicBits;
+        }
+        __syncwarp();
+        const uint4 c_lo = *reinterpret_cast<const uint4 *>(sc + enc_slot(lane));
+        const uint4 c_hi = *reinterpret_cast<const uint4 *>(sc + enc_slot(lane) + 4);
+        __syncwarp();                                        // all reads done before the next unit's writes
+        const uint32_t c4[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
+        uint32_t word[BITS];
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) word[i] = 0u;
+#pragma unroll
+        for (int g = 7; g >= 0; --g) {                       // last group first: each append shifts the word left
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) {
+                const uint32_t prod = (c4[g] & (0x01010101u << i)) * (0x10204080u >> i);
+                word[i] = __funnelshift_l(prod, word[i], 4);
+            }
+        }
+        const int64_t row = rg * R + (lane >> LOG2S);
+        const int w = seg * S + (lane & (S - 1));
+        if (row < rows && w < kw) {
+            const int len = k - 32 * w;
+            const uint32_t mask = len >= 32 ? 0xffffffffu : (len <= 0 ? 0u : ((1u << len) - 1u));
+            uint32_t *dst = planes + (row * BITS) * (int64_t)kw + w;
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) dst[(int64_t)i * kw] = word[i] & mask;
+            if (rowsum != nullptr && len > 0) {
+                int sum = 0;
+#pragma unroll
+                for (int i = 0; i < BITS; ++i) sum += __popc(word[i] & mask) << i;
+                atomicAdd(rowsum + row, sum);
+            }
+        }
     }
 }
 
@@ -195,6 +362,37 @@ int grid_for(int64_t warps_needed) {
     return (int)blocks;
 }
 
+// Order-preserving map between floats and unsigned keys (negative floats reversed below the positive ones).
+inline uint32_t enc_key_of(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+inline float enc_float_of(uint32_t key) {
+    const uint32_t u = (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+// Smallest finite float x with pred(fmaf(x, inv2s, 2.0f)) true, for a predicate that is monotone in x
+// (false below, true above), searched by bisection over the float ordering.
+template <typename Pred>
+inline float enc_first_true(float inv2s, Pred pred) {
+    uint32_t lo = enc_key_of(-3.0e38f), hi = enc_key_of(3.0e38f);      // pred(lo) false, pred(hi) true
+    while (hi - lo > 1u) {
+        const uint32_t mid = lo + (hi - lo) / 2u;
+        if (pred(fmaf(enc_float_of(mid), inv2s, 2.0f))) hi = mid; else lo = mid;
+    }
+    return enc_float_of(hi);
+}
+// Two-bit thresholds (see EncThresholds): t reaches 1 where ceil(v) - 1 >= 1, i.e. v > 1, and 3 where floor(v) >= 3.
+inline EncThresholds enc_thresholds2(float inv2s) {
+    EncThresholds th;
+    th.t_lo = enc_first_true(inv2s, [](float v) { return v > 1.0f; });
+    th.t_hi = enc_first_true(inv2s, [](float v) { return v >= 3.0f; });
+    return th;
+}
+
 template <int BITS>
 void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale, bool relu, uint32_t *planes,
                    int32_t *rowsum, cudaStream_t st) {
@@ -203,6 +401,28 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
     float lo, hi;
     qnn_clamp_bounds(BITS, scale, relu, &lo, &hi);
     const int kw = (int)qnn_row_words_i(k);
+    if (qnn_aligned(x, 16) && ldx % 4 == 0) {
+        // per-lane packing kernel; the ballot kernels below remain for unaligned inputs
+        int log2s = 2;
+        while ((1 << log2s) < kw && log2s < 5) ++log2s;
+        const int segs_l = (kw + (1 << log2s) - 1) >> log2s;
+        const int rpu_l = 32 >> log2s;
+        const int64_t n_units = qnn_ceil_div(rows, rpu_l) * segs_l;
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        int64_t blocks = qnn_ceil_div(n_units, kEncThreads / 32);
+        if (blocks > 4 * (int64_t)sms) blocks = 4 * (int64_t)sms;
+#define QNN_ENC_LANES(L_) \
+    encode_pack_lanes_kernel<BITS, L_><<<(int)blocks, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, hi, planes, rowsum, kw, segs_l, n_units)
+        switch (log2s) {
+            case 2: QNN_ENC_LANES(2); break;
+            case 3: QNN_ENC_LANES(3); break;
+            case 4: QNN_ENC_LANES(4); break;
+            default: QNN_ENC_LANES(5); break;
+        }
+#undef QNN_ENC_LANES
+        return;
+    }
     const int segs = kw / 4;
     int groups;
     int64_t total;                                   // warp-level work items
@@ -218,15 +438,24 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
     const int64_t nwarps = (int64_t)grid * (kEncThreads / 32);
     const int64_t row_step = nwarps / groups;
     const int grp_step = (int)(nwarps % groups);
-#define QNN_ENC(RPU_, FULL_)                                                                                       \
-    encode_pack_kernel<BITS, UN, RPU_, FULL_><<<grid, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, hi, planes, \
-                                                                           rowsum, groups, segs, kw, row_step, grp_step)
+    EncThresholds th = {0.0f, 0.0f};
+#define QNN_ENC(RPU_, FULL_, MODE_)                                                                  \
+    encode_pack_kernel<BITS, UN, RPU_, FULL_, MODE_><<<grid, kEncThreads, 0, st>>>(                  \
+        x, rows, k, ldx, inv2s, lo, hi, th, planes, rowsum, groups, segs, kw, row_step, grp_step)
     if (rpu == 1) {
-        if (k % 128 == 0) QNN_ENC(1, true); else QNN_ENC(1, false);
+        if constexpr (BITS <= 2) {
+            if (rowsum == nullptr) {
+                if (BITS == 2) th = enc_thresholds2(inv2s);
+                if (relu) { if (k % 128 == 0) QNN_ENC(1, true, 2); else QNN_ENC(1, false, 2); }
+                else      { if (k % 128 == 0) QNN_ENC(1, true, 1); else QNN_ENC(1, false, 1); }
+                return;
+            }
+        }
+        if (k % 128 == 0) QNN_ENC(1, true, 0); else QNN_ENC(1, false, 0);
     } else if (rpu == 2) {
-        if (k == 64) QNN_ENC(2, true); else QNN_ENC(2, false);
+        if (k == 64) QNN_ENC(2, true, 0); else QNN_ENC(2, false, 0);
     } else {
-        if (k == 32) QNN_ENC(4, true); else QNN_ENC(4, false);
+        if (k == 32) QNN_ENC(4, true, 0); else QNN_ENC(4, false, 0);
     }
 #undef QNN_ENC
 }
@@ -265,7 +494,7 @@ extern "C" int qnn_encode_pack(const float *x, int64_t rows, int k, int64_t ldx,
     if (k > (1 << 30) || rows > ((int64_t)1 << 40)) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool relu = (flags & QNN_RELU) != 0;
-    if (rowsum && k > 64 && cudaMemsetAsync(rowsum, 0, (size_t)rows * sizeof(int32_t), st) != cudaSuccess)
+    if (rowsum && (k > 64 || (qnn_aligned(x, 16) && ldx % 4 == 0)) && cudaMemsetAsync(rowsum, 0, (size_t)rows * sizeof(int32_t), st) != cudaSuccess)
         return QNN_E_CUDA;
 #define CALL(B) launch_encode<B>(x, rows, k, ldx, scale, relu, planes, rowsum, st)
     QNN_DISPATCH_BITS(bits, CALL)

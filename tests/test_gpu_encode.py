@@ -46,6 +46,16 @@ def test_encode_pack_bit_exact(env, bits, rows, k, ldx):
         got = planes.cpu().numpy().view(np.uint32)
         assert np.array_equal(got, want)
         assert np.array_equal(rowsum.cpu().numpy(), t.sum(axis=1))
+        # without the row sums (the kernels take a different code path for 1 and 2 bits then), and from a
+        # source that is only 4-byte aligned (no 16-byte vector loads)
+        planes.fill_(-1)
+        qnn.encode_pack(x_d, bits, scale, qnn.RELU if relu else 0, planes=planes, k=k)
+        assert np.array_equal(planes.cpu().numpy().view(np.uint32), want)
+        shifted = torch.empty(x_d.numel() + 1, dtype=torch.float32, device=dev)[1:].view(rows, ldx)
+        shifted.copy_(x_d)
+        planes.fill_(-1)
+        qnn.encode_pack(shifted, bits, scale, qnn.RELU if relu else 0, planes=planes, k=k)
+        assert np.array_equal(planes.cpu().numpy().view(np.uint32), want)
 
 
 def test_encode_pack_all_special_values_every_width(env):
