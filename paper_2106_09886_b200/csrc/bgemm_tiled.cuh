@@ -52,6 +52,10 @@ struct Params {
     int H, W, C, R, S, stride, pad, Ho, Wo, cw, piece;   // piece = words per copy (4, 2 or 1)
     int dil, transposed;                                  // KIND 2 only: dilation (>= 1), transposed flag
     uint32_t cw_magic, s_magic;                           // x / d == (x * magic) >> 20 for the ranges used
+    // exact division of any numerator below 2^31 by Wo, Ho*Wo and tiles_m: n / d == (n * magic) >> shift in 64 bits
+    // (see set_fastdiv).  fast_pix = 0: rows or images beyond that range, use plain 64-bit division.
+    uint32_t wo_magic, howo_magic, tm_magic;
+    int wo_shift, howo_shift, tm_shift, fast_pix;
     // optional per-feature affine applied after the scale: y = fma(y, ch_gamma[n], ch_beta[n]) (ch_beta may be NULL)
     const float *ch_gamma, *ch_beta;
     // fused next-layer encoder (optional): planes of the fp32 result, rows = output rows, k = Ng
@@ -67,6 +71,20 @@ inline void set_k_split(Params &p) {
     p.ntail = p.kwords % 8;
     if (p.ntail >= 4) { ++p.nfull; p.ntail = 0; }
     p.nstages = (p.nfull + (p.ntail > 0 ? 1 : 0) + kStageChunks - 1) / kStageChunks;
+}
+
+// Division by an invariant divisor d (1 <= d < 2^31) of numerators n < 2^31: with k = 31 + ceil(log2 d) and
+// magic = ceil(2^k / d) (< 2^32), floor(n * magic / 2^k) = floor(n / d) exactly (the error n * (magic*d - 2^k) / (d * 2^k)
+// stays below 1/d).  The tile bookkeeping divides row indices by the output width and by the pixels per image for
+// every tile; the generic 64-bit division costs over a hundred instructions each.
+inline void set_fastdiv(uint32_t d, uint32_t &magic, int &shift) {
+    int lg = 0;
+    while ((1ull << lg) < d) ++lg;
+    shift = 31 + lg;
+    magic = (uint32_t)(((1ull << shift) + d - 1) / d);
+}
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, uint32_t magic, int shift) {
+    return (uint32_t)(((uint64_t)n * magic) >> shift);
 }
 
 __device__ __forceinline__ uint32_t lop3_xor3(uint32_t a, uint32_t b, uint32_t c) {
@@ -185,8 +203,11 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
     };
     auto prep_tile = [&](int tile) {
         TileSrc t;
-        const int64_t m0 = (int64_t)(tile % p.tiles_m) * kBM;
-        const int n0 = (tile / p.tiles_m) * kBN;
+        // (the fully-connected kernels keep the plain division: one per tile, and the other form cost them 2%
+        // through code-generation side effects)
+        const int tile_n = CONV ? (int)fastdiv((uint32_t)tile, p.tm_magic, p.tm_shift) : tile / p.tiles_m;
+        const int64_t m0 = (int64_t)(tile - tile_n * p.tiles_m) * kBM;
+        const int n0 = tile_n * kBN;
         const int64_t am = m0 + srow;
         t.a_ok = a_unit && am < p.Mg;
         t.w_ok = (n0 + wrow) < p.Ng;
@@ -194,9 +215,19 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
         t.pixbase = 0; t.h0 = 0; t.w0 = 0;
         if (CONV) {
             const int64_t mm = t.a_ok ? am : 0;
-            const int wo = (int)(mm % p.Wo);
-            const int ho = (int)((mm / p.Wo) % p.Ho);
-            const int64_t n = mm / ((int64_t)p.Wo * p.Ho);
+            int wo, ho;
+            int64_t n;
+            if (p.fast_pix) {
+                const uint32_t m32 = (uint32_t)mm;
+                const uint32_t q = fastdiv(m32, p.wo_magic, p.wo_shift), img = fastdiv(m32, p.howo_magic, p.howo_shift);
+                wo = (int)(m32 - q * (uint32_t)p.Wo);
+                ho = (int)(q - img * (uint32_t)p.Ho);
+                n = img;
+            } else {
+                wo = (int)(mm % p.Wo);
+                ho = (int)((mm / p.Wo) % p.Ho);
+                n = mm / ((int64_t)p.Wo * p.Ho);
+            }
             t.h0 = (GENERAL && p.transposed) ? ho + p.pad : ho * p.stride - p.pad;
             t.w0 = (GENERAL && p.transposed) ? wo + p.pad : wo * p.stride - p.pad;
             t.pixbase = n * p.H * p.W;
@@ -458,8 +489,9 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
 
         // ---- epilogue: acc holds S = sum_ij 2^(i+j) X_ij.  out = n_valid*A*B - 2*S (Eq. 8), times alpha (Eq. 9).
         constexpr int AMAX = (1 << AB) - 1, PROD = AMAX * ((1 << WB) - 1);
-        const int64_t m0 = (int64_t)(tile % p.tiles_m) * kBM;
-        const int n0 = (tile / p.tiles_m) * kBN;
+        const int tile_n = CONV ? (int)fastdiv((uint32_t)tile, p.tm_magic, p.tm_shift) : tile / p.tiles_m;
+        const int64_t m0 = (int64_t)(tile - tile_n * p.tiles_m) * kBM;
+        const int n0 = tile_n * kBN;
 #pragma unroll
         for (int r = 0; r < TM; ++r) {
             const int64_t m = m0 + ty + 16 * r;
@@ -470,8 +502,16 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             if (CONV && row_ok) {
                 // Taps outside the image were staged as zero words: each contributed popc(w_j) to X_ij, i.e.
                 // AMAX * tapsum[n][tap] to S, and must not be counted in the length.
-                const int wo = (int)(m % p.Wo);
-                const int ho = (int)((m / p.Wo) % p.Ho);
+                int wo, ho;
+                if (p.fast_pix) {
+                    const uint32_t m32 = (uint32_t)m;
+                    const uint32_t q = fastdiv(m32, p.wo_magic, p.wo_shift), img = fastdiv(m32, p.howo_magic, p.howo_shift);
+                    wo = (int)(m32 - q * (uint32_t)p.Wo);
+                    ho = (int)(q - img * (uint32_t)p.Ho);
+                } else {
+                    wo = (int)(m % p.Wo);
+                    ho = (int)((m / p.Wo) % p.Ho);
+                }
                 const int hh = (GENERAL && p.transposed) ? ho + p.pad : ho * p.stride - p.pad;
                 const int ww = (GENERAL && p.transposed) ? wo + p.pad : wo * p.stride - p.pad;
                 int valid_taps = p.R * p.S;
@@ -515,28 +555,29 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 // two output rows (lanes 0-15: row ty even, lanes 16-31: row ty odd) x 16 consecutive features
                 // per c, so one ballot per (plane, c) yields half a word for each of the two rows; c = 0,1 form
                 // word n0/32 and c = 2,3 word n0/32 + 1.  Every lane takes part in every ballot.
-                int t[4];
+                uint32_t t[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int n = n0 + tx + 16 * c;
-                    const int code = qnn_code_t(fv[c], p.next_inv2s, p.next_half, p.next_lo, p.next_hi);
-                    t[c] = (row_ok && n < p.Ng) ? code : 0;                 // padding bits are 0
+                    const uint32_t code = qnn_code_bits(fv[c], p.next_inv2s, p.next_half, p.next_lo, p.next_hi);
+                    t[c] = (row_ok && n < p.Ng) ? code : 0u;                // padding bits are 0
                 }
                 const int lane = tid & 31;
-                const bool upper = lane >= 16;
+                const uint32_t halfsel = lane >= 16 ? 0x7632u : 0x5410u;    // this lane's row: upper / lower ballot halves
+                const bool storer = (lane & 15) == 0 && row_ok;
                 const int word0 = n0 >> 5;
-                for (int i = 0; i < p.next_bits; ++i) {
-                    const uint32_t b0 = __ballot_sync(0xffffffffu, (t[0] >> i) & 1);
-                    const uint32_t b1 = __ballot_sync(0xffffffffu, (t[1] >> i) & 1);
-                    const uint32_t b2 = __ballot_sync(0xffffffffu, (t[2] >> i) & 1);
-                    const uint32_t b3 = __ballot_sync(0xffffffffu, (t[3] >> i) & 1);
-                    if ((lane & 15) == 0 && row_ok) {
-                        const uint32_t w0 = upper ? ((b0 >> 16) | (b1 & 0xffff0000u)) : ((b0 & 0xffffu) | (b1 << 16));
-                        const uint32_t w1 = upper ? ((b2 >> 16) | (b3 & 0xffff0000u)) : ((b2 & 0xffffu) | (b3 << 16));
-                        uint32_t *dst = p.next_planes + (m * p.next_bits + i) * (int64_t)p.next_kw + word0;
-                        *reinterpret_cast<uint2 *>(dst) = make_uint2(w0, w1);
+                uint32_t *dst = p.next_planes + (m * p.next_bits) * (int64_t)p.next_kw + word0;
+                const bool last_tile_n = n0 + kBN >= p.Ng;
+                for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
+                    const uint32_t bit = 1u << i;
+                    const uint32_t b0 = __ballot_sync(0xffffffffu, t[0] & bit);
+                    const uint32_t b1 = __ballot_sync(0xffffffffu, t[1] & bit);
+                    const uint32_t b2 = __ballot_sync(0xffffffffu, t[2] & bit);
+                    const uint32_t b3 = __ballot_sync(0xffffffffu, t[3] & bit);
+                    if (storer) {
+                        *reinterpret_cast<uint2 *>(dst) = make_uint2(__byte_perm(b0, b1, halfsel), __byte_perm(b2, b3, halfsel));
                         // the last feature tile also clears the padding words of the row
-                        if (n0 + kBN >= p.Ng)
+                        if (last_tile_n)
                             for (int wz = word0 + 2; wz < p.next_kw; wz += 2)
                                 *reinterpret_cast<uint2 *>(dst + (wz - word0)) = make_uint2(0u, 0u);
                     }
@@ -638,6 +679,13 @@ inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     if (tiles_m * tiles_n > 0x7fffffff) return QNN_E_RANGE;
     q.tiles_m = (int)tiles_m;
     q.ntiles = (int)(tiles_m * tiles_n);
+    set_fastdiv((uint32_t)q.tiles_m, q.tm_magic, q.tm_shift);
+    q.fast_pix = 0;
+    if (CONV != 0 && q.Mg + kBM < (1ll << 31) && (int64_t)q.Ho * q.Wo < (1ll << 31) && q.Wo > 0 && q.Ho > 0) {
+        set_fastdiv((uint32_t)q.Wo, q.wo_magic, q.wo_shift);
+        set_fastdiv((uint32_t)((int64_t)q.Ho * q.Wo), q.howo_magic, q.howo_shift);
+        q.fast_pix = 1;
+    }
     if (CONV == 3) {               // one 9-word group per channel word, no tail
         q.nfull = q.cw;
         q.ntail = 0;

@@ -14,24 +14,14 @@ namespace {
 
 constexpr int kEncThreads = 256;
 
-// The code t of qnn_code_t without a float->int conversion.  Conversions run on the XU pipe, whose rate made
-// them the bottleneck of this kernel (ncu: XU saturated, DRAM at half its rate).  Two rewrites, both exact:
-//  * For x <= 0 the quantizer takes ceil(v) - 1, which equals floor(v) unless v is an integer; for a positive
-//    float v that is floor(pred(v)) with pred(v) the next float below v (bit pattern - 1): an integer v >= 1 loses
-//    less than 1, a non-integer v cannot fall below floor(v), which is itself a float.  The pre-clamp keeps
-//    v >= 2^(b-1) * (2^-10 - 2^-23) > 0, so the pattern never wraps.
-//  * floor(y) for 0 <= y < 2^23 is read from the mantissa of y + 2^23 rounded DOWN (one add on the FMA pipe):
-//    the sum's unit in the last place is 1, so rounding down yields exactly 2^23 + floor(y).
-// enc_code_bits returns that sum's bit pattern, 0x4B000000 + t.
-constexpr uint32_t kEncMagicBits = 0x4B000000u;             // bit pattern of 2^23
+// The encoders here take the code from qnn_code_bits (no float->int conversion: those run on the XU pipe, whose
+// rate made them the bottleneck of this kernel -- ncu showed XU saturated and DRAM at half its rate).
+constexpr uint32_t kEncMagicBits = 0x4B000000u;             // bit pattern of 2^23, the offset in qnn_code_bits
 __device__ __forceinline__ uint32_t enc_code_bits(float x, float inv2s, float half, float lo, float hi) {
-    x = fminf(fmaxf(x, lo), hi);          // NaN -> lo
-    const float v = __fmaf_rn(x, inv2s, half);
-    const int vb = __float_as_int(v) - ((x > 0.0f) ? 0 : 1);
-    return (uint32_t)__float_as_int(__fadd_rd(__int_as_float(vb), 8388608.0f));
+    return qnn_code_bits(x, inv2s, half, lo, hi);
 }
 __device__ __forceinline__ int enc_code_t(float x, float inv2s, float half, float lo, float hi) {
-    return (int)(enc_code_bits(x, inv2s, half, lo, hi) & 0xffu);
+    return (int)(qnn_code_bits(x, inv2s, half, lo, hi) & 0xffu);
 }
 
 // One- and two-bit codes are decided by comparisons alone.  The quantizer is a non-decreasing step function of x,

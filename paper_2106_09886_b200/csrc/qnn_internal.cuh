@@ -32,6 +32,17 @@ __device__ __forceinline__ int qnn_code_t(float x, float inv2s, float half, floa
     return pos ? f : ~f;
 }
 
+// The same code without a float->int conversion (those run on the XU pipe, which the contraction's popcounts
+// already saturate): returns the bit pattern 0x4B000000 + t, whose low 8 bits are t.  For x <= 0, ceil(v) - 1 is
+// floor of the next float below v (bit pattern - 1; v > 0 after the pre-clamp): an integer v loses less than 1, a
+// non-integer v cannot fall below floor(v).  floor(y) for 0 <= y < 2^23 is the mantissa of y + 2^23 rounded down.
+__device__ __forceinline__ uint32_t qnn_code_bits(float x, float inv2s, float half, float lo, float hi) {
+    x = fminf(fmaxf(x, lo), hi);          // NaN -> lo
+    const float v = __fmaf_rn(x, inv2s, half);
+    const int vb = __float_as_int(v) - ((x > 0.0f) ? 0 : 1);
+    return (uint32_t)__float_as_int(__fadd_rd(__int_as_float(vb), 8388608.0f));
+}
+
 // Pre-clamp bounds that make the integer clamp of the code unnecessary.  hi = 2^bits * scale * (1 - 2^-10)
 // lies between the range end r = (2^bits - 1) * scale and the point where v would reach 2^bits, with a margin
 // (2^-11 relative) far above the rounding of inv2s and of the multiply-add: every x in [r, hi] gives
