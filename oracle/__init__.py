@@ -15,6 +15,7 @@ What each function follows in the paper:
 * ``scale``        -- the fixed scaling factor of Eq. 9 / Alg. 1 forward pass.
 * ``mbit_encoder_forward`` / ``mbit_encoder_backward`` -- trigonometric encoder of Eq. 10 and its derivative, Eq. 12.
 * ``affine``       -- per-feature affine that replaces the scale when batch normalisation follows (Section 3.2).
+* ``conv_backward_data`` / ``conv_backward_weights`` -- Algorithm 1's backward products with forward() a convolution.
 * ``eq16_speedup`` -- the paper's analytic speed-up model S_MK (Eq. 16, Section 4.6), plain arithmetic.
 """
 from __future__ import annotations
@@ -59,6 +60,8 @@ def _load():
         lib.oracle_fc.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, p]
         lib.oracle_fc_sampled.argtypes = [p, p, c.c_size_t, c.c_size_t, p, p, p]
         lib.oracle_conv_out_dim.argtypes = [c.c_int] * 4
+        lib.oracle_conv_backward_data.argtypes = [p, p] + [c.c_int] * 11 + [c.c_float, p]
+        lib.oracle_conv_backward_weights.argtypes = [p, p] + [c.c_int] * 11 + [c.c_float, p]
         lib.oracle_conv2d.argtypes = [p, p] + [c.c_int] * 9 + [p]
         lib.oracle_conv2d_sampled.argtypes = [p, p] + [c.c_int] * 9 + [c.c_size_t, p, p, p]
         lib.oracle_scale.argtypes = [p, c.c_size_t, c.c_float, p]
@@ -288,6 +291,36 @@ def fc_backward_weights_sampled(g, qa, ab: int, wb: int, alpha: float, rows, col
                                                       rows.size, _ptr(rows), _ptr(cols), _ptr(out)),
            "fc_backward_weights_sampled")
     return out
+
+
+def conv_backward_data(g: np.ndarray, qw: np.ndarray, hw, stride: int, pad: int, ab: int, wb: int, alpha: float) -> np.ndarray:
+    """Algorithm 1, backward, convolution: g [N, Ho, Wo, Cout] = dC/d(out), qw [Cout, R, S, C], hw = (H, W) of the
+    layer's input -> float64 [ab, N, H, W, C], entry m-1 = g_{a^m}."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    qw = np.ascontiguousarray(qw, dtype=np.int16)
+    N, Ho, Wo, Cout = g.shape
+    Cout2, R, S, C = qw.shape
+    H, W = hw
+    assert Cout == Cout2 and Ho == conv_out_dim(H, R, stride, pad) and Wo == conv_out_dim(W, S, stride, pad)
+    ga = np.empty((ab, N, H, W, C), dtype=np.float64)
+    _check(_load().oracle_conv_backward_data(_ptr(g), _ptr(qw), N, H, W, C, Cout, R, S, stride, pad, ab, wb,
+                                         float(np.float32(alpha)), _ptr(ga)), "conv_backward_data")
+    return ga
+
+
+def conv_backward_weights(g: np.ndarray, qa: np.ndarray, rs, stride: int, pad: int, ab: int, wb: int, alpha: float) -> np.ndarray:
+    """Algorithm 1, backward, convolution: g [N, Ho, Wo, Cout], qa [N, H, W, C], rs = (R, S) of the kernel
+    -> float64 [wb, Cout, R, S, C], entry j-1 = g_{W^j}."""
+    g = np.ascontiguousarray(g, dtype=np.float32)
+    qa = np.ascontiguousarray(qa, dtype=np.int16)
+    N, Ho, Wo, Cout = g.shape
+    N2, H, W, C = qa.shape
+    R, S = rs
+    assert N == N2 and Ho == conv_out_dim(H, R, stride, pad) and Wo == conv_out_dim(W, S, stride, pad)
+    gw = np.empty((wb, Cout, R, S, C), dtype=np.float64)
+    _check(_load().oracle_conv_backward_weights(_ptr(g), _ptr(qa), N, H, W, C, Cout, R, S, stride, pad, ab, wb,
+                                            float(np.float32(alpha)), _ptr(gw)), "conv_backward_weights")
+    return gw
 
 
 def eq16_speedup(n: int, m_bits: int, k_bits: int, gamma: float = 1.91, beta: float | None = None, reg_len: int = 64):

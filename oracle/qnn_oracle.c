@@ -467,3 +467,78 @@ int oracle_fc_backward_weights_sampled(const float *g, const int16_t *qa, size_t
     }
     return ORACLE_OK;
 }
+
+/* ---- Backward products of a convolution layer (Algorithm 1, backward propagation, with forward() a convolution).
+ * Forward: out[n][ho][wo][co] = alpha * sum_m sum_j 2^(m+j-2) * sum_{r,s,c} a^m[n][ho*st-pad+r][wo*st-pad+s][c] * W^j[co][r][s][c],
+ * taps outside the image contributing nothing.  Each gradient is the derivative of that expression, written as the
+ * scatter / correlation it defines; g = dC/d(out), fp32 [N][Ho][Wo][Cout]. */
+
+/* ga[(m-1)*N*H*W*C + ((n*H + h)*W + w)*C + c] = g_{a^m}[n][h][w][c]: every (output, tap) that read the element
+ * sends its share back to it. */
+int oracle_conv_backward_data(const float *g, const int16_t *qw, int N, int H, int W, int C, int Cout, int R, int S,
+                              int stride, int pad, int ab, int wb, float alpha, double *ga) {
+    if (!g || !qw || !ga || ab < 1 || ab > 8 || wb < 1 || wb > 8 || stride < 1 || pad < 0) return ORACLE_E_ARG;
+    if (!codes_ok(qw, (size_t)Cout * R * S * C, wb)) return ORACLE_E_ARG;
+    const int Ho = oracle_conv_out_dim(H, R, stride, pad), Wo = oracle_conv_out_dim(W, S, stride, pad);
+    if (Ho < 1 || Wo < 1) return ORACLE_E_ARG;
+    const size_t img = (size_t)H * W * C, all = (size_t)N * img;
+    for (size_t i = 0; i < (size_t)ab * all; ++i) ga[i] = 0.0;
+    for (int m = 1; m <= ab; ++m) {
+#pragma omp parallel for schedule(static)
+        for (int n = 0; n < N; ++n)
+            for (int ho = 0; ho < Ho; ++ho)
+                for (int wo = 0; wo < Wo; ++wo)
+                    for (int r = 0; r < R; ++r)
+                        for (int s = 0; s < S; ++s) {
+                            const int hi = ho * stride - pad + r, wi = wo * stride - pad + s;
+                            if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;
+                            double *dst = ga + (size_t)(m - 1) * all + (size_t)n * img + ((size_t)hi * W + wi) * C;
+                            const float *gp = g + (((size_t)n * Ho + ho) * Wo + wo) * Cout;
+                            for (int c = 0; c < C; ++c) {
+                                double sum = 0.0;
+                                for (int j = 1; j <= wb; ++j) {
+                                    double part = 0.0;
+                                    for (int co = 0; co < Cout; ++co)
+                                        part += ((double)alpha * (double)gp[co]) *
+                                                plane_of(qw[(((size_t)co * R + r) * S + s) * C + c], wb, j);
+                                    sum += ldexp(part, m + j - 2);
+                                }
+                                dst[c] += sum;
+                            }
+                        }
+    }
+    return ORACLE_OK;
+}
+
+/* gw[(j-1)*Cout*R*S*C + ((co*R + r)*S + s)*C + c] = g_{W^j}[co][r][s][c]: correlation of g with the activation planes. */
+int oracle_conv_backward_weights(const float *g, const int16_t *qa, int N, int H, int W, int C, int Cout, int R, int S,
+                                 int stride, int pad, int ab, int wb, float alpha, double *gw) {
+    if (!g || !qa || !gw || ab < 1 || ab > 8 || wb < 1 || wb > 8 || stride < 1 || pad < 0) return ORACLE_E_ARG;
+    if (!codes_ok(qa, (size_t)N * H * W * C, ab)) return ORACLE_E_ARG;
+    const int Ho = oracle_conv_out_dim(H, R, stride, pad), Wo = oracle_conv_out_dim(W, S, stride, pad);
+    if (Ho < 1 || Wo < 1) return ORACLE_E_ARG;
+    const size_t wsz = (size_t)Cout * R * S * C;
+    for (int j = 1; j <= wb; ++j) {
+#pragma omp parallel for schedule(static)
+        for (int co = 0; co < Cout; ++co)
+            for (int r = 0; r < R; ++r)
+                for (int s = 0; s < S; ++s)
+                    for (int c = 0; c < C; ++c) {
+                        double sum = 0.0;
+                        for (int m = 1; m <= ab; ++m) {
+                            double part = 0.0;
+                            for (int n = 0; n < N; ++n)
+                                for (int ho = 0; ho < Ho; ++ho)
+                                    for (int wo = 0; wo < Wo; ++wo) {
+                                        const int hi = ho * stride - pad + r, wi = wo * stride - pad + s;
+                                        if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;
+                                        part += ((double)alpha * (double)g[(((size_t)n * Ho + ho) * Wo + wo) * Cout + co]) *
+                                                plane_of(qa[(((size_t)n * H + hi) * W + wi) * C + c], ab, m);
+                                    }
+                            sum += ldexp(part, m + j - 2);
+                        }
+                        gw[(size_t)(j - 1) * wsz + (((size_t)co * R + r) * S + s) * C + c] = sum;
+                    }
+    }
+    return ORACLE_OK;
+}

@@ -40,6 +40,9 @@ MUTATIONS = {
     "mbit_derivative_not_windowed": ("if (xn >= -1.0 && xn <= 1.0) {", "if (1) {"),
     "mbit_derivative_sine": ("const double d = k * pi * cos(k * pi * xn);", "const double d = k * pi * sin(k * pi * xn);"),
     "mbit_derivative_forgets_r": ("gx[e] = g / (double)r;", "gx[e] = g;"),
+    "conv_backward_data_taps_transposed": ("plane_of(qw[(((size_t)co * R + r) * S + s) * C + c], wb, j);", "plane_of(qw[(((size_t)co * S + s) * R + r) * C + c], wb, j);"),
+    "conv_backward_weights_drops_alpha": ("part += ((double)alpha * (double)g[(((size_t)n * Ho + ho) * Wo + wo) * Cout + co]) *", "part += ((double)g[(((size_t)n * Ho + ho) * Wo + wo) * Cout + co]) *"),
+    "conv_backward_data_ignores_stride": ("const int hi = ho * stride - pad + r, wi = wo * stride - pad + s;\n                            if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;\n                            double *dst", "const int hi = ho - pad + r, wi = wo - pad + s;\n                            if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;\n                            double *dst"),
     "scale_in_double": ("out[i] = (float)acc[i] * alpha;", "out[i] = (float)((double)acc[i] * (double)alpha * (1.0 + 1e-6));"),
 }
 

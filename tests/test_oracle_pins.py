@@ -508,6 +508,80 @@ def test_backward_products_special_cases(ab, wb):
     assert np.array_equal(oracle.fc_backward_weights_sampled(g, qa, ab, wb, alpha, rows, cols), gw[:, rows, cols])
 
 
+
+# ---- Algorithm 1 backward with forward() a convolution --------------------------------------------------------------
+
+def _conv_backward_case(seed, N, H, W, C, Cout, R, S, stride, pad, ab, wb):
+    rng = np.random.default_rng(seed)
+    qa = (2 * rng.integers(0, 2 ** ab, size=(N, H, W, C)) - (2 ** ab - 1)).astype(np.int16)
+    qw = (2 * rng.integers(0, 2 ** wb, size=(Cout, R, S, C)) - (2 ** wb - 1)).astype(np.int16)
+    Ho, Wo = oracle.conv_out_dim(H, R, stride, pad), oracle.conv_out_dim(W, S, stride, pad)
+    g = rng.standard_normal((N, Ho, Wo, Cout)).astype(np.float32)
+    alpha = float(np.float32(0.21 / ((2 ** ab - 1) * (2 ** wb - 1))))
+    return qa, qw, g, alpha
+
+
+@pytest.mark.parametrize("ab,wb,stride,pad", [(1, 1, 1, 1), (2, 3, 2, 1), (4, 2, 1, 0), (3, 3, 2, 2)])
+def test_conv_backward_is_the_exact_change_of_the_forward_under_a_plane_flip(ab, wb, stride, pad):
+    """The pinned forward convolution is linear in every plane entry: flipping one entry of a^m or W^j changes
+    C = <g, alpha * conv(qa, qw)> by exactly twice the gradient there (border elements, read by fewer taps, included)."""
+    N, H, W, C, Cout, R, S = 2, 6, 5, 3, 4, 3, 3
+    qa, qw, g, alpha = _conv_backward_case(10 * ab + wb, N, H, W, C, Cout, R, S, stride, pad, ab, wb)
+    ga = oracle.conv_backward_data(g, qw, (H, W), stride, pad, ab, wb, alpha)
+    gw = oracle.conv_backward_weights(g, qa, (R, S), stride, pad, ab, wb, alpha)
+    assert ga.shape == (ab, N, H, W, C) and gw.shape == (wb, Cout, R, S, C)
+
+    def cost(qa_, qw_):
+        return float(np.sum(g.astype(np.float64) * alpha * oracle.conv2d(qa_, qw_, stride, pad).astype(np.float64)))
+
+    pa, pw = _planes_pm1(qa.reshape(-1, C), ab).reshape((ab,) + qa.shape), _planes_pm1(qw.reshape(-1, C), wb).reshape((wb,) + qw.shape)
+    base = cost(qa, qw)
+    rng = np.random.default_rng(3)
+    corners = [(0, 0, 0, 0), (N - 1, H - 1, W - 1, C - 1), (0, H - 1, 0, 1)]
+    for it in range(30):
+        idx = corners[it] if it < len(corners) else tuple(int(rng.integers(0, d)) for d in qa.shape)
+        m = int(rng.integers(0, ab))
+        q2 = qa.copy()
+        q2[idx] -= np.int16(pa[(m,) + idx] * 2 * 2 ** m)
+        assert cost(q2, qw) - base == pytest.approx(-2 * pa[(m,) + idx] * ga[(m,) + idx], rel=1e-9, abs=1e-12)
+        idw = tuple(int(rng.integers(0, d)) for d in qw.shape)
+        j = int(rng.integers(0, wb))
+        w2 = qw.copy()
+        w2[idw] -= np.int16(pw[(j,) + idw] * 2 * 2 ** j)
+        assert cost(qa, w2) - base == pytest.approx(-2 * pw[(j,) + idw] * gw[(j,) + idw], rel=1e-9, abs=1e-12)
+
+
+@pytest.mark.parametrize("N,H,W,C,Cout,R,S,stride,pad,ab,wb", [(2, 7, 6, 5, 3, 3, 3, 1, 1, 2, 2), (1, 9, 9, 4, 6, 3, 2, 2, 1, 3, 1),
+                                                             (2, 5, 5, 8, 2, 1, 1, 2, 0, 1, 4), (1, 8, 7, 3, 5, 5, 5, 1, 2, 2, 2)])
+def test_conv_backward_matches_library_autograd(N, H, W, C, Cout, R, S, stride, pad, ab, wb):
+    """torch's conv2d differentiated in float64: the per-plane gradients are 2^(m-1) (2^(j-1)) times the gradient with
+    respect to the codes."""
+    import torch
+    qa, qw, g, alpha = _conv_backward_case(N + H + C, N, H, W, C, Cout, R, S, stride, pad, ab, wb)
+    a = torch.tensor(qa.transpose(0, 3, 1, 2).astype(np.float64), requires_grad=True)
+    w = torch.tensor(qw.transpose(0, 3, 1, 2).astype(np.float64), requires_grad=True)
+    out = alpha * torch.nn.functional.conv2d(a, w, stride=stride, padding=pad)
+    out.backward(torch.tensor(g.transpose(0, 3, 1, 2).astype(np.float64)))
+    da = a.grad.numpy().transpose(0, 2, 3, 1)
+    dw = w.grad.numpy().transpose(0, 2, 3, 1)
+    ga = oracle.conv_backward_data(g, qw, (H, W), stride, pad, ab, wb, alpha)
+    gw = oracle.conv_backward_weights(g, qa, (R, S), stride, pad, ab, wb, alpha)
+    for m in range(ab):
+        assert np.allclose(ga[m], 2.0 ** m * da, rtol=1e-12, atol=1e-14)
+    for j in range(wb):
+        assert np.allclose(gw[j], 2.0 ** j * dw, rtol=1e-12, atol=1e-14)
+
+
+def test_conv_backward_of_a_1x1_convolution_is_the_fc_backward():
+    ab, wb = 3, 2
+    qa, qw, g, alpha = _conv_backward_case(1, 2, 4, 3, 6, 5, 1, 1, 1, 0, ab, wb)
+    ga = oracle.conv_backward_data(g, qw, (4, 3), 1, 0, ab, wb, alpha)
+    gw = oracle.conv_backward_weights(g, qa, (1, 1), 1, 0, ab, wb, alpha)
+    g2, qa2, qw2 = g.reshape(-1, 5), qa.reshape(-1, 6), qw.reshape(5, 6)
+    assert np.allclose(ga.reshape(ab, -1, 6), oracle.fc_backward_data(g2, qw2, ab, wb, alpha), rtol=1e-13, atol=0)
+    assert np.allclose(gw.reshape(wb, 5, 6), oracle.fc_backward_weights(g2, qa2, ab, wb, alpha), rtol=1e-13, atol=0)
+
+
 # ---- Eq. 16 (Section 4.6): the analytic speed-up model -------------------------------------------------------------
 
 def test_eq16_reproduces_the_printed_two_bit_speedup(golden_dir):
