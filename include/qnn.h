@@ -229,6 +229,38 @@ int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_planes, size_t 
                                float alpha, float *gw, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Backward products of a convolution layer (Algorithm 1, backward propagation, with forward() the convolution of
+ * qnn_bconv2d: out[n][ho][wo][co] = alpha * sum_{r,s,c} qa[n][ho*stride - pad + r][wo*stride - pad + s][c] * qw[co][r][s][c],
+ * taps outside the image contributing nothing).  Given g = dC/d(out), fp32 [N][Ho][Wo][Cout]:
+ *   qnn_bconv2d_backward_data     G[n][h][w][c] = alpha * sum over (co, r, s) and the output pixels that read input
+ *                                 pixel (h, w) through tap (r, s) of g[n][ho][wo][co] * qw[co][r][s][c]; Algorithm 1's
+ *                                 per-plane gradient is g_{a^p} = 2^(p-1) * G.  x (optional, fp32 [N][H][W][C], with ab
+ *                                 and r) applies the encoder derivative of Eq. 12 as in qnn_bgemm_backward_data.
+ *   qnn_bconv2d_backward_weights  GW[co][r][s][c] = alpha * sum over the output pixels of g[n][ho][wo][co] *
+ *                                 qa[n][ho*stride - pad + r][wo*stride - pad + s][c]; g_{W^j} = 2^(j-1) * GW.
+ * Both run the TF32 tensor-core contraction of the fully-connected case on an explicit patch matrix held in the
+ * workspace: for the weights the im2col of the activation codes ([R*S*C][N*Ho*Wo] fp32), for the data the patch
+ * gradients ([N*Ho*Wo][R*S*C] fp32), which a gather then sums onto the pixels in a fixed tap order.  Error bound as
+ * for the fully-connected products with contraction lengths Cout (data; plus one fp32 addition per tap) and N*Ho*Wo
+ * (weights); integer-valued g with small sums is contracted exactly.
+ *   w_packed  blob of qnn_pack_weights(n_out = Cout, taps = R*S, c_in = C, bits = wb); a_planes [N*H*W][ab][qnn_row_words(C)]
+ *   g         device fp32, 16-byte aligned for backward_data (4-byte for backward_weights)
+ *   out / gw  device fp32 [N][H][W][C] / [Cout][R][S][C]
+ *   workspace device scratch owned by the caller, 256-byte aligned, at least qnn_bconv2d_backward_*_workspace(...)
+ *             bytes (0 from the query = geometry out of range: N*Ho*Wo, R*S*C and Cout at most 65535*32,
+ *             R*S*ceil(C/32) at most 65535).
+ * Errors as for qnn_bgemm_backward_*; waits are bounded and reported by qnn_tensor_path_status.
+ */
+size_t qnn_bconv2d_backward_data_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad);
+int qnn_bconv2d_backward_data(const float *g, const void *w_packed, int wb, int N, int H, int W, int C, int Cout, int R,
+                              int S, int stride, int pad, float alpha, const float *x, int ab, float r, float *out,
+                              void *workspace, size_t workspace_bytes, void *stream);
+size_t qnn_bconv2d_backward_weights_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad);
+int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_planes, int ab, int N, int H, int W, int C, int Cout,
+                                 int R, int S, int stride, int pad, float alpha, float *gw, void *workspace,
+                                 size_t workspace_bytes, void *stream);
+
+/*
  * Planes [rows][bits][qnn_row_words(k)] -> the odd codes q = sum_i 2^(i-1) * plane_i (Eq. 8) as fp32:
  * out[row*ld + col] (transpose = 0, ld >= k) or out[col*ld + row] (transpose != 0, ld >= rows).
  */

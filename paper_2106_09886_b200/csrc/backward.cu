@@ -1,4 +1,4 @@
-// Backward products of a fully-connected layer (Algorithm 1, backward propagation).
+// Backward products of a fully-connected and of a convolution layer (Algorithm 1, backward propagation).
 //
 // With g_hat = alpha * g the two products are dense real-by-integer contractions,
 //   G [r][k] = sum_n g_hat[r][n] * qw[n][k]      (g_{a^m} = 2^(m-1) * G,  since sum_j 2^(j-1) W^j = qw)
@@ -7,6 +7,10 @@
 // (tcgen05.mma, kind::tf32, accumulator in tensor memory), fed by TMA through a ring of mbarrier-guarded stages.
 // The integer codes (|q| <= 255) are exact in TF32; the gradient keeps 11 significant bits per element.
 // Bound: tensor pipe (2*M*N*K flop per call).
+// A convolution goes through the same GEMM on an explicit patch matrix: the weight gradient contracts g with the
+// im2col of the activation codes (unpacked straight from the planes into K-major order), the data gradient
+// multiplies g by the weight codes and gathers the patch gradients back onto the pixels (a gather, not a scatter
+// with atomics, so the fp32 sums have a fixed order).
 #include "tc_gemm.cuh"
 
 namespace {
@@ -103,6 +107,113 @@ int unpack_codes(const uint32_t *planes, long long rows, long long k, int bits, 
     return qnn_launch_status();
 }
 
+
+// ------------------------------------------------------------------------------------------------ convolution staging
+
+struct ConvGeom {
+    int N, H, W, C, Cout, R, S, stride, pad, Ho, Wo, cw;   // cw = ceil(C / 32) words per pixel (tap) and plane
+    long long Mg, Kg;                                      // N*Ho*Wo output pixels, R*S*C reduction length
+};
+
+// im2col of the activation codes, transposed: colt[(tap*C + c)][m] = qa[n][ho*st - pad + r][wo*st - pad + s][c] for
+// output pixel m = (n, ho, wo) and tap = r*S + s, 0 where the tap falls outside the image (the encoded tensor is
+// padded with true zeros).  One thread per output pixel and (tap, channel word): it reads the pixel's plane words
+// once and writes 32 channels; the 32 threads of a warp are consecutive pixels, so every store writes one line.
+template <int BITS>
+__global__ void __launch_bounds__(256) conv_codes_t_kernel(const uint32_t *__restrict__ planes, long long a_pitch, ConvGeom g,
+                                                          float *__restrict__ colt, long long ld) {
+    const long long m = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (m >= g.Mg) return;
+    const int tap = blockIdx.y / g.cw, cwi = blockIdx.y % g.cw;
+    const int r = tap / g.S, sx = tap % g.S;
+    const int wo = (int)(m % g.Wo), ho = (int)((m / g.Wo) % g.Ho);
+    const long long n = m / ((long long)g.Wo * g.Ho);
+    const int hi = ho * g.stride - g.pad + r, wi = wo * g.stride - g.pad + sx;
+    const bool inside = hi >= 0 && hi < g.H && wi >= 0 && wi < g.W;
+    uint32_t w[BITS];
+#pragma unroll
+    for (int b = 0; b < BITS; ++b)
+        w[b] = inside ? __ldg(planes + (((n * g.H + hi) * g.W + wi) * BITS + b) * a_pitch + cwi) : 0u;
+    const float amax = (float)((1 << BITS) - 1);
+    const int ncol = min(32, g.C - cwi * 32);
+    float *o = colt + ((long long)tap * g.C + cwi * 32) * ld + m;
+#pragma unroll 8
+    for (int c = 0; c < 32; ++c) {
+        int t = 0;
+#pragma unroll
+        for (int b = 0; b < BITS; ++b) t |= (int)((w[b] >> c) & 1u) << b;
+        if (c < ncol) o[c * ld] = inside ? (float)(2 * t) - amax : 0.0f;
+    }
+}
+
+// Packed convolution weights [Cout][bits][w_pitch] (tap-major words, each tap on a word boundary) -> codes transposed:
+// wqt[(tap*C + c)][co] = qw[co][tap][c].  One thread per output feature and (tap, channel word).
+template <int BITS>
+__global__ void __launch_bounds__(256) conv_weights_t_kernel(const uint32_t *__restrict__ wp, long long w_pitch, ConvGeom g,
+                                                            float *__restrict__ wqt, long long ld) {
+    const int co = blockIdx.x * 256 + threadIdx.x;
+    if (co >= g.Cout) return;
+    const int tap = blockIdx.y / g.cw, cwi = blockIdx.y % g.cw;
+    uint32_t w[BITS];
+#pragma unroll
+    for (int b = 0; b < BITS; ++b) w[b] = __ldg(wp + ((long long)co * BITS + b) * w_pitch + (long long)tap * g.cw + cwi);
+    const float amax = (float)((1 << BITS) - 1);
+    const int ncol = min(32, g.C - cwi * 32);
+    float *o = wqt + ((long long)tap * g.C + cwi * 32) * ld + co;
+#pragma unroll 8
+    for (int c = 0; c < 32; ++c) {
+        int t = 0;
+#pragma unroll
+        for (int b = 0; b < BITS; ++b) t |= (int)((w[b] >> c) & 1u) << b;
+        if (c < ncol) o[c * ld] = (float)(2 * t) - amax;
+    }
+}
+
+// Gathers the patch gradients back onto the input pixels: out[n][h][w][c] = sum over the taps (r, s) and output pixels
+// (ho, wo) with ho*st - pad + r = h and wo*st - pad + s = w of dcol[(n, ho, wo)][(r*S + s)*C + c], taps in
+// increasing (r, s) order (a gather, so the sum has a fixed order).  BITS > 0: the encoder derivative of Eq. 12 is
+// applied to the sum (x = what the previous layer fed its encoder, as in qnn_bgemm_backward_data).
+template <int BITS>
+__global__ void __launch_bounds__(256) conv_col2im_kernel(const float *__restrict__ dcol, ConvGeom g, const float *__restrict__ x,
+                                                         float r_range, MbitPlaneConsts enc, float *__restrict__ out) {
+    const long long total = (long long)g.N * g.H * g.W * g.C;
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+        const int c = (int)(i % g.C);
+        const long long pix = i / g.C;
+        const int w = (int)(pix % g.W), h = (int)((pix / g.W) % g.H);
+        const long long n = pix / ((long long)g.W * g.H);
+        float sum = 0.0f;
+        for (int r = 0; r < g.R; ++r) {
+            const int th = h + g.pad - r;
+            if (th < 0 || th % g.stride) continue;
+            const int ho = th / g.stride;
+            if (ho >= g.Ho) continue;
+            for (int sx = 0; sx < g.S; ++sx) {
+                const int tw = w + g.pad - sx;
+                if (tw < 0 || tw % g.stride) continue;
+                const int wo = tw / g.stride;
+                if (wo >= g.Wo) continue;
+                sum = __fadd_rn(sum, __ldg(dcol + ((n * g.Ho + ho) * g.Wo + wo) * g.Kg + (long long)(r * g.S + sx) * g.C + c));
+            }
+        }
+        if constexpr (BITS > 0) sum = mbit_backward_shared<BITS>(__ldg(x + i), r_range, sum, enc);
+        out[i] = sum;
+    }
+}
+
+bool conv_geom(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad, ConvGeom *g) {
+    if (N < 1 || H < 1 || W < 1 || C < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0) return false;
+    const long long Ho = ((long long)H + 2 * pad - R) / stride + 1, Wo = ((long long)W + 2 * pad - S) / stride + 1;
+    if ((long long)H + 2 * pad < R || (long long)W + 2 * pad < S || Ho < 1 || Wo < 1) return false;
+    g->N = N; g->H = H; g->W = W; g->C = C; g->Cout = Cout; g->R = R; g->S = S; g->stride = stride; g->pad = pad;
+    g->Ho = (int)Ho; g->Wo = (int)Wo; g->cw = (C + 31) / 32;
+    g->Mg = (long long)N * Ho * Wo;
+    g->Kg = (long long)R * S * C;
+    return true;
+}
+
+size_t round256(size_t v) { return (v + 255) / 256 * 256; }
+
 }  // namespace
 
 // Device address of the word in which a tensor-path kernel of any translation unit records a wait that gave up.
@@ -196,6 +307,124 @@ extern "C" int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_plan
     p.C = gw; p.ldc = (long long)k;
     if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
     return run_gemm<TC_TF32>(gt, ldm, aqt, ldm, p, st);
+}
+
+
+// ------------------------------------------------------------------------------------------------ convolution backward
+
+static bool conv_backward_dims_ok(const ConvGeom &g) {
+    return g.Mg <= (long long)DIM_LIMIT && g.Kg <= (long long)DIM_LIMIT && (size_t)g.Cout <= DIM_LIMIT &&
+           (long long)g.R * g.S * g.cw <= 65535 && (long long)g.N * g.H * g.W <= (1ll << 40);
+}
+
+extern "C" size_t qnn_bconv2d_backward_data_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad) {
+    ConvGeom g;
+    if (!conv_geom(N, H, W, C, Cout, R, S, stride, pad, &g) || !conv_backward_dims_ok(g)) return 0;
+    const size_t ldn = (size_t)pad32(Cout);
+    return round256((size_t)g.Kg * ldn * 4) + (Cout % 4 ? round256((size_t)g.Mg * ldn * 4) : 0) + round256((size_t)g.Mg * g.Kg * 4);
+}
+
+extern "C" int qnn_bconv2d_backward_data(const float *g, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
+                                         int R, int S, int stride, int pad, float alpha, const float *x, int ab, float r,
+                                         float *out, void *workspace, size_t workspace_bytes, void *stream) {
+    ConvGeom cg;
+    if (!g || !w_packed || !out || !workspace || !qnn_bits_ok(wb) || !conv_geom(N, H, W, C, Cout, R, S, stride, pad, &cg) ||
+        !conv_backward_dims_ok(cg))
+        return QNN_E_ARG;
+    if (x && !qnn_bits_ok(ab)) return QNN_E_ARG;
+    if (!(fabsf(alpha) <= 3.0e38f)) return QNN_E_SCALE;
+    if (x && (!(r >= 1e-30f) || !(r <= 1e30f))) return QNN_E_SCALE;
+    if (workspace_bytes < qnn_bconv2d_backward_data_workspace(N, H, W, C, Cout, R, S, stride, pad)) return QNN_E_ARG;
+    if (!qnn_aligned(g, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(workspace, 256) || !qnn_aligned(out, 4) ||
+        (x && !qnn_aligned(x, 4)))
+        return QNN_E_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long ldn = pad32(Cout);
+    char *ws = static_cast<char *>(workspace);
+    float *wqt = reinterpret_cast<float *>(ws);                         // [Kg][ldn]
+    ws += round256((size_t)cg.Kg * ldn * 4);
+    const dim3 wgrid((unsigned)qnn_ceil_div(Cout, 256), (unsigned)(R * S * cg.cw));
+    const long long w_pitch = qnn_w_row_words_i(R * S, C);
+#define CONV_W_CASE(B) case B: conv_weights_t_kernel<B><<<wgrid, 256, 0, st>>>(static_cast<const uint32_t *>(w_packed), w_pitch, cg, wqt, ldn); break;
+    switch (wb) {
+        CONV_W_CASE(1) CONV_W_CASE(2) CONV_W_CASE(3) CONV_W_CASE(4) CONV_W_CASE(5) CONV_W_CASE(6) CONV_W_CASE(7)
+        default: conv_weights_t_kernel<8><<<wgrid, 256, 0, st>>>(static_cast<const uint32_t *>(w_packed), w_pitch, cg, wqt, ldn); break;
+    }
+#undef CONV_W_CASE
+    int rc = qnn_launch_status();
+    if (rc != QNN_OK) return rc;
+    const float *a = g;
+    long long lda = Cout;
+    if (Cout % 4) {                                                     // rows of g are not 16-byte multiples
+        float *gp = reinterpret_cast<float *>(ws);
+        ws += round256((size_t)cg.Mg * ldn * 4);
+        copy_rows_kernel<<<148 * 8, 256, 0, st>>>(g, cg.Mg, (long long)Cout, gp, ldn);
+        if ((rc = qnn_launch_status()) != QNN_OK) return rc;
+        a = gp;
+        lda = ldn;
+    }
+    float *dcol = reinterpret_cast<float *>(ws);                        // [Mg][Kg]: gradient of every patch element
+    GemmParams p{};
+    p.M = (int)cg.Mg; p.N = (int)cg.Kg; p.K = Cout;
+    p.alpha = alpha;
+    p.C = dcol; p.ldc = cg.Kg;
+    if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
+    if ((rc = run_gemm<TC_TF32>(a, lda, wqt, ldn, p, st)) != QNN_OK) return rc;
+    const long long total = (long long)N * H * W * C;
+    const int blocks = (int)(qnn_ceil_div(total, 256) < 148 * 16 ? qnn_ceil_div(total, 256) : 148 * 16);
+    MbitPlaneConsts enc = x ? mbit_plane_consts(ab) : MbitPlaneConsts{};
+#define CONV_C2I_CASE(B) case B: conv_col2im_kernel<B><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out); break;
+    switch (x ? ab : 0) {
+        CONV_C2I_CASE(0) CONV_C2I_CASE(1) CONV_C2I_CASE(2) CONV_C2I_CASE(3) CONV_C2I_CASE(4) CONV_C2I_CASE(5) CONV_C2I_CASE(6)
+        CONV_C2I_CASE(7)
+        default: conv_col2im_kernel<8><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out); break;
+    }
+#undef CONV_C2I_CASE
+    return qnn_launch_status();
+}
+
+extern "C" size_t qnn_bconv2d_backward_weights_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride,
+                                                         int pad) {
+    ConvGeom g;
+    if (!conv_geom(N, H, W, C, Cout, R, S, stride, pad, &g) || !conv_backward_dims_ok(g)) return 0;
+    const size_t ldm = (size_t)pad32(g.Mg);
+    return round256((size_t)Cout * ldm * 4) + round256((size_t)g.Kg * ldm * 4);
+}
+
+extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_planes, int ab, int N, int H, int W, int C,
+                                            int Cout, int R, int S, int stride, int pad, float alpha, float *gw,
+                                            void *workspace, size_t workspace_bytes, void *stream) {
+    ConvGeom cg;
+    if (!g || !a_planes || !gw || !workspace || !qnn_bits_ok(ab) || !conv_geom(N, H, W, C, Cout, R, S, stride, pad, &cg) ||
+        !conv_backward_dims_ok(cg))
+        return QNN_E_ARG;
+    if (!(fabsf(alpha) <= 3.0e38f)) return QNN_E_SCALE;
+    if (workspace_bytes < qnn_bconv2d_backward_weights_workspace(N, H, W, C, Cout, R, S, stride, pad)) return QNN_E_ARG;
+    if (!qnn_aligned(g, 4) || !qnn_aligned(a_planes, 16) || !qnn_aligned(workspace, 256) || !qnn_aligned(gw, 4))
+        return QNN_E_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long ldm = pad32(cg.Mg);
+    float *gt = static_cast<float *>(workspace);                        // [Cout][ldm]: gt[co][m] = g[m][co]
+    float *colt = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)Cout * ldm * 4));   // [Kg][ldm]
+    const dim3 tgrid((unsigned)qnn_ceil_div(Cout, 32), (unsigned)qnn_ceil_div(cg.Mg, 32));
+    transpose_f32_kernel<<<tgrid, 256, 0, st>>>(g, cg.Mg, (long long)Cout, (long long)Cout, gt, ldm);
+    int rc = qnn_launch_status();
+    if (rc != QNN_OK) return rc;
+    const dim3 cgrid((unsigned)qnn_ceil_div(cg.Mg, 256), (unsigned)(R * S * cg.cw));
+    const long long a_pitch = qnn_row_words_i(C);
+#define CONV_A_CASE(B) case B: conv_codes_t_kernel<B><<<cgrid, 256, 0, st>>>(a_planes, a_pitch, cg, colt, ldm); break;
+    switch (ab) {
+        CONV_A_CASE(1) CONV_A_CASE(2) CONV_A_CASE(3) CONV_A_CASE(4) CONV_A_CASE(5) CONV_A_CASE(6) CONV_A_CASE(7)
+        default: conv_codes_t_kernel<8><<<cgrid, 256, 0, st>>>(a_planes, a_pitch, cg, colt, ldm); break;
+    }
+#undef CONV_A_CASE
+    if ((rc = qnn_launch_status()) != QNN_OK) return rc;
+    GemmParams p{};
+    p.M = Cout; p.N = (int)cg.Kg; p.K = (int)cg.Mg;
+    p.alpha = alpha;
+    p.C = gw; p.ldc = cg.Kg;
+    if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
+    return run_gemm<TC_TF32>(gt, ldm, colt, ldm, p, st);
 }
 
 extern "C" int qnn_tensor_path_status(unsigned int *status) {

@@ -22,7 +22,8 @@ EXPORTS = [
     "qnn_weights_row_words", "qnn_encode_pack", "qnn_pack_weights", "qnn_bgemm", "qnn_bconv2d",
     "qnn_bgemm_encode", "qnn_bconv2d_encode", "qnn_bconv2d_general", "qnn_mbit_encoder_forward",
     "qnn_mbit_encoder_backward", "qnn_bgemm_backward_data_workspace", "qnn_bgemm_backward_data",
-    "qnn_bgemm_backward_weights_workspace", "qnn_bgemm_backward_weights", "qnn_unpack_codes_f32",
+    "qnn_bgemm_backward_weights_workspace", "qnn_bgemm_backward_weights", "qnn_bconv2d_backward_data_workspace",
+    "qnn_bconv2d_backward_data", "qnn_bconv2d_backward_weights_workspace", "qnn_bconv2d_backward_weights", "qnn_unpack_codes_f32",
     "qnn_tensor_path_status", "qnn_bgemm_int8_tensor_workspace", "qnn_bgemm_int8_tensor",
     "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
 ]
@@ -68,6 +69,12 @@ def _load() -> C.CDLL:
     lib.qnn_bgemm_backward_weights_workspace.argtypes = [sz, sz, sz]
     lib.qnn_bgemm_backward_weights.argtypes = [p, p, sz, sz, sz, i, f, p, p, sz, p]
     lib.qnn_unpack_codes_f32.argtypes = [p, sz, sz, i, i, p, sz, p]
+    lib.qnn_bconv2d_backward_data_workspace.restype = sz
+    lib.qnn_bconv2d_backward_data_workspace.argtypes = [i] * 9
+    lib.qnn_bconv2d_backward_data.argtypes = [p, p, i] + [i] * 9 + [f, p, i, f, p, p, sz, p]
+    lib.qnn_bconv2d_backward_weights_workspace.restype = sz
+    lib.qnn_bconv2d_backward_weights_workspace.argtypes = [i] * 9
+    lib.qnn_bconv2d_backward_weights.argtypes = [p, p, i] + [i] * 9 + [f, p, p, sz, p]
     lib.qnn_tensor_path_status.argtypes = [C.POINTER(C.c_uint)]
     lib.qnn_bgemm_int8_tensor_workspace.restype = sz
     lib.qnn_bgemm_int8_tensor_workspace.argtypes = [i64, i, i]
@@ -296,6 +303,37 @@ def bgemm_backward_weights(g: torch.Tensor, a_planes: torch.Tensor, k: int, ab: 
     ws = _workspace(lib.qnn_bgemm_backward_weights_workspace(m, n, k), g.device, workspace)
     _check(lib.qnn_bgemm_backward_weights(_ptr(g), _ptr(a_planes), m, n, k, ab, float(alpha), _ptr(gw), _ptr(ws),
                                           ws.numel() * ws.element_size(), _stream(stream)), "qnn_bgemm_backward_weights")
+    return gw
+
+
+def bconv2d_backward_data(g: torch.Tensor, w_packed: torch.Tensor, wb: int, H: int, W: int, C: int, R: int, S: int,
+                          stride: int, pad: int, alpha: float, x: torch.Tensor | None = None, ab: int = 1, r: float = 1.0,
+                          out: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Algorithm 1 backward of a convolution, activation side: g fp32 [N, Ho, Wo, Cout], packed weights -> fp32 [N, H, W, C]."""
+    _dev(g, torch.float32, "g")
+    N, Cout = g.shape[0], g.shape[3]
+    if out is None:
+        out = torch.empty((N, H, W, C), dtype=torch.float32, device=g.device)
+    ws = _workspace(lib.qnn_bconv2d_backward_data_workspace(N, H, W, C, Cout, R, S, stride, pad), g.device, workspace)
+    _check(lib.qnn_bconv2d_backward_data(_ptr(g), _ptr(w_packed), wb, N, H, W, C, Cout, R, S, stride, pad, float(alpha),
+                                         _ptr(x), ab, float(r), _ptr(out), _ptr(ws), ws.numel() * ws.element_size(),
+                                         _stream(stream)), "qnn_bconv2d_backward_data")
+    return out
+
+
+def bconv2d_backward_weights(g: torch.Tensor, a_planes: torch.Tensor, ab: int, H: int, W: int, C: int, R: int, S: int,
+                             stride: int, pad: int, alpha: float, gw: torch.Tensor | None = None,
+                             workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Algorithm 1 backward of a convolution, weight side: g fp32 [N, Ho, Wo, Cout], a_planes [N*H*W, ab, row_words(C)]
+    -> GW fp32 [Cout, R, S, C]."""
+    _dev(g, torch.float32, "g")
+    N, Cout = g.shape[0], g.shape[3]
+    if gw is None:
+        gw = torch.empty((Cout, R, S, C), dtype=torch.float32, device=g.device)
+    ws = _workspace(lib.qnn_bconv2d_backward_weights_workspace(N, H, W, C, Cout, R, S, stride, pad), g.device, workspace)
+    _check(lib.qnn_bconv2d_backward_weights(_ptr(g), _ptr(a_planes), ab, N, H, W, C, Cout, R, S, stride, pad, float(alpha),
+                                            _ptr(gw), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)),
+           "qnn_bconv2d_backward_weights")
     return gw
 
 

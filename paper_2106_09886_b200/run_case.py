@@ -3,6 +3,7 @@
     python -m paper_2106_09886_b200.run_case gemm   --m 4096 --n 4096 --k 4096 --ab 2 --wb 2 [--reps 5]
     python -m paper_2106_09886_b200.run_case conv   --N 32 --H 14 --W 14 --C 256 --Cout 256 --R 3 --S 3 --stride 1 --pad 1 --ab 2 --wb 2
     python -m paper_2106_09886_b200.run_case encode --rows 4096 --k 4096 --bits 2
+    python -m paper_2106_09886_b200.run_case backward_conv --N 32 --H 14 --W 14 --C 256 --Cout 256
     python -m paper_2106_09886_b200.run_case stack  --net vgg16 [--batch 64] [--layers 0,1] [--table]
 
 Inputs are drawn on the device (half-normal activations, normal weights); this is a timing and
@@ -166,6 +167,31 @@ def time_backward(m, n, k, ab, wb, reps=5, warmup=3, dev="cuda:0", seed=0):
             "weights_tflops": fl / (tw * 1e-3) / 1e12}
 
 
+def time_backward_conv(N, H, W, C, Cout, R, S, stride, pad, ab, wb, reps=5, warmup=3, dev="cuda:0", seed=0):
+    """Backward products of one convolution layer: whole calls (patch staging + TF32 tensor-core GEMM + gather)."""
+    g = torch.Generator(device=dev).manual_seed(seed)
+    Ho, Wo = qnn.conv_out_dim(H, R, stride, pad), qnn.conv_out_dim(W, S, stride, pad)
+    grad = torch.randn((N, Ho, Wo, Cout), device=dev, generator=g)
+    x = torch.rand((N * H * W, C), device=dev, generator=g) * 2 - 1
+    a_planes = qnn.encode_pack(x, ab, 1.0 / (2 ** ab - 1))
+    w = torch.randn((Cout, R, S, C), device=dev, generator=g).clamp_(-1, 1)
+    packed = qnn.pack_weights(w, Cout, R * S, C, qnn.W_NTC, wb, 1.0 / (2 ** wb - 1))
+    alpha = 1.0 / ((2 ** ab - 1) * (2 ** wb - 1))
+    out = torch.empty((N, H, W, C), dtype=torch.float32, device=dev)
+    gw = torch.empty((Cout, R, S, C), dtype=torch.float32, device=dev)
+    wsd = torch.empty(qnn.lib.qnn_bconv2d_backward_data_workspace(N, H, W, C, Cout, R, S, stride, pad) + 256, dtype=torch.uint8, device=dev)
+    wsw = torch.empty(qnn.lib.qnn_bconv2d_backward_weights_workspace(N, H, W, C, Cout, R, S, stride, pad) + 256, dtype=torch.uint8, device=dev)
+    med = lambda f: statistics.median(_time_calls(f, reps, warmup))
+    td = med(lambda i: qnn.bconv2d_backward_data(grad, packed, wb, H, W, C, R, S, stride, pad, alpha, out=out, workspace=wsd))
+    tw = med(lambda i: qnn.bconv2d_backward_weights(grad, a_planes, ab, H, W, C, R, S, stride, pad, alpha, gw=gw, workspace=wsw))
+    status = qnn.tensor_path_status()
+    fl = 2.0 * N * Ho * Wo * Cout * R * S * C
+    return {"call": "qnn_bconv2d_backward", "N": N, "H": H, "W": W, "C": C, "Cout": Cout, "R": R, "S": S, "stride": stride,
+            "pad": pad, "ab": ab, "wb": wb, "status": status, "data_ms": td, "weights_ms": tw,
+            "data_tflops": fl / (td * 1e-3) / 1e12, "weights_tflops": fl / (tw * 1e-3) / 1e12,
+            "workspace_mb": [wsd.numel() / 1e6, wsw.numel() / 1e6]}
+
+
 def _report(call, Mg, Ng, Kg, ab, wb, times):
     ms = statistics.median(times)
     macs = float(Mg) * Ng * Kg
@@ -196,12 +222,16 @@ def main():
     bw.add_argument("--k", type=int, default=4096)
     bw.add_argument("--ab", type=int, default=2)
     bw.add_argument("--wb", type=int, default=2)
+    bc = sub.add_parser("backward_conv")
+    for name, default in (("N", 32), ("H", 14), ("W", 14), ("C", 256), ("Cout", 256), ("R", 3), ("S", 3),
+                          ("stride", 1), ("pad", 1), ("ab", 2), ("wb", 2)):
+        bc.add_argument(f"--{name}", type=int, default=default)
     k = sub.add_parser("stack")
     k.add_argument("--net", choices=["resnet18", "resnet18_p1", "resnet18_p2", "vgg16"], default="resnet18")
     k.add_argument("--batch", type=int, default=0)
     k.add_argument("--layers", type=str, default="")
     k.add_argument("--table", action="store_true")
-    for s in (g, c, e, k, mb, bw):
+    for s in (g, c, e, k, mb, bw, bc):
         s.add_argument("--reps", type=int, default=5)
         s.add_argument("--warmup", type=int, default=3)
         s.add_argument("--sets", type=int, default=3)
@@ -212,6 +242,8 @@ def main():
         r = time_conv(a.N, a.H, a.W, a.C, a.Cout, a.R, a.S, a.stride, a.pad, a.ab, a.wb, a.reps, a.warmup, a.sets)
     elif a.case == "backward":
         r = time_backward(a.m, a.n, a.k, a.ab, a.wb, a.reps, a.warmup)
+    elif a.case == "backward_conv":
+        r = time_backward_conv(a.N, a.H, a.W, a.C, a.Cout, a.R, a.S, a.stride, a.pad, a.ab, a.wb, a.reps, a.warmup)
     elif a.case == "mbit":
         r = time_mbit(a.n, a.bits, a.reps, a.warmup)
     elif a.case == "stack":

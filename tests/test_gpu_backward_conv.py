@@ -1,0 +1,142 @@
+"""GPU parity of the backward products of a convolution layer (Algorithm 1 backward; TF32 tensor-core contractions
+on an explicit patch matrix) against the CPU oracle.
+
+Tolerance, element by element, as for the fully-connected products:
+    |got - want| <= alpha * sum |g| * |q| * (2^-10 + (L + T) * 2^-24)
+over the terms of that element's sum, with L the contraction length on the tensor cores (Cout for the data gradient,
+N*Ho*Wo for the weight gradient) and T = R*S the fp32 additions of the gather that follows (data gradient only).
+Integer-valued g with alpha a power of two is contracted exactly and compared with ==, which pins every index of the
+patch staging, the tap-major weight layout and the gather independently of rounding."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import oracle_weight_planes
+
+pytestmark = pytest.mark.gpu
+
+# (N, H, W, C, Cout, R, S, stride, pad): ragged channel counts, strides, 1x1, a 5x5, Cout % 4 != 0 (padded copy of g)
+GEOMS = [(2, 6, 5, 3, 4, 3, 3, 1, 1), (1, 9, 9, 40, 6, 3, 3, 2, 1), (3, 8, 8, 64, 16, 1, 1, 2, 0), (2, 7, 6, 33, 5, 5, 5, 1, 2),
+         (2, 14, 14, 128, 32, 3, 3, 1, 1), (1, 5, 4, 70, 130, 3, 2, 1, 0), (5, 12, 12, 16, 24, 3, 3, 2, 2)]
+
+
+def _codes(rng, shape, bits):
+    return (2 * rng.integers(0, 2 ** bits, size=shape) - (2 ** bits - 1)).astype(np.int16)
+
+
+def _packed_weights_dev(qw, wb, dev):
+    """The blob qnn_pack_weights would write for these codes, assembled from the oracle's canonical packer."""
+    import torch
+    Cout, R, S, C = qw.shape
+    planes, tapsum = oracle_weight_planes(qw.reshape(Cout, R * S, C), wb)
+    blob = np.concatenate([planes.reshape(-1).view(np.uint8), tapsum.reshape(-1).view(np.uint8)])
+    return torch.from_numpy(blob).to(dev)
+
+
+def _case(seed, geom, ab, wb, integer_g):
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    rng = np.random.default_rng(seed)
+    qa, qw = _codes(rng, (N, H, W, C), ab), _codes(rng, (Cout, R, S, C), wb)
+    Ho, Wo = oracle.conv_out_dim(H, R, stride, pad), oracle.conv_out_dim(W, S, stride, pad)
+    g = (rng.integers(-8, 9, size=(N, Ho, Wo, Cout)) if integer_g else rng.standard_normal((N, Ho, Wo, Cout))).astype(np.float32)
+    return qa, qw, g
+
+
+@pytest.mark.parametrize("geom", GEOMS)
+@pytest.mark.parametrize("wb", [1, 3, 8])
+def test_conv_backward_data_exact_on_integer_gradients(geom, wb):
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(sum(geom) + wb, geom, 1, wb, True)
+    want = oracle.conv_backward_data(g, qw, (H, W), stride, pad, 1, wb, 0.25)[0]
+    got = qnn.bconv2d_backward_data(torch.from_numpy(g).to(dev), _packed_weights_dev(qw, wb, dev), wb, H, W, C, R, S,
+                                    stride, pad, 0.25).cpu().numpy()
+    assert qnn.tensor_path_status() == 0
+    assert np.array_equal(got.astype(np.float64), want)
+
+
+@pytest.mark.parametrize("geom", GEOMS)
+@pytest.mark.parametrize("ab", [1, 2, 8])
+def test_conv_backward_weights_exact_on_integer_gradients(geom, ab):
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(sum(geom) * 3 + ab, geom, ab, 1, True)
+    want = oracle.conv_backward_weights(g, qa, (R, S), stride, pad, ab, 1, 0.25)[0]
+    planes = torch.from_numpy(oracle.pack_planes(qa.reshape(-1, C), ab).view(np.int32)).to(dev)
+    got = qnn.bconv2d_backward_weights(torch.from_numpy(g).to(dev), planes, ab, H, W, C, R, S, stride, pad, 0.25).cpu().numpy()
+    assert qnn.tensor_path_status() == 0
+    assert np.array_equal(got.astype(np.float64), want)
+
+
+@pytest.mark.parametrize("geom,ab,wb", [((2, 14, 14, 64, 48, 3, 3, 1, 1), 2, 2), ((4, 16, 16, 32, 64, 3, 3, 2, 1), 3, 4),
+                                        ((1, 10, 9, 100, 36, 1, 1, 1, 0), 8, 8)])
+def test_conv_backward_within_tf32_bound(geom, ab, wb):
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(sum(geom), geom, ab, wb, False)
+    alpha = float(np.float32(0.8 / ((2 ** ab - 1) * (2 ** wb - 1))))
+    gd = torch.from_numpy(g).to(dev)
+    G = qnn.bconv2d_backward_data(gd, _packed_weights_dev(qw, wb, dev), wb, H, W, C, R, S, stride, pad, alpha).cpu().numpy()
+    planes = torch.from_numpy(oracle.pack_planes(qa.reshape(-1, C), ab).view(np.int32)).to(dev)
+    GW = qnn.bconv2d_backward_weights(gd, planes, ab, H, W, C, R, S, stride, pad, alpha).cpu().numpy()
+    assert qnn.tensor_path_status() == 0
+    ga = oracle.conv_backward_data(g, qw, (H, W), stride, pad, ab, wb, alpha)
+    gw = oracle.conv_backward_weights(g, qa, (R, S), stride, pad, ab, wb, alpha)
+    # sums of magnitudes: the same two oracle functions on |g| and on all-(+max) stand-ins are not available for
+    # arbitrary codes, so take them from the plain definition with absolute values (1-bit planes of +1 = |q| bound)
+    Mg = g.shape[0] * g.shape[1] * g.shape[2]
+    mag_d = oracle.conv_backward_data(np.abs(g), np.full_like(qw, 2 ** wb - 1), (H, W), stride, pad, 1, wb, alpha)[0]
+    mag_w = oracle.conv_backward_weights(np.abs(g), np.full_like(qa, 2 ** ab - 1), (R, S), stride, pad, ab, 1, alpha)[0]
+    bd = mag_d * (2.0 ** -10 + (Cout + R * S) * 2.0 ** -24)
+    bw = mag_w * (2.0 ** -10 + Mg * 2.0 ** -24)
+    for p in range(ab):
+        assert np.all(np.abs(2.0 ** p * G.astype(np.float64) - ga[p]) <= 2.0 ** p * bd * (1 + 2.0 ** -20) + 1e-30)
+    for j in range(wb):
+        assert np.all(np.abs(2.0 ** j * GW.astype(np.float64) - gw[j]) <= 2.0 ** j * bw * (1 + 2.0 ** -20) + 1e-30)
+    assert np.sqrt(np.mean((G - ga[0]) ** 2)) <= 0.1 * np.sqrt(np.mean(bd ** 2))
+    assert np.sqrt(np.mean((GW - gw[0]) ** 2)) <= 0.1 * np.sqrt(np.mean(bw ** 2))
+
+
+def test_conv_backward_data_through_the_encoder():
+    """With x given the gather applies Eq. 12 to gc_p = 2^(p-1) * G: compared with the oracle's two steps chained."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    geom, ab, wb = (2, 9, 8, 24, 16, 3, 3, 1, 1), 3, 2
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(11, geom, ab, wb, True)
+    rng = np.random.default_rng(5)
+    x = (rng.random((N, H, W, C)) * 2.4 - 1.2).astype(np.float32)          # some elements outside [-r, r]
+    r = 1.0
+    got = qnn.bconv2d_backward_data(torch.from_numpy(g).to(dev), _packed_weights_dev(qw, wb, dev), wb, H, W, C, R, S, stride,
+                                    pad, 0.25, x=torch.from_numpy(x).to(dev), ab=ab, r=r).cpu().numpy()
+    assert qnn.tensor_path_status() == 0
+    ga = oracle.conv_backward_data(g, qw, (H, W), stride, pad, ab, wb, 0.25)       # exact here (integer g)
+    want = oracle.mbit_encoder_backward(x.reshape(-1), ga.reshape(ab, -1), ab, r).reshape(x.shape)
+    # the products are exact; what remains is the binary32 evaluation of Eq. 12 (same bound as the stand-alone kernel)
+    k = np.array([(2 ** ab - 1) / 2 ** m for m in range(1, ab + 1)])
+    tol = (np.abs(ga).reshape(ab, -1) * (k * np.pi * (np.pi * k + 8))[:, None]).sum(axis=0).reshape(x.shape) * 2.0 ** -24 / r
+    assert np.all(np.abs(got - want) <= tol + 1e-30)
+    assert np.all(got[np.abs(x) > r] == 0.0)
+
+
+def test_conv_backward_rejects_bad_arguments():
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    g = torch.zeros((1, 4, 4, 8), device=dev)
+    assert qnn.lib.qnn_bconv2d_backward_data_workspace(1, 2, 2, 8, 8, 3, 3, 1, 0) == 0          # kernel larger than input
+    assert qnn.lib.qnn_bconv2d_backward_weights_workspace(1, 4, 4, 8, 8, 3, 3, 0, 1) == 0        # stride 0
+    qw = np.ones((8, 3, 3, 8), dtype=np.int16)
+    blob = _packed_weights_dev(qw, 1, dev)
+    small = torch.empty(16, dtype=torch.uint8, device=dev)
+    with pytest.raises(qnn.QnnError):
+        qnn.bconv2d_backward_data(g, blob, 1, 4, 4, 8, 3, 3, 1, 1, 1.0, workspace=small)
+    with pytest.raises(qnn.QnnError):
+        qnn.bconv2d_backward_data(g, blob, 9, 4, 4, 8, 3, 3, 1, 1, 1.0)
