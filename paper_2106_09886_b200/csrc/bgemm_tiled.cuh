@@ -171,6 +171,10 @@ __device__ __forceinline__ void pair9(const uint32_t (&ta)[9], const uint32_t (&
 template <int AB, int WB, int KIND, int TM, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p) {
     constexpr bool CONV = KIND != 0, GENERAL = KIND == 2, G9 = KIND == 3;
+    // multiply-shift division in the tile bookkeeping: convolutions with ab <= 4 only (the fully-connected kernels
+    // divide once per tile, and both they and the 16-row-tile kernels for ab >= 5 ran 2-5% slower with it compiled
+    // in, through register-allocation side effects)
+    constexpr bool FASTDIV = CONV && AB <= 4;
     constexpr int kBM = 16 * TM;
     constexpr int A_UNITS = kBM * AB * kStageChunks;      // (row, plane, group) units per stage
     constexpr int W_UNITS = kBN * WB * kStageChunks;
@@ -203,9 +207,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
     };
     auto prep_tile = [&](int tile) {
         TileSrc t;
-        // (the fully-connected kernels keep the plain division: one per tile, and the other form cost them 2%
-        // through code-generation side effects)
-        const int tile_n = CONV ? (int)fastdiv((uint32_t)tile, p.tm_magic, p.tm_shift) : tile / p.tiles_m;
+        const int tile_n = FASTDIV ? (int)fastdiv((uint32_t)tile, p.tm_magic, p.tm_shift) : tile / p.tiles_m;
         const int64_t m0 = (int64_t)(tile - tile_n * p.tiles_m) * kBM;
         const int n0 = tile_n * kBN;
         const int64_t am = m0 + srow;
@@ -217,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             const int64_t mm = t.a_ok ? am : 0;
             int wo, ho;
             int64_t n;
-            if (p.fast_pix) {
+            if (FASTDIV && p.fast_pix) {
                 const uint32_t m32 = (uint32_t)mm;
                 const uint32_t q = fastdiv(m32, p.wo_magic, p.wo_shift), img = fastdiv(m32, p.howo_magic, p.howo_shift);
                 wo = (int)(m32 - q * (uint32_t)p.Wo);
@@ -489,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
 
         // ---- epilogue: acc holds S = sum_ij 2^(i+j) X_ij.  out = n_valid*A*B - 2*S (Eq. 8), times alpha (Eq. 9).
         constexpr int AMAX = (1 << AB) - 1, PROD = AMAX * ((1 << WB) - 1);
-        const int tile_n = CONV ? (int)fastdiv((uint32_t)tile, p.tm_magic, p.tm_shift) : tile / p.tiles_m;
+        const int tile_n = FASTDIV ? (int)fastdiv((uint32_t)tile, p.tm_magic, p.tm_shift) : tile / p.tiles_m;
         const int64_t m0 = (int64_t)(tile - tile_n * p.tiles_m) * kBM;
         const int n0 = tile_n * kBN;
 #pragma unroll
@@ -503,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 // Taps outside the image were staged as zero words: each contributed popc(w_j) to X_ij, i.e.
                 // AMAX * tapsum[n][tap] to S, and must not be counted in the length.
                 int wo, ho;
-                if (p.fast_pix) {
+                if (FASTDIV && p.fast_pix) {
                     const uint32_t m32 = (uint32_t)m;
                     const uint32_t q = fastdiv(m32, p.wo_magic, p.wo_shift), img = fastdiv(m32, p.howo_magic, p.howo_shift);
                     wo = (int)(m32 - q * (uint32_t)p.Wo);
