@@ -41,7 +41,7 @@ AB, WB = 2, 2
 NBUF = 4           # rotating input/output sets: 4 x (64 MiB in + 64 MiB out) >> 126 MB of L2
 METRIC = "binary TOPS, qnn_encode_pack + qnn_bgemm (equiv. int GOPS and % of roofline alongside)"
 UNIT = "binary TOPS"
-E2E_CHUNK_ROWS, E2E_STREAMS = 512, 4
+E2E_CHUNK_ROWS, E2E_STREAMS = 1024, 8   # measured best of a sweep (256..2048 rows, 2..32 streams)
 POPC_PER_WORD = 0.5   # popcounts the tiled kernel issues per 32-bit xor word (7:3 bit-column counters)
 
 
@@ -451,12 +451,14 @@ def run_gpu(args):
     gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
 
     # ---- end to end through the host-buffer entry point
-    e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(E2E_STREAMS)]
+    e2e_streams = [torch.cuda.Stream(device=dev) for _ in range(args.e2e_streams)]
 
-    def e2e_step(i):
+    def e2e_step(i, last=True):
+        # consecutive steps pipeline into each other on the same streams (step i+1's copies in overlap step i's
+        # kernels and copies out); the last step of a batch joins the streams before the closing event
         b = i % NBUF
         qnn.fc_forward_host_pipelined(a_host, AB, sa, 0, packed, WB, Ng, alpha, out_host, a_bufs[b], planes[b],
-                                      out_bufs[b], E2E_CHUNK_ROWS, e2e_streams)
+                                      out_bufs[b], args.e2e_chunk_rows, e2e_streams, join=last)
 
     e2e_steps = max(3, min(args.steps, 50))
     for i in range(3):
@@ -465,7 +467,7 @@ def run_gpu(args):
     s2, t2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s2.record()
     for i in range(e2e_steps):
-        e2e_step(i)
+        e2e_step(i, last=(i == e2e_steps - 1))
     t2.record()
     barrier()
     e2e_ms_total = s2.elapsed_time(t2)
@@ -501,8 +503,8 @@ def run_gpu(args):
             "gpu_launches": 2 * args.steps,
             "e2e": {"value": ops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": Mg * Kg * 4, "d2h_bytes_per_step": Mg * Ng * 4, "steps": e2e_steps,
-                    "api": f"qnn_fc_forward_host_pipelined (pinned host buffers, {E2E_CHUNK_ROWS}-row chunks over "
-                           f"{E2E_STREAMS} streams)", "checksum": checksum},
+                    "api": f"qnn_fc_forward_host_pipelined (pinned host buffers, {args.e2e_chunk_rows}-row chunks over "
+                           f"{args.e2e_streams} streams, consecutive steps pipelined)", "checksum": checksum},
             "roofline": {"kernel": "qnn_bgemm", "bound": "alu", "achieved": achieved, "peak": kernel_peak,
                          "unit": UNIT, "frac": achieved / kernel_peak, "traffic": traffic,
                          "peak_source": "popcount issue rate measured in this run by the register-resident xor+popc+add "
@@ -541,6 +543,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["graft", "reference"], default="graft")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-chunk-rows", type=int, default=E2E_CHUNK_ROWS, help="rows per chunk of the end-to-end pipeline")
+    ap.add_argument("--e2e-streams", type=int, default=E2E_STREAMS, help="streams of the end-to-end pipeline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":

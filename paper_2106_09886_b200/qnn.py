@@ -387,9 +387,12 @@ def fc_forward_host(x_host: torch.Tensor, ab: int, scale_a: float, flags: int, w
 
 def fc_forward_host_pipelined(x_host: torch.Tensor, ab: int, scale_a: float, flags: int, w_packed: torch.Tensor, wb: int,
                               Ng: int, alpha: float, out_host: torch.Tensor, x_dev: torch.Tensor,
-                              planes_dev: torch.Tensor, out_dev: torch.Tensor, rows_per_chunk: int, streams) -> torch.Tensor:
+                              planes_dev: torch.Tensor, out_dev: torch.Tensor, rows_per_chunk: int, streams,
+                              join: bool = True) -> torch.Tensor:
     """Row-chunked FC layer from pinned host memory over several torch streams.  The streams are made to wait
-    for the current stream first, and the current stream waits for all of them afterwards."""
+    for the current stream first, and (join=True) the current stream waits for all of them afterwards.  With
+    join=False consecutive calls on the same streams pipeline into each other (chunk i of the next call follows
+    chunk i of this one on its stream); the caller joins the streams before reading out_host."""
     Mg, Kg = x_host.shape
     cur = torch.cuda.current_stream()
     for s in streams:
@@ -398,8 +401,9 @@ def fc_forward_host_pipelined(x_host: torch.Tensor, ab: int, scale_a: float, fla
     _check(lib.qnn_fc_forward_host_pipelined(_ptr(x_host), Mg, Kg, ab, float(scale_a), flags, _ptr(w_packed), wb, Ng,
                                              float(alpha), _ptr(out_host), _ptr(x_dev), _ptr(planes_dev), _ptr(out_dev),
                                              rows_per_chunk, arr, len(streams)), "qnn_fc_forward_host_pipelined")
-    for s in streams:
-        cur.wait_stream(s)
+    if join:
+        for s in streams:
+            cur.wait_stream(s)
     return out_host
 
 
