@@ -249,6 +249,8 @@ int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_planes, size_t 
  *   workspace device scratch owned by the caller, 256-byte aligned, at least qnn_bconv2d_backward_*_workspace(...)
  *             bytes (0 from the query = geometry out of range: N*Ho*Wo, R*S*C and Cout at most 65535*32,
  *             R*S*ceil(C/32) at most 65535).
+ * The weight gradients (convolution and fully-connected) split a long contraction over the thread blocks when the result
+ * has few tiles and add the partial products in a fixed order: results repeat bit for bit from call to call.
  * Errors as for qnn_bgemm_backward_*; waits are bounded and reported by qnn_tensor_path_status.
  */
 size_t qnn_bconv2d_backward_data_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad);

@@ -282,7 +282,7 @@ extern "C" int qnn_bgemm_backward_data(const float *g, const uint32_t *w_planes,
 
 extern "C" size_t qnn_bgemm_backward_weights_workspace(size_t m, size_t n, size_t k) {
     if (!backward_dims_ok(m, n, k)) return 0;
-    return (n + k) * (size_t)pad32((long long)m) * sizeof(float);
+    return (n + k) * (size_t)pad32((long long)m) * sizeof(float) + gemm_split_workspace((long long)n, (long long)k, (long long)m);
 }
 
 extern "C" int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_planes, size_t m, size_t n, size_t k, int ab,
@@ -306,7 +306,8 @@ extern "C" int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_plan
     p.alpha = alpha;
     p.C = gw; p.ldc = (long long)k;
     if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
-    return run_gemm<TC_TF32>(gt, ldm, aqt, ldm, p, st);
+    // a small n x k result against a long batch: the contraction over the batch is split over the CTAs
+    return run_gemm_tf32_split(gt, ldm, aqt, ldm, p, aqt + (size_t)k * ldm, st);
 }
 
 
@@ -388,7 +389,7 @@ extern "C" size_t qnn_bconv2d_backward_weights_workspace(int N, int H, int W, in
     ConvGeom g;
     if (!conv_geom(N, H, W, C, Cout, R, S, stride, pad, &g) || !conv_backward_dims_ok(g)) return 0;
     const size_t ldm = (size_t)pad32(g.Mg);
-    return round256((size_t)Cout * ldm * 4) + round256((size_t)g.Kg * ldm * 4);
+    return round256((size_t)Cout * ldm * 4) + round256((size_t)g.Kg * ldm * 4) + round256(gemm_split_workspace(Cout, g.Kg, g.Mg));
 }
 
 extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_planes, int ab, int N, int H, int W, int C,
@@ -424,7 +425,9 @@ extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_pl
     p.alpha = alpha;
     p.C = gw; p.ldc = cg.Kg;
     if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
-    return run_gemm<TC_TF32>(gt, ldm, colt, ldm, p, st);
+    // few output tiles (Cout x R*S*C) against a contraction over every output pixel: split it over the CTAs
+    void *split_ws = reinterpret_cast<char *>(colt) + round256((size_t)cg.Kg * ldm * 4);
+    return run_gemm_tf32_split(gt, ldm, colt, ldm, p, split_ws, st);
 }
 
 extern "C" int qnn_tensor_path_status(unsigned int *status) {

@@ -142,6 +142,11 @@ struct GemmParams {
     MbitPlaneConsts enc;                // constants of Eq. 12 for `bits` planes
     int tiles_n, tiles;
     int whole_items, items;             // work items: tiles [0, whole_items) whole, the rest split into two halves along N
+    // Split contraction (ksplit > 1; for products with few output tiles and a long K): work item w = tile * ksplit + s
+    // contracts K blocks [s * kb_per_split, (s + 1) * kb_per_split) and writes alpha times its partial product to
+    // C + s * split_stride (dense partial buffers); sum_partials_kernel then adds the ksplit buffers in index order.
+    int ksplit, kb_per_split;
+    long long split_stride;
 };
 
 // One column of a 32 x 32 chunk (this lane's), rows_here rows: C = Eq. 12 applied to the staged products and x.
@@ -168,17 +173,24 @@ __device__ __forceinline__ void epilogue_encoder(float *cptr, long long ldc, con
 // CTAs) are split into two halves along N so that the round takes about half a tile's time instead of a whole one.
 struct WorkItem {
     int m0, n0, width;
+    int kb0, kb1, split;                // K blocks [kb0, kb1) of this item; index of its partial buffer
 };
 template <int BN>
-__device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p) {
+__device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p, int nkb) {
     int tile = w, off = 0, width = BN;
+    if (p.ksplit > 1) {
+        tile = w / p.ksplit;
+        const int sp = w - tile * p.ksplit;
+        const int kb0 = sp * p.kb_per_split;
+        return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN, BN, kb0, min(nkb, kb0 + p.kb_per_split), sp};
+    }
     if (w >= p.whole_items) {
         const int r = w - p.whole_items;
         tile = p.whole_items + (r >> 1);
         off = (r & 1) * (BN / 2);
         width = BN / 2;
     }
-    return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN + off, width};
+    return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN + off, width, 0, nkb, 0};
 }
 
 template <int BN, int STAGES>
@@ -235,9 +247,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         if (lane == 0) {
             long long it = 0;                                 // stage uses so far, over all tiles
             for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x) {
-                const WorkItem wi = work_item<BN>(w, p);
+                const WorkItem wi = work_item<BN>(w, p, nkb);
                 const bool whole = wi.width == BN;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                for (int kb = wi.kb0; kb < wi.kb1; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                     if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err)) break;
@@ -256,12 +268,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             long long it = 0;
             int local = 0;
             for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x, ++local) {
-                const uint32_t idesc = work_item<BN>(w, p).width == BN ? idesc_kmajor<BN, KIND>() : idesc_kmajor<BN / 2, KIND>();
+                const WorkItem wi = work_item<BN>(w, p, nkb);
+                const uint32_t idesc = wi.width == BN ? idesc_kmajor<BN, KIND>() : idesc_kmajor<BN / 2, KIND>();
                 const int buf = local & 1;
                 if (!mbar_wait(&acc_empty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag, 3, p.err)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                for (int kb = wi.kb0; kb < wi.kb1; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
                     if (!mbar_wait(&full[s], ph, abort_flag, 1, p.err)) break;
@@ -270,7 +283,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     const uint64_t b_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES + L::A_BYTES));
 #pragma unroll
                     for (int j = 0; j < BK_BYTES / MMA_K_BYTES; ++j)   // 32 bytes along K per step = 2 descriptor address units
-                        tc_mma<KIND>(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, (kb | j) != 0 ? 1u : 0u);
+                        tc_mma<KIND>(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, ((kb - wi.kb0) | j) != 0 ? 1u : 0u);
                     tc_commit(&empty[s]);
                 }
                 tc_commit(&acc_full[buf]);
@@ -281,7 +294,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         const int half = (warp - 2) >> 2;                  // which of the two warps of this quarter
         int local = 0;
         for (int w = blockIdx.x; w < p.items; w += gridDim.x, ++local) {
-            const WorkItem wi = work_item<BN>(w, p);
+            const WorkItem wi = work_item<BN>(w, p, nkb);
             const int m0 = wi.m0, n0 = wi.n0;
             const int buf = local & 1;
             if (!mbar_wait(&acc_full[buf], (uint32_t)(local >> 1) & 1u, abort_flag, 2, p.err)) break;
@@ -315,7 +328,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     for (int i = 0; i < 32; ++i) stage[lane * 33 + i] = __fmul_rn(__uint_as_float(v[i]), p.alpha);
                     __syncwarp();
                     if (col < p.N) {
-                        float *cptr = p.C + (long long)(m0 + q * 32) * p.ldc + col;
+                        float *cptr = p.C + (long long)wi.split * p.split_stride + (long long)(m0 + q * 32) * p.ldc + col;
                         if (p.x) {
                             const float *xptr = p.x + (long long)(m0 + q * 32) * p.ldx + col;
                             switch (p.bits) {
@@ -407,11 +420,18 @@ int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtens
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return QNN_E_ARG;
     p.tiles_n = (int)tiles_n;
     p.tiles = (int)(tiles_m * tiles_n);
-    const int grid = p.tiles < sms ? p.tiles : sms;
-    const int rem = p.tiles % grid;
-    const bool split = rem > 0 && 2 * rem <= grid;
-    p.whole_items = split ? p.tiles - rem : p.tiles;
-    p.items = split ? p.tiles + rem : p.tiles;
+    int grid = p.tiles < sms ? p.tiles : sms;
+    if (p.ksplit > 1) {
+        if ((long long)p.tiles * p.ksplit > 0x7FFFFFFFll) return QNN_E_ARG;
+        p.whole_items = p.items = p.tiles * p.ksplit;
+        grid = p.items < sms ? p.items : sms;
+    } else {
+        p.ksplit = 1;
+        const int rem = p.tiles % grid;
+        const bool split = rem > 0 && 2 * rem <= grid;
+        p.whole_items = split ? p.tiles - rem : p.tiles;
+        p.items = split ? p.tiles + rem : p.tiles;
+    }
     tc_gemm_kernel<BN, STAGES, KIND><<<grid, GEMM_THREADS, L::TOTAL, st>>>(map_a, map_b, map_b_half, p);
     return qnn_launch_status();
 }
@@ -443,6 +463,57 @@ int run_gemm(const void *A, long long lda, const void *B, long long ldb, GemmPar
         return QNN_E_CUDA;
     return wide ? launch_gemm<256, 4, KIND>(map_a, map_b, map_b_half, p, sms, st)
                 : launch_gemm<128, 6, KIND>(map_a, map_b, map_b_half, p, sms, st);
+}
+
+// C[i][j] = sum over s (in increasing order: a fixed summation order) of part[s][i][j]; dense partial buffers [M][N].
+__global__ void __launch_bounds__(256) sum_partials_kernel(const float *__restrict__ part, int ksplit, long long stride,
+                                                          long long M, long long N, float *__restrict__ C, long long ldc) {
+    const long long total = M * N;
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+        float sum = part[i];
+        for (int sp = 1; sp < ksplit; ++sp) sum = __fadd_rn(sum, part[(long long)sp * stride + i]);
+        C[(i / N) * ldc + i % N] = sum;
+    }
+}
+
+// How many ways to split the contraction of an M x N x K TF32 product so that about two work items per SM exist
+// (sized for 148 SMs, independent of the device so that workspace queries and calls agree): 1 when the output
+// already has that many 128 x 128 tiles or K is short.  Every split gets at least four 32-element K blocks.
+int gemm_ksplit(long long M, long long N, long long K, int *kb_per_split) {
+    const long long tiles = ((M + BM - 1) / BM) * ((N + 127) / 128);
+    const long long nkb = (K + 31) / 32;
+    long long want = (2 * 148) / tiles;
+    if (want > nkb / 4) want = nkb / 4;
+    if (want > 64) want = 64;
+    if (want < 2) { *kb_per_split = (int)nkb; return 1; }
+    const long long per = (nkb + want - 1) / want;
+    *kb_per_split = (int)per;
+    return (int)((nkb + per - 1) / per);                  // every split non-empty
+}
+size_t gemm_split_workspace(long long M, long long N, long long K) {
+    int per;
+    const int ks = gemm_ksplit(M, N, K, &per);
+    return ks > 1 ? (size_t)ks * (size_t)M * (size_t)N * sizeof(float) : 0;
+}
+
+// run_gemm<TC_TF32> with the contraction split over CTAs when the output has few tiles; split_ws holds the partial
+// products (gemm_split_workspace bytes, 16-byte aligned).  No fused encoder epilogue in this form.  Only 128 x 128
+// tiles occur here: a split is planned only when the output has fewer tiles than the wide form needs.
+int run_gemm_tf32_split(const void *A, long long lda, const void *B, long long ldb, GemmParams p, void *split_ws,
+                        cudaStream_t st) {
+    int per;
+    const int ks = gemm_ksplit(p.M, p.N, p.K, &per);
+    if (ks <= 1 || p.x) return run_gemm<TC_TF32>(A, lda, B, ldb, p, st);
+    float *C = p.C;
+    const long long ldc = p.ldc;
+    p.ksplit = ks; p.kb_per_split = per;
+    p.C = static_cast<float *>(split_ws); p.ldc = p.N; p.split_stride = (long long)p.M * p.N;
+    const int rc = run_gemm<TC_TF32>(A, lda, B, ldb, p, st);
+    if (rc != QNN_OK) return rc;
+    const long long total = (long long)p.M * p.N;
+    const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+    sum_partials_kernel<<<blocks, 256, 0, st>>>(p.C, ks, p.split_stride, p.M, p.N, C, ldc);
+    return qnn_launch_status();
 }
 
 }  // namespace

@@ -72,6 +72,27 @@ def test_conv_backward_weights_exact_on_integer_gradients(geom, ab):
     assert np.array_equal(got.astype(np.float64), want)
 
 
+def test_conv_backward_weights_split_contraction_is_exact_and_repeatable():
+    """Few output tiles against thousands of output pixels: the contraction is split over many CTAs and the partial
+    products are summed in a fixed order, so integer gradients stay exact and two calls agree bit for bit."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    geom, ab = (8, 28, 28, 32, 16, 3, 3, 1, 1), 2
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(77, geom, ab, 1, True)
+    want = oracle.conv_backward_weights(g, qa, (R, S), stride, pad, ab, 1, 0.25)[0]
+    planes = torch.from_numpy(oracle.pack_planes(qa.reshape(-1, C), ab).view(np.int32)).to(dev)
+    gd = torch.from_numpy(g).to(dev)
+    got = qnn.bconv2d_backward_weights(gd, planes, ab, H, W, C, R, S, stride, pad, 0.25).cpu().numpy()
+    assert qnn.tensor_path_status() == 0
+    assert np.array_equal(got.astype(np.float64), want)
+    gr = torch.from_numpy(np.random.default_rng(1).standard_normal(g.shape).astype(np.float32)).to(dev)
+    a1 = qnn.bconv2d_backward_weights(gr, planes, ab, H, W, C, R, S, stride, pad, 0.37).cpu().numpy()
+    a2 = qnn.bconv2d_backward_weights(gr, planes, ab, H, W, C, R, S, stride, pad, 0.37).cpu().numpy()
+    assert np.array_equal(a1, a2)
+
+
 @pytest.mark.parametrize("geom,ab,wb", [((2, 14, 14, 64, 48, 3, 3, 1, 1), 2, 2), ((4, 16, 16, 32, 64, 3, 3, 2, 1), 3, 4),
                                         ((1, 10, 9, 100, 36, 1, 1, 1, 0), 8, 8)])
 def test_conv_backward_within_tf32_bound(geom, ab, wb):
