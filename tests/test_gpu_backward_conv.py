@@ -124,6 +124,28 @@ def test_conv_backward_within_tf32_bound(geom, ab, wb):
     assert np.sqrt(np.mean((GW - gw[0]) ** 2)) <= 0.1 * np.sqrt(np.mean(bw ** 2))
 
 
+def test_conv_backward_config2_layer_exact():
+    """The 3x3, 256 -> 256 channel layer of the single-convolution configuration at 14 x 14 (batch 8 of its 32, which
+    the oracle finishes in seconds): many tiles, a ragged last one, 2304-long patches, a split weight contraction."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    geom, ab, wb = (8, 14, 14, 256, 256, 3, 3, 1, 1), 2, 2
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(2, geom, ab, wb, True)
+    gd = torch.from_numpy(g).to(dev)
+    G = qnn.bconv2d_backward_data(gd, _packed_weights_dev(qw, wb, dev), wb, H, W, C, R, S, stride, pad, 0.125).cpu().numpy()
+    planes = torch.from_numpy(oracle.pack_planes(qa.reshape(-1, C), ab).view(np.int32)).to(dev)
+    GW = qnn.bconv2d_backward_weights(gd, planes, ab, H, W, C, R, S, stride, pad, 0.125).cpu().numpy()
+    assert qnn.tensor_path_status() == 0
+    ga = oracle.conv_backward_data(g, qw, (H, W), stride, pad, ab, wb, 0.125)
+    gw = oracle.conv_backward_weights(g, qa, (R, S), stride, pad, ab, wb, 0.125)
+    for p in range(ab):          # g_{a^p} = 2^(p-1) * G, exactly (integer gradients, sums far below 2^24)
+        assert np.array_equal(2.0 ** p * G.astype(np.float64), ga[p])
+    for j in range(wb):
+        assert np.array_equal(2.0 ** j * GW.astype(np.float64), gw[j])
+
+
 def test_conv_backward_data_through_the_encoder():
     """With x given the gather applies Eq. 12 to gc_p = 2^(p-1) * G: compared with the oracle's two steps chained."""
     import torch
