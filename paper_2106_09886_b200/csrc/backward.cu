@@ -173,31 +173,51 @@ __global__ void __launch_bounds__(256) conv_weights_t_kernel(const uint32_t *__r
 // (ho, wo) with ho*st - pad + r = h and wo*st - pad + s = w of dcol[(n, ho, wo)][(r*S + s)*C + c], taps in
 // increasing (r, s) order (a gather, so the sum has a fixed order).  BITS > 0: the encoder derivative of Eq. 12 is
 // applied to the sum (x = what the previous layer fed its encoder, as in qnn_bgemm_backward_data).
-template <int BITS>
+// One thread per pixel and VEC consecutive channels (VEC = 4 when C is a multiple of 4: 16-byte accesses, a quarter of
+// the index arithmetic); the tap loops run in 32-bit arithmetic, only the row offset into dcol is 64-bit.
+template <int BITS, int VEC>
 __global__ void __launch_bounds__(256) conv_col2im_kernel(const float *__restrict__ dcol, ConvGeom g, const float *__restrict__ x,
                                                          float r_range, MbitPlaneConsts enc, float *__restrict__ out) {
-    const long long total = (long long)g.N * g.H * g.W * g.C;
+    const int cv = g.C / VEC;                                          // channel groups per pixel
+    const long long total = (long long)g.N * g.H * g.W * cv;
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
-        const int c = (int)(i % g.C);
-        const long long pix = i / g.C;
-        const int w = (int)(pix % g.W), h = (int)((pix / g.W) % g.H);
-        const long long n = pix / ((long long)g.W * g.H);
-        float sum = 0.0f;
+        const long long pix = i / cv;
+        const int c = (int)(i - pix * cv) * VEC;
+        const long long nh = pix / g.W;
+        const int w = (int)(pix - nh * g.W);
+        const long long n = nh / g.H;
+        const int h = (int)(nh - n * g.H);
+        float sum[VEC];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) sum[v] = 0.0f;
         for (int r = 0; r < g.R; ++r) {
             const int th = h + g.pad - r;
-            if (th < 0 || th % g.stride) continue;
+            if (th < 0) break;                                         // larger r only moves further up
             const int ho = th / g.stride;
-            if (ho >= g.Ho) continue;
+            if (ho * g.stride != th || ho >= g.Ho) continue;
+            const long long rowbase = (n * g.Ho + ho) * g.Wo;
             for (int sx = 0; sx < g.S; ++sx) {
                 const int tw = w + g.pad - sx;
-                if (tw < 0 || tw % g.stride) continue;
+                if (tw < 0) break;
                 const int wo = tw / g.stride;
-                if (wo >= g.Wo) continue;
-                sum = __fadd_rn(sum, __ldg(dcol + ((n * g.Ho + ho) * g.Wo + wo) * g.Kg + (long long)(r * g.S + sx) * g.C + c));
+                if (wo * g.stride != tw || wo >= g.Wo) continue;
+                const float *src = dcol + (rowbase + wo) * g.Kg + (r * g.S + sx) * g.C + c;
+                if (VEC == 4) {
+                    const float4 d = __ldcs(reinterpret_cast<const float4 *>(src));
+                    sum[0] = __fadd_rn(sum[0], d.x); sum[1 % VEC] = __fadd_rn(sum[1 % VEC], d.y);
+                    sum[2 % VEC] = __fadd_rn(sum[2 % VEC], d.z); sum[3 % VEC] = __fadd_rn(sum[3 % VEC], d.w);
+                } else {
+                    sum[0] = __fadd_rn(sum[0], __ldcs(src));
+                }
             }
         }
-        if constexpr (BITS > 0) sum = mbit_backward_shared<BITS>(__ldg(x + i), r_range, sum, enc);
-        out[i] = sum;
+        const long long o = pix * g.C + c;
+        if constexpr (BITS > 0) {
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) sum[v] = mbit_backward_shared<BITS>(__ldg(x + o + v), r_range, sum[v], enc);
+        }
+        if (VEC == 4) *reinterpret_cast<float4 *>(out + o) = make_float4(sum[0], sum[1 % VEC], sum[2 % VEC], sum[3 % VEC]);
+        else out[o] = sum[0];
     }
 }
 
@@ -371,14 +391,20 @@ extern "C" int qnn_bconv2d_backward_data(const float *g, const void *w_packed, i
     p.C = dcol; p.ldc = cg.Kg;
     if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
     if ((rc = run_gemm<TC_TF32>(a, lda, wqt, ldn, p, st)) != QNN_OK) return rc;
-    const long long total = (long long)N * H * W * C;
-    const int blocks = (int)(qnn_ceil_div(total, 256) < 148 * 16 ? qnn_ceil_div(total, 256) : 148 * 16);
+    // 16-byte accesses need C % 4 == 0 (then every patch row, R*S*C floats, and every pixel start on 16-byte
+    // boundaries of the 256-byte aligned workspace) and a 16-byte aligned output
+    const bool vec4 = C % 4 == 0 && qnn_aligned(out, 16);
+    const long long total = (long long)N * H * W * (vec4 ? C / 4 : C);
+    const int blocks = (int)(qnn_ceil_div(total, 256) < 148 * 64 ? qnn_ceil_div(total, 256) : 148 * 64);
     MbitPlaneConsts enc = x ? mbit_plane_consts(ab) : MbitPlaneConsts{};
-#define CONV_C2I_CASE(B) case B: conv_col2im_kernel<B><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out); break;
+#define CONV_C2I_CASE(B)                                                                          \
+    case B:                                                                                       \
+        if (vec4) conv_col2im_kernel<B, 4><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out);     \
+        else conv_col2im_kernel<B, 1><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out);          \
+        break;
     switch (x ? ab : 0) {
         CONV_C2I_CASE(0) CONV_C2I_CASE(1) CONV_C2I_CASE(2) CONV_C2I_CASE(3) CONV_C2I_CASE(4) CONV_C2I_CASE(5) CONV_C2I_CASE(6)
-        CONV_C2I_CASE(7)
-        default: conv_col2im_kernel<8><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out); break;
+        CONV_C2I_CASE(7) CONV_C2I_CASE(8)
     }
 #undef CONV_C2I_CASE
     return qnn_launch_status();
