@@ -194,26 +194,32 @@ encode_pack_lanes_kernel(const float *__restrict__ x, int64_t rows, int k, int64
     constexpr int S = 1 << LOG2S, R = 32 >> LOG2S;
     const int64_t nwarps = (int64_t)gridDim.x * (kEncThreads / 32);
     const int ca = lane >> 3, cc = lane & 7;                 // load role: word ca + 4j of the unit, 16-byte piece cc
-    // Piece j of this lane is word ca + 4j of the unit: row j / (S/4) of the unit, and within that row's segment
-    // element 128*(j % (S/4)) + 4*lane.  With S fixed at compile time every piece is a constant offset from one base.
-    constexpr int JPR = S / 4;                               // pieces per lane and row
+    // Piece j of this lane is word ca + 4j of the unit.  S >= 4: row j / (S/4) of the unit, and within that row's
+    // segment element 128*(j % (S/4)) + 4*lane.  S < 4 (rows of at most 64 elements): row (ca >> LOG2S) + (4/S)*j,
+    // element 32*(ca % S) + 4*cc.  With S fixed at compile time every piece is a constant offset from one base.
+    constexpr int JPR = S >= 4 ? S / 4 : 1;                  // pieces per lane and row (S >= 4)
+    constexpr int RSTEP = S >= 4 ? 0 : 4 / S;                // rows between consecutive pieces of a lane (S < 4)
+    const int row0 = S >= 4 ? 0 : (ca >> LOG2S);             // row of piece 0 within the unit
+    const int el0 = S >= 4 ? 4 * lane : 32 * (ca & (S - 1)) + 4 * cc;   // element of piece 0 within the segment
 
     for (int64_t u = (int64_t)blockIdx.x * (kEncThreads / 32) + warp; u < n_units; u += nwarps) {
         const int64_t rg = u / segs;                         // warp-uniform
         const int seg = (int)(u - rg * segs);
-        const float *xl = x + rg * R * ldx + (int64_t)seg * S * 32 + 4 * lane;
+        const float *xl = x + (rg * R + row0) * ldx + (int64_t)seg * S * 32 + el0;
         const int64_t rows_left = rows - rg * R;
         const int k_left = k - seg * S * 32;                 // elements of the row from this segment on (may be <= 0)
         float4 f[8];
         if (rows_left >= R && k_left >= S * 32) {            // the whole unit is inside the tensor
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                f[j] = __ldcs(reinterpret_cast<const float4 *>(xl + (int64_t)(j / JPR) * ldx + 128 * (j % JPR)));
+                f[j] = __ldcs(reinterpret_cast<const float4 *>(xl + (int64_t)(S >= 4 ? j / JPR : RSTEP * j) * ldx +
+                                                               (S >= 4 ? 128 * (j % JPR) : 0)));
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int r = j / JPR, e = 128 * (j % JPR) + 4 * lane;
-                const float *src = xl + (int64_t)r * ldx + 128 * (j % JPR);
+                const int dr = S >= 4 ? j / JPR : RSTEP * j, de = S >= 4 ? 128 * (j % JPR) : 0;
+                const int r = row0 + dr, e = el0 + de;
+                const float *src = xl + (int64_t)dr * ldx + de;
                 f[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 if (r < rows_left) {
                     if (e + 4 <= k_left) {
@@ -258,6 +264,16 @@ encode_pack_lanes_kernel(const float *__restrict__ x, int64_t rows, int k, int64
             uint32_t *dst = planes + (row * BITS) * (int64_t)kw + w;
 #pragma unroll
             for (int i = 0; i < BITS; ++i) dst[(int64_t)i * kw] = word[i] & mask;
+            if constexpr (S < 4) {
+                // rows of one or two words: the row's storage is four words, the lane of word 0 clears the rest
+                if (w == 0) {
+#pragma unroll
+                    for (int i = 0; i < BITS; ++i) {
+                        if (S == 1) dst[(int64_t)i * kw + 1] = 0u;
+                        *reinterpret_cast<uint2 *>(dst + (int64_t)i * kw + 2) = make_uint2(0u, 0u);
+                    }
+                }
+            }
             if (rowsum != nullptr && len > 0) {
                 int sum = 0;
 #pragma unroll
@@ -393,9 +409,12 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
     const int kw = (int)qnn_row_words_i(k);
     if (qnn_aligned(x, 16) && ldx % 4 == 0) {
         // per-lane packing kernel; the ballot kernels below remain for unaligned inputs
-        int log2s = 2;
-        while ((1 << log2s) < kw && log2s < 5) ++log2s;
-        const int segs_l = (kw + (1 << log2s) - 1) >> log2s;
+        // S = 2^log2s words per row segment: the real words of the row when they are at most 32 (rows of one or two
+        // words get S = 1 or 2; their padding words are cleared by the lane of word 0), else 32 with several segments
+        const int cw_real = (k + 31) / 32;
+        int log2s = 0;
+        while ((1 << log2s) < cw_real && log2s < 5) ++log2s;
+        const int segs_l = log2s < 2 ? 1 : (kw + (1 << log2s) - 1) >> log2s;
         const int rpu_l = 32 >> log2s;
         const int64_t n_units = qnn_ceil_div(rows, rpu_l) * segs_l;
         int dev = 0, sms = 148;
@@ -405,6 +424,8 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
 #define QNN_ENC_LANES(L_) \
     encode_pack_lanes_kernel<BITS, L_><<<(int)blocks, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, hi, planes, rowsum, kw, segs_l, n_units)
         switch (log2s) {
+            case 0: QNN_ENC_LANES(0); break;
+            case 1: QNN_ENC_LANES(1); break;
             case 2: QNN_ENC_LANES(2); break;
             case 3: QNN_ENC_LANES(3); break;
             case 4: QNN_ENC_LANES(4); break;
