@@ -169,6 +169,43 @@ def test_conv_backward_data_through_the_encoder():
     assert np.all(got[np.abs(x) > r] == 0.0)
 
 
+@pytest.mark.parametrize("geom", [(2, 14, 14, 128, 32, 3, 3, 1, 1), (1, 5, 4, 70, 130, 3, 2, 1, 0), (8, 28, 28, 32, 16, 3, 3, 1, 1)])
+def test_conv_backward_stays_inside_its_buffers(geom):
+    """Outputs and the workspace (exactly the size the query returns) sit between sentinel regions; nothing outside them
+    may change, whichever staging path (padded copy of g, split contraction) the geometry takes."""
+    import torch
+    from paper_2106_09886_b200 import qnn
+    dev = torch.device("cuda:0")
+    N, H, W, C, Cout, R, S, stride, pad = geom
+    qa, qw, g = _case(5, geom, 2, 2, True)
+    gd = torch.from_numpy(g).to(dev)
+    planes = torch.from_numpy(oracle.pack_planes(qa.reshape(-1, C), 2).view(np.int32)).to(dev)
+    blob = _packed_weights_dev(qw, 2, dev)
+    G = 4096                                                   # guard bytes on each side (keeps 256-byte alignment)
+
+    def guarded(nbytes):
+        buf = torch.full((G + nbytes + G,), 0xA5, dtype=torch.uint8, device=dev)
+        return buf, buf[G:G + nbytes]
+
+    def intact(buf, nbytes):
+        return bool((buf[:G] == 0xA5).all()) and bool((buf[G + nbytes:] == 0xA5).all())
+
+    nd = qnn.lib.qnn_bconv2d_backward_data_workspace(N, H, W, C, Cout, R, S, stride, pad)
+    nw = qnn.lib.qnn_bconv2d_backward_weights_workspace(N, H, W, C, Cout, R, S, stride, pad)
+    wsd_buf, wsd = guarded(nd)
+    wsw_buf, wsw = guarded(nw)
+    out_buf, out_b = guarded(N * H * W * C * 4)
+    gw_buf, gw_b = guarded(Cout * R * S * C * 4)
+    out = out_b.view(torch.float32).view(N, H, W, C)
+    gw = gw_b.view(torch.float32).view(Cout, R, S, C)
+    qnn.bconv2d_backward_data(gd, blob, 2, H, W, C, R, S, stride, pad, 0.25, out=out, workspace=wsd)
+    qnn.bconv2d_backward_weights(gd, planes, 2, H, W, C, R, S, stride, pad, 0.25, gw=gw, workspace=wsw)
+    assert qnn.tensor_path_status() == 0
+    assert intact(wsd_buf, nd) and intact(wsw_buf, nw) and intact(out_buf, out_b.numel()) and intact(gw_buf, gw_b.numel())
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), oracle.conv_backward_data(g, qw, (H, W), stride, pad, 1, 2, 0.25)[0])
+    assert np.array_equal(gw.cpu().numpy().astype(np.float64), oracle.conv_backward_weights(g, qa, (R, S), stride, pad, 2, 1, 0.25)[0])
+
+
 def test_conv_backward_rejects_bad_arguments():
     import torch
     from paper_2106_09886_b200 import qnn
