@@ -6,7 +6,8 @@
 //
 // Mapping: lane <-> output feature (32 consecutive features per pass), so every store is one coalesced
 // 128-byte row segment; a warp takes 32 output pixels at a time, lane L assembles pixel L's ab patch words,
-// and the pixels' words are then handed round with shuffles.  Per output: ab*wb (xor, popc, multiply-add).
+// and the pixels' words are then handed round with shuffles.  Per output: ab*wb xors and as many popcounts, fewer for
+// 4 x 4 and 3 x 3 bits (dense_weighted_count).
 // Taps outside the image are left as zero bits and corrected with tapsum exactly as in the tiled kernel.
 #pragma once
 #include "qnn_internal.cuh"
@@ -28,6 +29,53 @@ struct Params {
     int32_t *acc;
     int H, W, C, R, S, stride, pad, Ho, Wo;
 };
+
+
+// sum_ij 2^(i+j) popc(a_i xor w_j) for single-word operands.  The popcount pipe is the binding unit of this kernel
+// (one popcount per plane pair and output), so for the widest cases the ab*wb xor words are first compressed across
+// PAIRS: words of equal weight 2^(i+j) go through full adders on bit columns (sum keeps the weight, carry doubles it),
+// 16 words -> 10 for 4 x 4 bits and 9 -> 7 for 3 x 3 bits, at two three-input logic operations per adder.
+__device__ __forceinline__ void dense_fa(uint32_t a, uint32_t b, uint32_t c, uint32_t &sum, uint32_t &carry) {
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(sum) : "r"(a), "r"(b), "r"(c));
+    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(carry) : "r"(a), "r"(b), "r"(c));
+}
+template <int AB, int WB>
+__device__ __forceinline__ int dense_weighted_count(const uint32_t (&a)[AB], const uint32_t (&w)[WB]) {
+    if constexpr (AB == 4 && WB == 4) {
+        uint32_t x[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[i][j] = a[i] ^ w[j];
+        uint32_t s2, c2, s3a, c3a, s3, c3b, s4a, c4a, s4, c4b, s5, c5;
+        dense_fa(x[0][2], x[1][1], x[2][0], s2, c2);          // weight 4 -> 4 + 8
+        dense_fa(x[0][3], x[1][2], x[2][1], s3a, c3a);        // weight 8 -> 8 + 16
+        dense_fa(x[3][0], c2, s3a, s3, c3b);
+        dense_fa(x[1][3], x[2][2], x[3][1], s4a, c4a);        // weight 16 -> 16 + 32
+        dense_fa(c3a, c3b, s4a, s4, c4b);
+        dense_fa(x[2][3], x[3][2], c4a, s5, c5);              // weight 32 -> 32 + 64
+        return __popc(x[0][0]) + 2 * (__popc(x[0][1]) + __popc(x[1][0])) + 4 * __popc(s2) + 8 * __popc(s3) +
+               16 * __popc(s4) + 32 * (__popc(s5) + __popc(c4b)) + 64 * (__popc(x[3][3]) + __popc(c5));
+    } else if constexpr (AB == 3 && WB == 3) {
+        uint32_t x[3][3];
+#pragma unroll
+        for (int i = 0; i < 3; ++i)
+#pragma unroll
+            for (int j = 0; j < 3; ++j) x[i][j] = a[i] ^ w[j];
+        uint32_t s2, c2, s3, c3;
+        dense_fa(x[0][2], x[1][1], x[2][0], s2, c2);          // weight 4 -> 4 + 8
+        dense_fa(x[1][2], x[2][1], c2, s3, c3);               // weight 8 -> 8 + 16
+        return __popc(x[0][0]) + 2 * (__popc(x[0][1]) + __popc(x[1][0])) + 4 * __popc(s2) + 8 * __popc(s3) +
+               16 * (__popc(x[2][2]) + __popc(c3));
+    } else {
+        int s = 0;
+#pragma unroll
+        for (int i = 0; i < AB; ++i)
+#pragma unroll
+            for (int j = 0; j < WB; ++j) s += __popc(a[i] ^ w[j]) * (1 << (i + j));
+        return s;
+    }
+}
 
 template <int AB, int WB>
 __global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) {
@@ -91,13 +139,10 @@ __global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) 
             const float gam = affine ? __ldg(p.ch_gamma + n) : 1.0f;
             const float bet = (affine && p.ch_beta) ? __ldg(p.ch_beta + n) : 0.0f;
             for (int rr = 0; rr < rows_here; ++rr) {
-                int s_acc = 0;
+                uint32_t arow[AB];
 #pragma unroll
-                for (int i = 0; i < AB; ++i) {
-                    const uint32_t ai = __shfl_sync(0xffffffffu, mine[i], rr);
-#pragma unroll
-                    for (int j = 0; j < WB; ++j) s_acc += __popc(ai ^ wreg[j]) * (1 << (i + j));
-                }
+                for (int i = 0; i < AB; ++i) arow[i] = __shfl_sync(0xffffffffu, mine[i], rr);
+                const int s_acc = dense_weighted_count<AB, WB>(arow, wreg);
                 uint32_t inv = __shfl_sync(0xffffffffu, invalid, rr);
                 int n_valid = (taps - __popc(inv)) * p.C;
                 int corr = 0;
