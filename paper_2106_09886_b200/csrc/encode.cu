@@ -1,11 +1,12 @@
 // qnn_encode_pack, qnn_pack_weights, qnn_absmax_f32: real tensors -> bit planes.
 //
-// Activations (qnn_encode_pack) take one of two kernels:
+// Activations (qnn_encode_pack) take one of three kernels:
 //  * encode_pack_lanes_kernel (source 16-byte aligned, ldx a multiple of 4: the usual case): a lane owns a
 //    whole output word, i.e. 32 consecutive elements; see the comment above the kernel.
 //  * encode_pack_kernel (any alignment): a warp owns 128 consecutive elements of one row, lane L reads
 //    elements 32*j + L (four coalesced 128-byte requests) and one __ballot_sync per plane and j turns the
 //    warp's 32 decisions into one canonical word (lane L -> bit L); lane i stores plane i's four words.
+//  * encode_pack_tiny_kernel (rows of at most 8 elements, or at most 32 from an unaligned source): a thread owns a row.
 // The weight packer (offline) uses the ballot scheme as well.
 #include "qnn_internal.cuh"
 #include <string.h>
@@ -284,6 +285,35 @@ encode_pack_lanes_kernel(const float *__restrict__ x, int64_t rows, int k, int64
     }
 }
 
+// Rows of a few elements (a first layer's 3-channel pixels): one thread per row.  The thread reads its k <= 32 values,
+// builds the row's single word of every plane itself and stores it with the three padding words as one 16-byte
+// vector; consecutive threads hold consecutive rows, so a warp's stores fill whole lines.  Works for any alignment
+// of x and any ldx.  The work per element grows with bits (three logic operations per element and plane), which is
+// why longer rows take the kernels above; here the stores (16 bytes per row and plane) dominate.
+template <int BITS>
+__global__ void __launch_bounds__(kEncThreads)
+encode_pack_tiny_kernel(const float *__restrict__ x, int64_t rows, int k, int64_t ldx, float inv2s, float lo, float hi,
+                        uint32_t *__restrict__ planes, int32_t *__restrict__ rowsum) {
+    const float half = (float)(1 << (BITS - 1));
+    for (int64_t row = (int64_t)blockIdx.x * kEncThreads + threadIdx.x; row < rows; row += (int64_t)gridDim.x * kEncThreads) {
+        const float *src = x + row * ldx;
+        uint32_t word[BITS];
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) word[i] = 0u;
+        int sum = 0;
+        for (int c = 0; c < k; ++c) {
+            const uint32_t t = qnn_code_bits(__ldg(src + c), inv2s, half, lo, hi) & 0xffu;
+            sum += (int)t;
+#pragma unroll
+            for (int i = 0; i < BITS; ++i) word[i] |= ((t >> i) & 1u) << c;
+        }
+        uint4 *dst = reinterpret_cast<uint4 *>(planes + row * BITS * 4);
+#pragma unroll
+        for (int i = 0; i < BITS; ++i) dst[i] = make_uint4(word[i], 0u, 0u, 0u);
+        if (rowsum != nullptr) rowsum[row] = sum;
+    }
+}
+
 // Offline weight packer: one warp per (output feature, group of 4 words).  A word
 // covers 32 input channels of one tap; the source index follows the layout flag.
 template <int BITS>
@@ -407,7 +437,15 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
     float lo, hi;
     qnn_clamp_bounds(BITS, scale, relu, &lo, &hi);
     const int kw = (int)qnn_row_words_i(k);
-    if (qnn_aligned(x, 16) && ldx % 4 == 0) {
+    const bool lanes_ok = qnn_aligned(x, 16) && ldx % 4 == 0;
+    if (k <= 8 || (k <= 32 && !lanes_ok)) {
+        // one thread per row (kw == 4: one real word and three padding words per plane)
+        int64_t blocks = qnn_ceil_div(rows, kEncThreads);
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        encode_pack_tiny_kernel<BITS><<<(int)blocks, kEncThreads, 0, st>>>(x, rows, k, ldx, inv2s, lo, hi, planes, rowsum);
+        return;
+    }
+    if (lanes_ok) {
         // per-lane packing kernel; the ballot kernels below remain for unaligned inputs
         // S = 2^log2s words per row segment: the real words of the row when they are at most 32 (rows of one or two
         // words get S = 1 or 2; their padding words are cleared by the lane of word 0), else 32 with several segments
