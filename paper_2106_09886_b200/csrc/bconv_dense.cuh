@@ -129,35 +129,51 @@ __global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) 
                 }
         }
         const int rows_here = (int)((p.Mg - batch * 32) < 32 ? (p.Mg - batch * 32) : 32);
-        for (int cb = 0; cb < ncb; ++cb) {
-            const int n = cb * 32 + lane;
-            const bool n_ok = n < p.Ng;
-            uint32_t wreg[WB];
+        // two blocks of 32 features per pass: the pixel's words, its border mask and the row bookkeeping are
+        // fetched once for both
+        for (int cb = 0; cb < ncb; cb += 2) {
+            const bool two = cb + 1 < ncb;                                // warp-uniform
+            int n[2];
+            bool n_ok[2], affine[2];
+            uint32_t wreg[2][WB];
+            float gam[2], bet[2];
 #pragma unroll
-            for (int j = 0; j < WB; ++j) wreg[j] = n_ok ? wd_s[j * p.Ng + n] : 0u;
-            const bool affine = p.ch_gamma != nullptr && n_ok;
-            const float gam = affine ? __ldg(p.ch_gamma + n) : 1.0f;
-            const float bet = (affine && p.ch_beta) ? __ldg(p.ch_beta + n) : 0.0f;
+            for (int h = 0; h < 2; ++h) {
+                n[h] = (cb + h) * 32 + lane;
+                n_ok[h] = n[h] < p.Ng;
+#pragma unroll
+                for (int j = 0; j < WB; ++j) wreg[h][j] = n_ok[h] ? wd_s[j * p.Ng + n[h]] : 0u;
+                affine[h] = p.ch_gamma != nullptr && n_ok[h];
+                gam[h] = affine[h] ? __ldg(p.ch_gamma + n[h]) : 1.0f;
+                bet[h] = (affine[h] && p.ch_beta) ? __ldg(p.ch_beta + n[h]) : 0.0f;
+            }
             for (int rr = 0; rr < rows_here; ++rr) {
                 uint32_t arow[AB];
 #pragma unroll
                 for (int i = 0; i < AB; ++i) arow[i] = __shfl_sync(0xffffffffu, mine[i], rr);
-                const int s_acc = dense_weighted_count<AB, WB>(arow, wreg);
+                int s_acc[2];
+                s_acc[0] = dense_weighted_count<AB, WB>(arow, wreg[0]);
+                s_acc[1] = two ? dense_weighted_count<AB, WB>(arow, wreg[1]) : 0;
                 uint32_t inv = __shfl_sync(0xffffffffu, invalid, rr);
-                int n_valid = (taps - __popc(inv)) * p.C;
-                int corr = 0;
+                const int n_valid = (taps - __popc(inv)) * p.C;
+                int corr[2] = {0, 0};
                 while (inv != 0u) {                                       // warp-uniform: the row is the same for all lanes
                     const int t = __ffs(inv) - 1;
                     inv &= inv - 1u;
-                    if (n_ok) corr += ts_s[t * p.Ng + n];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        if (n_ok[h]) corr[h] += ts_s[t * p.Ng + n[h]];
                 }
-                if (n_ok) {
-                    const int32_t v = n_valid * PROD - 2 * (s_acc - AMAX * corr);
-                    const int64_t o = (batch * 32 + rr) * (int64_t)p.Ng + n;
+                const int64_t o_row = (batch * 32 + rr) * (int64_t)p.Ng;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (!n_ok[h]) continue;
+                    const int32_t v = n_valid * PROD - 2 * (s_acc[h] - AMAX * corr[h]);
+                    const int64_t o = o_row + n[h];
                     if (p.acc) p.acc[o] = v;
                     if (p.out) {
                         float y = __fmul_rn(__int2float_rn(v), p.alpha);
-                        if (affine) y = __fmaf_rn(y, gam, bet);
+                        if (affine[h]) y = __fmaf_rn(y, gam[h], bet[h]);
                         p.out[o] = y;
                     }
                 }
