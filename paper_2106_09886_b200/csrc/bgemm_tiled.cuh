@@ -553,35 +553,43 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                 }
             }
             if (FUSED && p.next_planes != nullptr) {
-                // Next layer's encoder on the fp32 result (Alg. 1 forward: scale, then MBitEncoder).  A warp holds
-                // two output rows (lanes 0-15: row ty even, lanes 16-31: row ty odd) x 16 consecutive features
-                // per c, so one ballot per (plane, c) yields half a word for each of the two rows; c = 0,1 form
-                // word n0/32 and c = 2,3 word n0/32 + 1.  Every lane takes part in every ballot.
-                uint32_t t[4];
+                // Next layer's encoder on the fp32 result (Alg. 1 forward: scale, then MBitEncoder), first half: the
+                // codes of this thread's outputs go to the tile's code matrix in shared memory, one byte each
+                // (0 outside the problem, so that padding bits come out as 0).
+                uint8_t *codes = reinterpret_cast<uint8_t *>(smem + 2 * BUF_VEC);        // [kBM][64]
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int n = n0 + tx + 16 * c;
                     const uint32_t code = qnn_code_bits(fv[c], p.next_inv2s, p.next_half, p.next_lo, p.next_hi);
-                    t[c] = (row_ok && n < p.Ng) ? code : 0u;                // padding bits are 0
+                    codes[(ty + 16 * r) * kBN + tx + 16 * c] = (row_ok && n < p.Ng) ? (uint8_t)code : (uint8_t)0;
                 }
-                const int lane = tid & 31;
-                const uint32_t halfsel = lane >= 16 ? 0x7632u : 0x5410u;    // this lane's row: upper / lower ballot halves
-                const bool storer = (lane & 15) == 0 && row_ok;
-                const int word0 = n0 >> 5;
-                uint32_t *dst = p.next_planes + (m * p.next_bits) * (int64_t)p.next_kw + word0;
-                const bool last_tile_n = n0 + kBN >= p.Ng;
-                for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
-                    const uint32_t bit = 1u << i;
-                    const uint32_t b0 = __ballot_sync(0xffffffffu, t[0] & bit);
-                    const uint32_t b1 = __ballot_sync(0xffffffffu, t[1] & bit);
-                    const uint32_t b2 = __ballot_sync(0xffffffffu, t[2] & bit);
-                    const uint32_t b3 = __ballot_sync(0xffffffffu, t[3] & bit);
-                    if (storer) {
-                        *reinterpret_cast<uint2 *>(dst) = make_uint2(__byte_perm(b0, b1, halfsel), __byte_perm(b2, b3, halfsel));
-                        // the last feature tile also clears the padding words of the row
-                        if (last_tile_n)
-                            for (int wz = word0 + 2; wz < p.next_kw; wz += 2)
-                                *reinterpret_cast<uint2 *>(dst + (wz - word0)) = make_uint2(0u, 0u);
+            }
+        }
+        if (FUSED && p.next_planes != nullptr) {
+            // Second half: thread (row, w) owns word w (32 features) of tile row `row`: it reads the 32 code bytes and
+            // moves bit i of each byte into plane i's word four bytes at a time with one mask and one multiply
+            // (((c & (0x01010101 << i)) * (0x10204080 >> i)) >> 28 = the four bits; the partial products land on
+            // distinct bits), appended by a funnel shift.  Replaces one warp ballot per plane and 16 features.
+            __syncthreads();                       // the code matrix is complete (the next tile's stage barriers
+                                                   // order these reads before its epilogue writes)
+            if (tid < 2 * kBM) {
+                const int row = tid >> 1, wsel = tid & 1;
+                const int64_t m = m0 + row;
+                if (m < p.Mg) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(smem + 2 * BUF_VEC) + row * 4 + wsel * 2;
+                    const uint4 lo4 = src[0], hi4 = src[1];
+                    const uint32_t c4[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+                    const int word0 = (n0 >> 5) + wsel;
+                    uint32_t *dst = p.next_planes + (m * p.next_bits) * (int64_t)p.next_kw + word0;
+                    const bool clear_pad = wsel == 0 && n0 + kBN >= p.Ng;   // the last feature tile clears the row's padding words
+                    for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
+                        const uint32_t mask = 0x01010101u << i, mul = 0x10204080u >> i;
+                        uint32_t word = 0u;
+#pragma unroll
+                        for (int g = 7; g >= 0; --g) word = __funnelshift_l((c4[g] & mask) * mul, word, 4);
+                        if (word0 < p.next_kw) *dst = word;
+                        if (clear_pad)
+                            for (int wz = (n0 >> 5) + 2; wz < p.next_kw; ++wz) dst[wz - word0] = 0u;
                     }
                 }
             }
@@ -671,7 +679,7 @@ template <int AB, int WB, int CONV, int TM, bool FUSED>
 inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     constexpr int kBM = 16 * TM;
     constexpr size_t ext = (CONV == 3) ? ((size_t)kStageChunks * (AB * kBM + WB * kBN) + 3u) / 4u * 16u : 0u;   // ninth words
-    constexpr size_t smem = 2u * (kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u + ext);
+    constexpr size_t smem = 2u * (kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u + ext) + (FUSED ? (size_t)kBM * kBN : 0u);   // + the chaining epilogue's code matrix
     if (smem > 48u * 1024u &&
         cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV, TM, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
