@@ -48,7 +48,7 @@ __device__ __forceinline__ void enc_ballots_small(float x, const EncThresholds t
 
 // A unit is 128 consecutive elements: four ballots per plane give four canonical words.  For rows
 // longer than 64 elements a unit is a 128-element segment of one row (RPU = 1); for shorter rows
-// (NHWC activations with few channels) a unit spans RPU = 2 (k <= 64) or 4 (k <= 32) whole rows so
+// (33..64 elements, from an unaligned source) a unit spans RPU = 2 whole rows so
 // that the lanes stay busy.  UN units are loaded before the first ballot, so 4*UN independent
 // 128-byte requests per warp are in flight.  Unit indices advance incrementally (no division in the loop).
 // MODE 0: any width, codes from the quantizer's formula; MODE 1 / 2 (BITS <= 2, RPU = 1, no rowsum): codes from
@@ -475,7 +475,7 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
     const int segs = kw / 4;
     int groups;
     int64_t total;                                   // warp-level work items
-    const int rpu = (k <= 32) ? 4 : (k <= 64 ? 2 : 1);
+    const int rpu = (k <= 64) ? 2 : 1;               // (rows of at most 32 elements never get here: one thread per row above)
     if (rpu == 1) {
         groups = (int)qnn_ceil_div(segs, UN);
         total = rows * groups;
@@ -501,10 +501,8 @@ void launch_encode(const float *x, int64_t rows, int k, int64_t ldx, float scale
             }
         }
         if (k % 128 == 0) QNN_ENC(1, true, 0); else QNN_ENC(1, false, 0);
-    } else if (rpu == 2) {
-        if (k == 64) QNN_ENC(2, true, 0); else QNN_ENC(2, false, 0);
     } else {
-        if (k == 32) QNN_ENC(4, true, 0); else QNN_ENC(4, false, 0);
+        if (k == 64) QNN_ENC(2, true, 0); else QNN_ENC(2, false, 0);
     }
 #undef QNN_ENC
 }

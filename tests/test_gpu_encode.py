@@ -24,7 +24,8 @@ def special_values(scale, bits):
 
 
 @pytest.mark.parametrize("bits", range(1, 9))
-@pytest.mark.parametrize("rows,k,ldx", [(1, 1, 1), (3, 31, 31), (5, 33, 40), (7, 127, 127), (2, 129, 129),
+@pytest.mark.parametrize("rows,k,ldx", [(1, 1, 1), (3, 31, 31), (5, 33, 40), (7, 127, 127), (2, 129, 129), (6, 5, 12), (4, 20, 21),
+                                        (300, 3, 3), (9, 50, 51),
                                         (9, 300, 333), (4, 1000, 1000), (33, 512, 512)])
 def test_encode_pack_bit_exact(env, bits, rows, k, ldx):
     torch, qnn, dev = env
