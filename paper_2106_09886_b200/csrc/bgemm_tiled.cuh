@@ -204,6 +204,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
         int64_t pixbase;        // conv: n*H*W of the row's image
         int h0, w0;             // conv: top-left input coordinate of the row's window
         bool a_ok, w_ok;
+        int tile_n;             // feature tile (selects the weights)
     };
     auto prep_tile = [&](int tile) {
         TileSrc t;
@@ -211,6 +212,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
         const int64_t m0 = (int64_t)(tile - tile_n * p.tiles_m) * kBM;
         const int n0 = tile_n * kBN;
         const int64_t am = m0 + srow;
+        t.tile_n = tile_n;
         t.a_ok = a_unit && am < p.Mg;
         t.w_ok = (n0 + wrow) < p.Ng;
         t.a = p.a + ((int64_t)(t.a_ok ? am : 0) * AB + a_plane) * p.a_pitch;
@@ -243,6 +245,13 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
         return t;
     };
 
+    // 9-word-group kernels keep the weights resident: their tiles have one or two stages, so stage s of every tile
+    // lands in the same buffer (two stages) or the buffers alternate (one stage), and a CTA walks many row tiles of one
+    // feature tile.  w_tag[buf] records which (feature tile, stage) weights buffer `buf` holds, already re-coded; a
+    // stage whose weights are there copies and re-codes only its activations (two thirds of a stage's copies are
+    // weights).  The tags are the same in every thread of the CTA.
+    int w_tag0 = -1, w_tag1 = -1;
+    bool w_fresh0 = false, w_fresh1 = false;   // weights copied for the pending stage of that buffer: re-code them
     // Copies stage `stage` of the tile described by `t` into buffer `buf` (asynchronously; one commit group).
     auto issue_stage = [&](const TileSrc &t, int stage, int buf) {
         const uint32_t a_smem = smem_base + (uint32_t)buf * BUF_VEC * 16u;
@@ -265,10 +274,14 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
                     }
                 }
             }
+            const int tag = t.tile_n * 2 + stage;
+            const bool fresh = (buf ? w_tag1 : w_tag0) != tag;
+            if (buf) { w_tag1 = tag; w_fresh1 = fresh; } else { w_tag0 = tag; w_fresh0 = fresh; }
 #pragma unroll
             for (int q = 0; q < W_Q; ++q) {
                 const int u = tid + q * kThreads;
                 if ((W_UNITS % kThreads) != 0 && u >= W_UNITS) break;
+                if (!fresh) break;                                           // these weights are resident
                 const int rp = u % (kBN * WB), ch = u / (kBN * WB);
                 const int plane = rp / kBN;
                 const int gi = stage * kStageChunks + ch;
@@ -370,6 +383,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             for (int q = 0; q < W_Q; ++q) {
                 const int u = tid + q * kThreads;
                 if ((W_UNITS % kThreads) != 0 && u >= W_UNITS) break;
+                if (!(buf ? w_fresh1 : w_fresh0)) break;                     // resident weights are already re-coded
                 const int rp = u % (kBN * WB), ch = u / (kBN * WB);
                 const int plane = rp / kBN;
                 if (stage * kStageChunks + ch >= p.nfull) continue;
