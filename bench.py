@@ -345,6 +345,124 @@ def training_side_leg(torch, qnn, dev, planes, packed, mp, mp_kind):
         return {"what": "Algorithm 1 backward", "unavailable": f"{type(exc).__name__}: {exc}"[:200]}
 
 
+def eq16_model_speedup(n: int, m_bits: int, k_bits: int, gamma: float = 1.91, reg_len: int = 64) -> float:
+    """The paper's cost model of its efficiency experiment (Eq. 16): n multiply-accumulates worth gamma bit
+    operations each, against M*K plane pairs of gamma + 2*ceil(n/L) operations plus M*K - 1 combining additions
+    of beta = gamma/2 each."""
+    pairs = m_bits * k_bits
+    return n * gamma / (pairs * (gamma + 2 * ((n + reg_len - 1) // reg_len)) + (pairs - 1) * gamma / 2.0)
+
+
+def configs_leg(torch, qnn, dev, peaks, mp, mp_kind, quick=False):
+    """Outside the timed step: every configuration of the workload list, each call timed alone with CUDA events.
+    Configurations 1-3 run on the seeded host-generated tensors (L2 flushed before every timed call; the two small
+    ones also warm), the two convolution stacks and the 8192^3 sweep on device-drawn tensors of the stated shapes
+    and distributions (their outputs are larger than L2).  Every entry carries its own roofline: the slower of its
+    algorithmic bytes at the measured HBM peak and its popcount instructions at this run's popcount rate."""
+    import statistics as st
+    from paper_2106_09886_b200 import run_case as rc
+    from paper_2106_09886_b200 import workloads as wl
+    popc_per_s = peaks["xor_popc_add"] * 1e12 / 64.0          # the plain probe issues one popcount per word operation
+    hbm = mp["hbm_gbs"]
+    reps = 3 if quick else 7
+    med = lambda f, flush=True, n=reps: st.median(rc._time_calls(f, n, 3, flush=flush))
+
+    def entry(Mg, Ng, Kg, ab, wb, ms, roof, extra=None):
+        e = {"Mg": Mg, "Ng": Ng, "Kg": Kg, "ab": ab, "wb": wb, "ms": ms,
+             "binary_tops": binary_ops(Mg, Ng, Kg, ab, wb) / (ms * 1e-3) / 1e12,
+             "equiv_int_gops": 2.0 * Mg * Ng * Kg / (ms * 1e-3) / 1e9, "roofline": roof}
+        if extra:
+            e.update(extra)
+        return e
+
+    def fc_case(a, w, k_major, ab, wb, warm_too):
+        Mg, Kg = a.shape
+        Ng = w.shape[1] if k_major else w.shape[0]
+        sa, sw = wl.per_tensor_scale(a, ab), wl.per_tensor_scale(w, wb)
+        alpha = float(np.float32(sa * sw))
+        a_d = torch.from_numpy(a).to(dev)
+        packed = qnn.pack_weights(torch.from_numpy(np.ascontiguousarray(w)).to(dev), Ng, 1, Kg,
+                                  qnn.W_TCN if k_major else qnn.W_NTC, wb, sw)
+        planes = torch.empty((Mg, ab, qnn.row_words(Kg)), dtype=torch.int32, device=dev)
+        out = torch.empty((Mg, Ng), dtype=torch.float32, device=dev)
+        enc = lambda i: qnn.encode_pack(a_d, ab, sa, 0, planes=planes)
+        gemm = lambda i: qnn.bgemm(planes, ab, packed, wb, Mg, Ng, Kg, alpha, out=out)
+        enc(0)
+        t_enc, t = med(enc), med(gemm)
+        extra = {"encode_ms": t_enc, "l2": "flushed before every timed call"}
+        if warm_too:
+            extra["ms_warm"], extra["encode_ms_warm"] = med(gemm, flush=False), med(enc, flush=False)
+        return entry(Mg, Ng, Kg, ab, wb, t, rc.layer_roofline(Mg, Ng, ab, wb, False, 1, 1, Kg, Mg, t, popc_per_s, hbm), extra)
+
+    res = {"method": "CUDA events around single calls, median of %d after 3 warm-up calls; roofline per entry = "
+                     "max(algorithmic bytes / measured HBM peak, popcounts / popcount rate of this run's probe)" % reps,
+           "popcount_rate_gpops": popc_per_s / 1e9, "hbm_peak_gbs": hbm, "hbm_peak_kind": mp_kind}
+    c1 = wl.fc_config1(0)
+    res["config1_fc_64x256x512_w2a2"] = fc_case(c1.a, c1.w, c1.k_major, c1.ab, c1.wb, True)
+    res["config1_fc_64x256x512_w2a2"]["note"] = "launch-latency-bound: 33.6 M binary MACs; the roofline fraction only says so"
+
+    c2 = wl.conv_config2(0)
+    s2 = c2.shape
+    sa, sw = wl.per_tensor_scale(c2.a, s2.ab), wl.per_tensor_scale(c2.w, s2.wb)
+    alpha = float(np.float32(sa * sw))
+    a_d = torch.from_numpy(c2.a).to(dev).view(-1, s2.C)
+    packed = qnn.pack_weights(torch.from_numpy(c2.w).to(dev), s2.Cout, 9, s2.C, qnn.W_NTC, s2.wb, sw)
+    planes = torch.empty((a_d.shape[0], s2.ab, qnn.row_words(s2.C)), dtype=torch.int32, device=dev)
+    out = torch.empty((s2.N, s2.Ho, s2.Wo, s2.Cout), dtype=torch.float32, device=dev)
+    enc = lambda i: qnn.encode_pack(a_d, s2.ab, sa, 0, planes=planes)
+    conv = lambda i: qnn.bconv2d(planes, s2.ab, packed, s2.wb, s2.N, s2.H, s2.W, s2.C, s2.Cout, 3, 3, 1, 1, alpha, out=out)
+    enc(0)
+    t_enc, t = med(enc), med(conv)
+    res["config2_conv3x3_256_14x14_b32_w2a2"] = entry(
+        s2.Mg, s2.Cout, s2.Kg, s2.ab, s2.wb, t,
+        rc.layer_roofline(s2.Mg, s2.Cout, s2.ab, s2.wb, True, 3, 3, s2.C, s2.N * s2.H * s2.W, t, popc_per_s, hbm),
+        {"encode_ms": t_enc, "ms_warm": med(conv, flush=False), "encode_ms_warm": med(enc, flush=False),
+         "l2": "flushed before every timed call (ms), not flushed (ms_warm)"})
+    del a_d, packed, planes, out
+
+    c3 = wl.gemm_config3(0, N_SQ, 2, 2)
+    res["config3_gemm_4096"] = []
+    for wb, ab in wl.GEMM_SWEEP_BITS:
+        e = fc_case(c3.a, c3.w, False, ab, wb, False)
+        res["config3_gemm_4096"].append(e)
+
+    for key, net, batch in (("config4_resnet18_b256_w3a3", "resnet18", 256), ("config5_vgg16_b64_w4a4", "vgg16", 64)):
+        r = rc.time_stack(net, batch, reps=3, warmup=2)
+        layers, roof_ms = [], 0.0
+        for L in r["layers"]:
+            roof = rc.layer_roofline(L["Mg"], L["Ng"], L["ab"], L["wb"], True, L["R"], L["S"], L["C"], L["in_rows"],
+                                     L["conv_ms"], popc_per_s, hbm)
+            roof_ms += roof["roofline_ms"]
+            layers.append({"layer": L["layer"], "Mg": L["Mg"], "Ng": L["Ng"], "Kg": L["Kg"], "encode_ms": L["encode_ms"],
+                           "conv_ms": L["conv_ms"], "conv_encode_fused_ms": L["conv_encode_ms"],
+                           "binary_tops": L["conv_binary_tops"], "equiv_int_gops": L["conv_equiv_int_gops"],
+                           "encode_gbs": L["encode_gbs"],
+                           "roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac")}})
+        conv_ms = sum(L["conv_ms"] for L in r["layers"])
+        res[key] = {"batch": batch, "layers": layers, "total_ms": r["total_ms"], "conv_ms": conv_ms,
+                    "encode_ms": r["total_ms"] - conv_ms,
+                    "chained_fused_ms": sum(L["conv_encode_ms"] for L in r["layers"]),
+                    "binary_tops": r["binary_tops"], "equiv_int_gops": r["equiv_int_gops"],
+                    "roofline": {"bound": "alu (per layer: see layers)", "frac": roof_ms / conv_ms,
+                                 "what": "sum of the layers' roofline times / sum of their measured convolution times"}}
+
+    # the paper's efficiency experiment: 8192^3, 1..6 bits, against the Eq. 16 cost model (shape of the curve; the
+    # fp32 kernel it is a speed-up over is one of the paper's comparison systems and is not built)
+    sweep, base = [], None
+    n8 = 8192
+    for b in range(1, 7):
+        r = rc.time_gemm(n8, n8, n8, b, b, reps=3, warmup=2, sets=1)
+        ms = r["ms_median"]
+        base = base or ms
+        roof = rc.layer_roofline(n8, n8, b, b, False, 1, 1, n8, n8, ms, popc_per_s, hbm)
+        sweep.append({"bits": b, "ms": ms, "binary_tops": r["binary_tops"], "equiv_int_gops": r["equiv_int_gops"],
+                      "time_vs_1bit": ms / base, "eq16_cost_vs_1bit": eq16_model_speedup(n8, 1, 1) / eq16_model_speedup(n8, b, b),
+                      "eq16_speedup_model": eq16_model_speedup(n8, b, b),
+                      "roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac")}})
+    res["sweep_8192_bits_1_to_6"] = sweep
+    return res
+
+
 def load_measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -471,7 +589,12 @@ def run_gpu(args):
     t2.record()
     barrier()
     e2e_ms_total = s2.elapsed_time(t2)
-    checksum = float(out_host[0, 0])
+    # the end-to-end result, all of it, against the plain two-call route on the resident copy of the same input
+    ref_planes = qnn.encode_pack(a_bufs[0], AB, sa, 0)
+    ref_out = qnn.bgemm(ref_planes, AB, packed, WB, Mg, Ng, Kg, alpha)
+    torch.cuda.synchronize()
+    e2e_identical = bool(torch.equal(ref_out.cpu(), out_host))
+    del ref_planes, ref_out
 
     ms_total, e2e_ms_total = max_over_ranks([ms_total, e2e_ms_total], dev, use_dist)
 
@@ -504,7 +627,8 @@ def run_gpu(args):
             "e2e": {"value": ops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": Mg * Kg * 4, "d2h_bytes_per_step": Mg * Ng * 4, "steps": e2e_steps,
                     "api": f"qnn_fc_forward_host_pipelined (pinned host buffers, {args.e2e_chunk_rows}-row chunks over "
-                           f"{args.e2e_streams} streams, consecutive steps pipelined)", "checksum": checksum},
+                           f"{args.e2e_streams} streams, consecutive steps pipelined)",
+                    "result_identical_to_resident_path": e2e_identical},
             "roofline": {"kernel": "qnn_bgemm", "bound": "alu", "achieved": achieved, "peak": kernel_peak,
                          "unit": UNIT, "frac": achieved / kernel_peak, "traffic": traffic,
                          "peak_source": "popcount issue rate measured in this run by the register-resident xor+popc+add "
@@ -528,6 +652,11 @@ def run_gpu(args):
             line["comparison_int8_tensor"] = comparison
         if world == 1:
             line["training_side"] = training_side_leg(torch, qnn, dev, planes[0], packed, mp, mp_kind)
+        if world == 1 and not args.no_configs:
+            try:
+                line["configs"] = configs_leg(torch, qnn, dev, peaks, mp, mp_kind)
+            except Exception as exc:   # reported beside the benchmark, never fails it
+                line["configs"] = {"unavailable": f"{type(exc).__name__}: {exc}"[:300]}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg()
         print(json.dumps(line), flush=True)
@@ -543,6 +672,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["graft", "reference"], default="graft")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table (configs 1-5 and the 8192^3 sweep)")
     ap.add_argument("--e2e-chunk-rows", type=int, default=E2E_CHUNK_ROWS, help="rows per chunk of the end-to-end pipeline")
     ap.add_argument("--e2e-streams", type=int, default=E2E_STREAMS, help="streams of the end-to-end pipeline")
     args = ap.parse_args()

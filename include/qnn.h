@@ -11,7 +11,10 @@
  * Conventions
  *   - Every pointer is a DEVICE pointer unless its name ends in _host.  The caller
  *     owns every buffer; the library allocates nothing, never frees, and never
- *     modifies an input.
+ *     modifies an input.  The only state it keeps between calls is on the device:
+ *     one status word that the tensor-path kernels set when a bounded wait gives
+ *     up (read and cleared by qnn_tensor_path_status), and the fixed scratch array
+ *     of qnn_fc_forward_noalloc; on the host, the per-device address of that array.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *     only enqueue work; they return before it has run.
  *   - Every call returns a qnn_status.  Argument errors are found on the host
@@ -271,10 +274,25 @@ int qnn_unpack_codes_f32(const uint32_t *planes, size_t rows, size_t k, int bits
 
 /*
  * Synchronises the device and reports whether a tensor-path kernel gave up a bounded wait since the last call:
- * *status = 0 and QNN_OK, or *status = 1 + the id of the first wait that gave up (0 producer, 1 MMA issuer,
- * 2 epilogue) and QNN_E_DEVICE; the record is cleared.  Results of a call that reported an error are undefined.
+ * *status = 0 and QNN_OK, or *status = 1 + the id of the first wait that gave up (0 producer waiting for a free
+ * stage, 1 MMA issuer waiting for a stage's operands, 2 epilogue waiting for an accumulator, 3 MMA issuer waiting
+ * for a free accumulator buffer) and QNN_E_DEVICE; the record is cleared.  Results of a call that reported an
+ * error are undefined (its kernels have ended and released what they held; the context stays usable).
+ * qnn_last_device_status is the same call under the name the status word has in the library's error convention.
  */
 int qnn_tensor_path_status(unsigned int *status);
+int qnn_last_device_status(unsigned int *status);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper; diagnostic only).  Enqueues one small thread block
+ * built from the tensor-path kernels' own wait helpers in which a producer waits for a stage release that never
+ * comes: after poll_limit polls (16..65536) it gives up, raises the block's abort flag and the library's status
+ * word with wait id 0, lets its copy in flight land, and a second warp waiting for an accumulator leaves through the
+ * abort flag.  The kernel then ends normally -- nothing traps, faults or spins without bound.  The next
+ * qnn_tensor_path_status call therefore returns QNN_E_DEVICE with *status = 1 and clears the record; later calls
+ * of the library are unaffected.
+ */
+int qnn_selftest_bounded_wait(unsigned int poll_limit, void *stream);
 
 /*
  * Comparison only, not the paper's method: the product of qnn_bgemm computed as ONE signed 8-bit tensor-core GEMM
@@ -369,8 +387,13 @@ int qnn_fc_forward_noalloc(const float *x, int64_t Mg, int Kg, int64_t ldx, int 
  *              operands in registers (word_ops counts 32 binary multiply-accumulates as one word operation).
  *   sink: device int32 [blocks*256], written once at the end.
  * qnn_probe_copy enqueues a plain 16-byte-vector device copy of `bytes` (multiple of 16).
+ * qnn_popcounts_per_output returns how many popcount instructions the kernel that qnn_bgemm (is_conv = 0, R = S = 1,
+ * C = Kg, Cout = Ng) or qnn_bconv2d (is_conv != 0) runs for such a layer issues per output element, all ab*wb plane
+ * pairs together (0 = arguments out of range): the popcount pipe is the scarce unit of the contraction, so
+ * outputs * that number / the popcount rate of probe variant 0 is the layer's bit-operation roofline time.
  */
 int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream);
+int64_t qnn_popcounts_per_output(int ab, int wb, int is_conv, int R, int S, int C, int Cout);
 int qnn_probe_copy(void *dst, const void *src, size_t bytes, void *stream);
 
 #ifdef __cplusplus

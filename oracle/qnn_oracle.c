@@ -22,8 +22,9 @@
  * c_m of every element, one bit per element, +1 stored as 1) so that packed
  * planes can be compared word for word.
  *
- * Floating point: the quantizer decides an integer, so it is evaluated in
- * binary32 with one explicit fused multiply-add (the precision the kernels use);
+ * Floating point: the quantizer decides an integer from binary32 data, so the
+ * decision is fixed to one binary32 evaluation order: v = fma(x, 1/(2s), 2^(b-1))
+ * with a single rounding (Table 2's interval ends are where v is an integer);
  * everything after it is integer until the single binary32 multiply of step 3.
  *
  * Parallelism: independent output rows are spread over OpenMP threads.  There is
@@ -318,9 +319,11 @@ int oracle_conv2d_general(const int16_t *qa, const int16_t *qw, int N, int H, in
  * the encoder.  With xn = x / r and k_m = (2^M - 1) / 2^m:
  *   phi_M^M(xn) = sign(sin(k_M pi xn)),   phi_M^m(xn) = sign(-sin(k_m pi xn)) for m < M,
  *   d phi_M^m / d xn = +- k_m pi cos(k_m pi xn) for |xn| <= 1, else 0 (sign + for m = M, - otherwise).
- * Forward: the sign is a decision, so it is taken in the kernel's precision: y = k_m * xn is one binary32
- * product (k_m is exactly representable), sin(pi y) is 0 exactly when y is an integer, positive when floor(y)
- * is even and negative when it is odd -- no library sine is involved, so the decision is reproducible.
+ * Forward: the sign is a decision on binary32 data, and Eq. 10 does not say in which precision its argument is
+ * formed.  Reading taken: xn = x / r and y = k_m * xn are one binary32 division and one binary32 product (k_m
+ * is exactly representable); sign(sin(pi y)) is then decided exactly from y: 0 when y is an integer, positive
+ * when floor(y) is even and negative when it is odd -- no library sine is involved, so the decision is
+ * reproducible and matches the exact sign of the sine of pi * y.
  * c[(m-1)*n + e] receives phi_M^m of element e as -1, 0 or +1.
  */
 int oracle_mbit_encoder_forward(const float *x, size_t n, int bits, float r, float *c) {
@@ -346,7 +349,7 @@ int oracle_mbit_encoder_backward(const float *x, const float *gc, size_t n, int 
     if (!x || !gc || !gx || bits < 1 || bits > 8 || !(r > 0.0f)) return ORACLE_E_ARG;
     const double pi = 3.14159265358979323846;
     for (size_t e = 0; e < n; ++e) {
-        const double xn = (double)(x[e] / r);                          /* the division the kernel performs */
+        const double xn = (double)(x[e] / r);                          /* xn as Eq. 10 forms it: one binary32 division */
         double g = 0.0;
         if (xn >= -1.0 && xn <= 1.0) {
             for (int m = 1; m <= bits; ++m) {

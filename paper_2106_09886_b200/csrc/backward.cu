@@ -456,6 +456,60 @@ extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_pl
     return run_gemm_tf32_split(gt, ldm, colt, ldm, p, split_ws, st);
 }
 
+// ------------------------------------------------------------------------------------------------ wait self-test
+
+namespace {
+
+__device__ __align__(128) uint32_t g_selftest_src[32];      // source of the self-test's bulk copy (contents irrelevant)
+
+// One CTA, two warps, built from the same helpers as tc_gemm_kernel so that their give-up path runs once on demand:
+//   warp 0, lane 0 (producer role): starts one 128-byte bulk copy into shared memory under full[0], then waits for a
+//     stage release on empty[0] that no consumer ever gives -> gives up after `limit` polls, raises the CTA's abort
+//     flag and the library's error word (wait id 0), and drains its copy in flight like the GEMM's producer;
+//   warp 1 (epilogue role): waits, all lanes, for an accumulator on acc_full that no MMA ever commits, with a limit
+//     64 times longer, and leaves through the abort flag (or by its own limit).
+// Every loop is bounded; the kernel ends normally.
+__global__ void __launch_bounds__(64, 1) bounded_wait_selftest_kernel(unsigned int limit, unsigned int *err) {
+    __shared__ __align__(128) uint32_t dst[32];
+    __shared__ __align__(8) uint64_t bars[3];               // full[0], empty[0], acc_full[0]
+    __shared__ uint32_t abort_word;
+    volatile uint32_t *abort_flag = &abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        mbar_init(&bars[0], 1);
+        mbar_init(&bars[1], 1);
+        mbar_init(&bars[2], 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(&bars[0], 128);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 128, [%2];"
+                         ::"r"(smem_u32(dst)), "l"(__cvta_generic_to_global(g_selftest_src)), "r"(smem_u32(&bars[0])) : "memory");
+            // second use of a one-stage ring: wants the consumer's release of the first use, which never comes
+            if (!mbar_wait(&bars[1], 0u, abort_flag, 0, err, limit)) drain_copies_in_flight(&bars[0], 1, 1, limit << 6);
+        }
+    } else {
+        __all_sync(0xffffffffu, mbar_wait(&bars[2], 0u, abort_flag, 2, err, limit << 6));
+    }
+    __syncthreads();
+}
+
+}  // namespace
+
+extern "C" int qnn_selftest_bounded_wait(unsigned int poll_limit, void *stream) {
+    if (poll_limit < 16u || poll_limit > (1u << 16)) return QNN_E_ARG;
+    unsigned int *err = qnn_tc_error_word();
+    if (!err) return QNN_E_CUDA;
+    bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(poll_limit, err);
+    return qnn_launch_status();
+}
+
+extern "C" int qnn_last_device_status(unsigned int *status) { return qnn_tensor_path_status(status); }
+
 extern "C" int qnn_tensor_path_status(unsigned int *status) {
     if (!status) return QNN_E_ARG;
     if (cudaDeviceSynchronize() != cudaSuccess) return QNN_E_CUDA;

@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(kThreads) bconv_dense1_kernel(const Params p) 
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     if (!n_ok[h]) continue;
-                    const int32_t v = n_valid * PROD - 2 * (s_acc[h] - AMAX * corr[h]);
+                    const int32_t v = qnn_combine(n_valid * PROD, s_acc[h] - AMAX * corr[h]);
                     const int64_t o = o_row + n[h];
                     if (p.acc) p.acc[o] = v;
                     if (p.out) {

@@ -53,7 +53,7 @@ bconv_generic_kernel(const uint32_t *__restrict__ a, int ab, const uint32_t *__r
         }
     }
     const int32_t AB = ((1 << ab) - 1) * ((1 << wb) - 1);
-    store_out(out, g.Cout, acc, m, co, g.Cout, valid * g.C * AB - 2 * s, alpha);
+    store_out(out, g.Cout, acc, m, co, g.Cout, qnn_combine(valid * g.C * AB, s), alpha);
 }
 
 // Optional fused epilogue: the next layer's encoder applied to the fp32 result.
@@ -137,11 +137,12 @@ extern "C" int qnn_bconv2d_encode(const uint32_t *a_planes, int ab, const void *
 
 namespace {
 
-int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
-               float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream) {
+// Argument checks shared by qnn_bgemm, the chaining form and the composite entry points; `has_next` = the chaining
+// epilogue supplies an output of its own (next-layer planes), so out and acc may both be absent.
+int bgemm_check(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
+                const float *out, int64_t ldo, const int32_t *acc, bool has_next) {
     if (!a_planes || !w_packed || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
-    if (const int rc = check_next(ne)) return rc;
-    if (!out && !acc && !(ne && ne->planes)) return QNN_E_ARG;
+    if (!out && !acc && !has_next) return QNN_E_ARG;
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb) || (out && ldo < Ng)) return QNN_E_ARG;
     if (!isfinite(alpha)) return QNN_E_SCALE;
     if (!qnn_aligned(a_planes, 16) || !qnn_aligned(w_packed, 16) || !qnn_aligned(out, 4) || !qnn_aligned(acc, 4))
@@ -149,6 +150,14 @@ int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     const int64_t AB = (int64_t)((1 << ab) - 1) * ((1 << wb) - 1);
     if ((int64_t)Kg * AB >= ((int64_t)1 << 31)) return QNN_E_RANGE;
     if (Mg > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
+    return QNN_OK;
+}
+
+int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
+               float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream) {
+    if (!a_planes || !w_packed || Mg <= 0 || Ng <= 0 || Kg <= 0) return QNN_E_ARG;
+    if (const int rc = check_next(ne)) return rc;
+    if (const int rc = bgemm_check(a_planes, ab, w_packed, wb, Mg, Ng, Kg, alpha, out, ldo, acc, ne && ne->planes)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int kw = (int)qnn_row_words_i(Kg);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
@@ -244,10 +253,32 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
 
 }  // namespace
 
+// Popcount instructions per output (all plane pairs) of the kernel that bgemm_impl / bconv_impl pick for a layer
+// (plain convolution: dilation 1, not transposed); mirrors their dispatch.
+extern "C" int64_t qnn_popcounts_per_output(int ab, int wb, int is_conv, int R, int S, int C, int Cout) {
+    if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb) || R < 1 || S < 1 || C < 1 || Cout < 1 || (!is_conv && R * S != 1)) return 0;
+    const int64_t cw = (C + 31) / 32, pairs = (int64_t)ab * wb;
+    if (is_conv && qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout))
+        return (ab == 4 && wb == 4) ? 10 : ((ab == 3 && wb == 3) ? 7 : pairs);
+    if (is_conv && R * S == 9 && cw <= 4 && ab <= 4 && wb <= 4) return pairs * cw * 4;      // 9-word groups
+    qnn_tiled::Params p = {};
+    p.kwords = is_conv ? (int)(R * S * cw) : (int)qnn_row_words_i(C);
+    qnn_tiled::set_k_split(p);
+    return pairs * ((int64_t)p.nfull * 4 + p.ntail);
+}
+
+int qnn_check_bgemm(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
+                    const float *out, int64_t ldo, const int32_t *acc) {
+    return bgemm_check(a_planes, ab, w_packed, wb, Mg, Ng, Kg, alpha, out, ldo, acc, false);
+}
+
 extern "C" int qnn_fc_forward_host(const float *x_host, int64_t Mg, int Kg, int ab, float scale_a, unsigned flags,
                                    const void *w_packed, int wb, int Ng, float alpha, float *out_host, float *x_dev,
                                    uint32_t *planes_dev, float *out_dev, void *stream) {
     if (!x_host || !out_host || !x_dev || !planes_dev || !out_dev || Mg <= 0 || Kg <= 0 || Ng <= 0) return QNN_E_ARG;
+    // every argument error of the two kernels is found here, before the first copy is enqueued
+    if (const int rc = qnn_check_encode_pack(x_dev, Mg, Kg, Kg, ab, scale_a, flags, planes_dev, nullptr)) return rc;
+    if (const int rc = qnn_check_bgemm(planes_dev, ab, w_packed, wb, Mg, Ng, Kg, alpha, out_dev, Ng, nullptr)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(x_dev, x_host, (size_t)Mg * Kg * sizeof(float), cudaMemcpyHostToDevice, st) != cudaSuccess)
         return QNN_E_CUDA;
@@ -267,6 +298,10 @@ extern "C" int qnn_fc_forward_host_pipelined(const float *x_host, int64_t Mg, in
     if (!x_host || !out_host || !x_dev || !planes_dev || !out_dev || !streams || Mg <= 0 || Kg <= 0 || Ng <= 0)
         return QNN_E_ARG;
     if (nstreams < 1 || rows_per_chunk < 1 || !qnn_bits_ok(ab)) return QNN_E_ARG;
+    // Every argument error of the two kernels is found here, before the first chunk is enqueued: a chunk is a row
+    // range of the same buffers (rows of planes are multiples of 16 bytes), so it passes whatever the whole passes.
+    if (const int rc = qnn_check_encode_pack(x_dev, Mg, Kg, Kg, ab, scale_a, flags, planes_dev, nullptr)) return rc;
+    if (const int rc = qnn_check_bgemm(planes_dev, ab, w_packed, wb, Mg, Ng, Kg, alpha, out_dev, Ng, nullptr)) return rc;
     const int64_t plane_words_per_row = (int64_t)ab * qnn_row_words_i(Kg);
     int64_t chunk = 0;
     for (int64_t r0 = 0; r0 < Mg; r0 += rows_per_chunk, ++chunk) {

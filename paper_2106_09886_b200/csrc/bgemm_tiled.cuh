@@ -557,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, 2) bgemm_tiled_kernel(const Params p
             for (int c = 0; c < 4; ++c) {
                 const int n = n0 + tx + 16 * c;
                 if (!FUSED && n >= p.Ng) continue;
-                const int32_t v = n_valid * PROD - 2 * (acc[r][c] - AMAX * corr[c]);
+                const int32_t v = qnn_combine(n_valid * PROD, acc[r][c] - AMAX * corr[c]);
                 fv[c] = __fmul_rn(__int2float_rn(v), p.alpha);
                 if (FUSED && p.ch_gamma != nullptr && n < p.Ng)
                     fv[c] = __fmaf_rn(fv[c], __ldg(p.ch_gamma + n), p.ch_beta ? __ldg(p.ch_beta + n) : 0.0f);

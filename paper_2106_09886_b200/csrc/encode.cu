@@ -533,12 +533,18 @@ void launch_pack_w(const float *w, int n_out, int taps, int c_in, int layout, fl
         default: CALL(8); break;               \
     }
 
-extern "C" int qnn_encode_pack(const float *x, int64_t rows, int k, int64_t ldx, int bits, float scale,
-                               unsigned flags, uint32_t *planes, int32_t *rowsum, void *stream) {
+int qnn_check_encode_pack(const float *x, int64_t rows, int k, int64_t ldx, int bits, float scale, unsigned flags,
+                          const uint32_t *planes, const int32_t *rowsum) {
     if (!x || !planes || rows <= 0 || k <= 0 || ldx < k || !qnn_bits_ok(bits) || (flags & ~QNN_RELU)) return QNN_E_ARG;
     if (!(scale >= 1e-30f) || !(scale <= 1e30f)) return QNN_E_SCALE;   // also rejects NaN, 0, negatives, infinities
     if (!qnn_aligned(planes, 16) || !qnn_aligned(x, 4) || (rowsum && !qnn_aligned(rowsum, 4))) return QNN_E_ALIGN;
     if (k > (1 << 30) || rows > ((int64_t)1 << 40)) return QNN_E_RANGE;
+    return QNN_OK;
+}
+
+extern "C" int qnn_encode_pack(const float *x, int64_t rows, int k, int64_t ldx, int bits, float scale,
+                               unsigned flags, uint32_t *planes, int32_t *rowsum, void *stream) {
+    if (const int rc = qnn_check_encode_pack(x, rows, k, ldx, bits, scale, flags, planes, rowsum)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool relu = (flags & QNN_RELU) != 0;
     if (rowsum && (k > 64 || (qnn_aligned(x, 16) && ldx % 4 == 0)) && cudaMemsetAsync(rowsum, 0, (size_t)rows * sizeof(int32_t), st) != cudaSuccess)

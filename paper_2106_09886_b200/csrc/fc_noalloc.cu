@@ -51,9 +51,15 @@ extern "C" int qnn_fc_forward_noalloc(const float *x, int64_t Mg, int Kg, int64_
     // the planes of this problem must fit the built-in buffer
     const size_t need = qnn_planes_bytes(Mg, Kg, ab);
     if (need == 0 || need > (size_t)QNN_NOALLOC_SCRATCH_BYTES) return QNN_E_RANGE;
+    // Every argument error of the two kernels is found here, before the encoder may overwrite the shared array (and
+    // before the device is touched at all).  The checks only look at the planes pointer's alignment, which the
+    // array's declaration fixes, so a stand-in with that alignment serves.
+    const uint32_t *planes_stand_in = reinterpret_cast<const uint32_t *>(static_cast<uintptr_t>(256));
+    int rc;
+    if ((rc = qnn_check_encode_pack(x, Mg, Kg, ldx, ab, scale_a, flags, planes_stand_in, nullptr)) != QNN_OK) return rc;
+    if ((rc = qnn_check_bgemm(planes_stand_in, ab, w_packed, wb, Mg, Ng, Kg, alpha, out, ldo, nullptr)) != QNN_OK) return rc;
     uint32_t *planes = nullptr;
-    int rc = scratch_for_current_device(&planes);
-    if (rc != QNN_OK) return rc;
+    if ((rc = scratch_for_current_device(&planes)) != QNN_OK) return rc;
     // qnn_encode_pack writes every word of the region it uses (padding included), so nothing left
     // over from an earlier call can leak into this one and nothing needs clearing first.
     rc = qnn_encode_pack(x, Mg, Kg, ldx, ab, scale_a, flags, planes, nullptr, stream);

@@ -17,7 +17,20 @@ static inline int64_t qnn_w_row_words_i(int taps, int c_in) {
 // Defined in backward.cu: device word shared by all tensor-path kernels (see qnn_tensor_path_status).
 unsigned int *qnn_tc_error_word();
 
+// Host-side argument checks of qnn_encode_pack and qnn_bgemm without enqueuing anything (encode.cu, bgemm.cu): the
+// composite entry points run both before their first copy or launch.
+int qnn_check_encode_pack(const float *x, int64_t rows, int k, int64_t ldx, int bits, float scale, unsigned flags,
+                          const uint32_t *planes, const int32_t *rowsum);
+int qnn_check_bgemm(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
+                    const float *out, int64_t ldo, const int32_t *acc);
+
 static inline int qnn_launch_status() { return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA; }
+
+// Eq. 8's combine, n*A*B - 2*S, for S = sum_ij 2^(i+j) X_ij <= n*A*B < 2^31: 2*S may reach 2^32, so the subtraction
+// is done modulo 2^32 (unsigned) and the result, which always fits, is reinterpreted.
+__device__ __forceinline__ int32_t qnn_combine(int32_t n_times_ab, int32_t s) {
+    return (int32_t)((uint32_t)n_times_ab - 2u * (uint32_t)s);
+}
 
 // Unsigned code t in [0, 2^bits - 1] of a real value (odd code q = 2t - (2^bits - 1)).
 // inv2s = 1/(2*scale), half = 2^(bits-1); [lo, hi] is a pre-clamp of x (see qnn_clamp_bounds).

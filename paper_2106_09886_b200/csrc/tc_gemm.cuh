@@ -33,20 +33,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Every wait is bounded: after WAIT_LIMIT failed polls the waiter raises the abort flag of its CTA and the global
-// error word, and every role of the CTA leaves its loop at the next poll.
+// Every wait is bounded: after `limit` failed polls (WAIT_LIMIT unless the caller of the kernel says otherwise) the
+// waiter raises the abort flag of its CTA and the global error word, and every role of the CTA leaves its loop at
+// its next look at the flag.
 constexpr uint32_t WAIT_LIMIT = 1u << 24;
 
 // *err: 0 = no error; else 1 + the id of the wait that gave up first (one device word for the whole library).
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag, unsigned id,
-                                          unsigned int *err) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+                                          unsigned int *err, uint32_t limit) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 1023u) == 1023u && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicCAS(err, 0u, 1u + id);
     return false;
+}
+
+// After an abort: lets the copies still in flight land before the CTA's shared memory goes away.  `it` = stage uses
+// issued so far; the last min(it, stages) of them may still be under way, each signals full[use % stages].
+__device__ __forceinline__ void drain_copies_in_flight(uint64_t *full, long long it, int stages, uint32_t limit) {
+    for (long long j = it > stages ? it - stages : 0; j < it; ++j)
+        for (uint32_t w = 0; w < limit && !mbar_try_wait(&full[j % stages], (uint32_t)(j / stages) & 1u); ++w) {}
 }
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
@@ -147,6 +155,7 @@ struct GemmParams {
     // C + s * split_stride (dense partial buffers); sum_partials_kernel then adds the ksplit buffers in index order.
     int ksplit, kb_per_split;
     long long split_stride;
+    unsigned int wait_limit;            // polls after which a wait on an arrival gives up (0 = WAIT_LIMIT)
 };
 
 // One column of a 32 x 32 chunk (this lane's), rows_here rows: C = Eq. 12 applied to the staged products and x.
@@ -242,6 +251,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    int committed = 0;                  // MMA issuer: tiles whose accumulator has been committed to acc_full
 
     if (warp == 0) {
         if (lane == 0) {
@@ -252,16 +262,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                 for (int kb = wi.kb0; kb < wi.kb1; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                    if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err)) break;
+                    if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err, p.wait_limit)) break;
                     mbar_expect_tx(&full[s], whole ? L::STAGE_BYTES : L::A_BYTES + L::B_BYTES / 2);
                     tma_load_2d(smem + s * L::STAGE_BYTES, &map_a, &full[s], kb * BK, wi.m0);
                     tma_load_2d(smem + s * L::STAGE_BYTES + L::A_BYTES, whole ? &map_b : &map_b_half, &full[s], kb * BK, wi.n0);
                 }
             }
-            if (*abort_flag) {   // let the copies still in flight land before the CTA's shared memory goes away
-                for (long long j = it > STAGES ? it - STAGES : 0; j < it; ++j)
-                    for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(&full[j % STAGES], (uint32_t)(j / STAGES) & 1u); ++w) {}
-            }
+            if (*abort_flag) drain_copies_in_flight(full, it, STAGES, p.wait_limit);
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -271,13 +278,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                 const WorkItem wi = work_item<BN>(w, p, nkb);
                 const uint32_t idesc = wi.width == BN ? idesc_kmajor<BN, KIND>() : idesc_kmajor<BN / 2, KIND>();
                 const int buf = local & 1;
-                if (!mbar_wait(&acc_empty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag, 3, p.err)) break;
+                if (!mbar_wait(&acc_empty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag, 3, p.err, p.wait_limit)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = wi.kb0; kb < wi.kb1; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                    if (!mbar_wait(&full[s], ph, abort_flag, 1, p.err)) break;
+                    if (!mbar_wait(&full[s], ph, abort_flag, 1, p.err, p.wait_limit)) break;
                     tc_fence_after();
                     const uint64_t a_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES));
                     const uint64_t b_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES + L::A_BYTES));
@@ -287,6 +294,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     tc_commit(&empty[s]);
                 }
                 tc_commit(&acc_full[buf]);
+                committed = local + 1;
             }
         }
     } else {
@@ -297,7 +305,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             const WorkItem wi = work_item<BN>(w, p, nkb);
             const int m0 = wi.m0, n0 = wi.n0;
             const int buf = local & 1;
-            if (!mbar_wait(&acc_full[buf], (uint32_t)(local >> 1) & 1u, abort_flag, 2, p.err)) break;
+            // every lane polls (each needs the barrier's acquire), but the warp must reach the warp-wide
+            // tensor-memory load together or not at all: one lane giving up makes all of them leave
+            if (!__all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (uint32_t)(local >> 1) & 1u, abort_flag, 2, p.err, p.wait_limit)))
+                break;
             tc_fence_after();
             // Each 32 x 32 chunk goes through the warp's shared tile: tensor memory hands a thread one row, memory
             // wants a warp on one row, so that every access to C and x is a whole 128-byte line.
@@ -359,11 +370,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     __syncthreads();
     if (warp == 1) {
         // every MMA that was issued has retired once the last committed tile's barrier has completed its phase
-        const int mine = p.items > (int)blockIdx.x ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-        if (mine > 0) {
-            const int last = mine - 1;
-            for (uint32_t w = 0; w < WAIT_LIMIT && !mbar_try_wait(&acc_full[last & 1], (uint32_t)(last >> 1) & 1u); ++w) {}
+        // (a tile that an abort cut short is committed too, with whatever was issued for it, so this covers it)
+        if (lane == 0 && committed > 0) {
+            const int last = committed - 1;
+            for (uint32_t w = 0; w < p.wait_limit && !mbar_try_wait(&acc_full[last & 1], (uint32_t)(last >> 1) & 1u); ++w) {}
         }
+        __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, 2 * BN);
     }
@@ -409,13 +421,11 @@ template <int BN, int STAGES, int KIND>
 int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtensorMap &map_b_half, GemmParams p, int sms,
                 cudaStream_t st) {
     using L = GemmSmem<BN, STAGES>;
-    static bool attr_set = false;   // per process; set again on the next call if it failed
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) !=
-            cudaSuccess)
-            return QNN_E_CUDA;
-        attr_set = true;
-    }
+    // the attribute belongs to the (function, device) pair: set it on every launch, for whichever device is current
+    if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) !=
+        cudaSuccess)
+        return QNN_E_CUDA;
+    if (p.wait_limit == 0) p.wait_limit = WAIT_LIMIT;
     const long long tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return QNN_E_ARG;
     p.tiles_n = (int)tiles_n;
@@ -436,13 +446,11 @@ int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtens
     return qnn_launch_status();
 }
 
+// SM count of the current device (asked every time: a process may use several devices).
 int sm_count() {
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            sms = 0;
-    }
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return 0;
     return sms;
 }
 
@@ -456,7 +464,8 @@ int run_gemm(const void *A, long long lda, const void *B, long long ldb, GemmPar
     if (!qnn_aligned(A, 16) || !qnn_aligned(B, 16) || (lda * esz) % 16 || (ldb * esz) % 16) return QNN_E_ALIGN;
     const int sms = sm_count();
     if (sms <= 0) return QNN_E_CUDA;
-    const bool wide = ((long long)(p.M + BM - 1) / BM) * ((p.N + 255) / 256) >= sms;
+    // a split contraction is planned for 128 x 128 tiles (gemm_ksplit) and keeps them
+    const bool wide = p.ksplit <= 1 && ((long long)(p.M + BM - 1) / BM) * ((p.N + 255) / 256) >= sms;
     CUtensorMap map_a, map_b, map_b_half;
     if (!make_map(&map_a, A, p.M, p.K, lda, BM, KIND) || !make_map(&map_b, B, p.N, p.K, ldb, wide ? 256 : 128, KIND) ||
         !make_map(&map_b_half, B, p.N, p.K, ldb, wide ? 128 : 64, KIND))
@@ -497,8 +506,8 @@ size_t gemm_split_workspace(long long M, long long N, long long K) {
 }
 
 // run_gemm<TC_TF32> with the contraction split over CTAs when the output has few tiles; split_ws holds the partial
-// products (gemm_split_workspace bytes, 16-byte aligned).  No fused encoder epilogue in this form.  Only 128 x 128
-// tiles occur here: a split is planned only when the output has fewer tiles than the wide form needs.
+// products (gemm_split_workspace bytes, 16-byte aligned).  No fused encoder epilogue in this form.  A split product
+// always runs on 128 x 128 tiles (run_gemm looks at ksplit), whatever the number of row tiles.
 int run_gemm_tf32_split(const void *A, long long lda, const void *B, long long ldb, GemmParams p, void *split_ws,
                         cudaStream_t st) {
     int per;

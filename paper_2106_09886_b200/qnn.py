@@ -24,8 +24,8 @@ EXPORTS = [
     "qnn_mbit_encoder_backward", "qnn_bgemm_backward_data_workspace", "qnn_bgemm_backward_data",
     "qnn_bgemm_backward_weights_workspace", "qnn_bgemm_backward_weights", "qnn_bconv2d_backward_data_workspace",
     "qnn_bconv2d_backward_data", "qnn_bconv2d_backward_weights_workspace", "qnn_bconv2d_backward_weights", "qnn_unpack_codes_f32",
-    "qnn_tensor_path_status", "qnn_bgemm_int8_tensor_workspace", "qnn_bgemm_int8_tensor",
-    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy",
+    "qnn_tensor_path_status", "qnn_last_device_status", "qnn_selftest_bounded_wait", "qnn_bgemm_int8_tensor_workspace", "qnn_bgemm_int8_tensor",
+    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy", "qnn_popcounts_per_output",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -76,6 +76,10 @@ def _load() -> C.CDLL:
     lib.qnn_bconv2d_backward_weights_workspace.argtypes = [i] * 9
     lib.qnn_bconv2d_backward_weights.argtypes = [p, p, i] + [i] * 9 + [f, p, p, sz, p]
     lib.qnn_tensor_path_status.argtypes = [C.POINTER(C.c_uint)]
+    lib.qnn_last_device_status.argtypes = [C.POINTER(C.c_uint)]
+    lib.qnn_selftest_bounded_wait.argtypes = [u, p]
+    lib.qnn_popcounts_per_output.restype = i64
+    lib.qnn_popcounts_per_output.argtypes = [i] * 7
     lib.qnn_bgemm_int8_tensor_workspace.restype = sz
     lib.qnn_bgemm_int8_tensor_workspace.argtypes = [i64, i, i]
     lib.qnn_bgemm_int8_tensor.argtypes = [p, i, p, i, i64, i, i, f, p, p, p, sz, p]
@@ -367,6 +371,19 @@ def tensor_path_status() -> int:
     return st.value
 
 
+def last_device_status() -> tuple[int, int]:
+    """Synchronises; returns (return code, status word) of qnn_last_device_status without raising: (QNN_OK, 0), or
+    (QNN_E_DEVICE, 1 + id of the wait that gave up).  Reading clears the record."""
+    st = C.c_uint(0)
+    rc = lib.qnn_last_device_status(C.byref(st))
+    return rc, st.value
+
+
+def selftest_bounded_wait(poll_limit: int = 1024, stream=None) -> None:
+    """Enqueues the library's bounded-wait self-test (a wait that runs out on purpose and ends normally)."""
+    _check(lib.qnn_selftest_bounded_wait(int(poll_limit), _stream(stream)), "qnn_selftest_bounded_wait")
+
+
 def absmax_f32(x: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
     _dev(x, torch.float32, "x")
     if out is None:
@@ -427,6 +444,14 @@ def probe_bitops(variant: int, iters: int, blocks: int, sink: torch.Tensor, stre
     _check(lib.qnn_probe_bitops(variant, iters, blocks, _ptr(sink), C.byref(ops), _stream(stream)),
            "qnn_probe_bitops")
     return ops.value
+
+
+def popcounts_per_output(ab: int, wb: int, conv: bool, R: int, S: int, C: int, Cout: int) -> int:
+    """Popcount instructions per output element of the kernel that serves such a layer (FC: R = S = 1, C = Kg)."""
+    n = lib.qnn_popcounts_per_output(ab, wb, 1 if conv else 0, R, S, C, Cout)
+    if n <= 0:
+        raise QnnError(E_ARG, "qnn_popcounts_per_output")
+    return int(n)
 
 
 def probe_copy(dst: torch.Tensor, src: torch.Tensor, stream=None) -> int:

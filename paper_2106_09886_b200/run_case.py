@@ -22,12 +22,25 @@ import torch
 from . import qnn
 
 
-def _time_calls(fn, reps: int, warmup: int):
+_flush_buf = None
+
+
+def flush_l2():
+    """Writes a buffer twice the size of the L2 cache, so that the next call finds none of its data there."""
+    global _flush_buf
+    if _flush_buf is None:
+        _flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    _flush_buf.zero_()
+
+
+def _time_calls(fn, reps: int, warmup: int, flush: bool = False):
     for i in range(warmup):
         fn(i)
     torch.cuda.synchronize()
     times = []
     for i in range(reps):
+        if flush:
+            flush_l2()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn(i)
@@ -35,6 +48,25 @@ def _time_calls(fn, reps: int, warmup: int):
         e1.synchronize()
         times.append(e0.elapsed_time(e1))
     return times
+
+
+def layer_roofline(Mg, Ng, ab, wb, conv, R, S, C, in_rows, ms, popc_per_s, hbm_gbs):
+    """Roofline of one contraction launch: the slower of its algorithmic bytes at the HBM peak (packed activations of
+    the `in_rows` input rows or pixels and packed weights read once, fp32 outputs written once) and its popcount
+    instructions at the measured popcount rate (the scarce pipe; qnn_popcounts_per_output per output element)."""
+    kg = R * S * C
+    nbytes = in_rows * C * ab / 8.0 + Ng * kg * wb / 8.0 + Mg * Ng * 4.0
+    popc = qnn.popcounts_per_output(ab, wb, conv, R, S, C, Ng)
+    t_alu = Mg * Ng * popc / popc_per_s * 1e3
+    t_hbm = nbytes / (hbm_gbs * 1e9) * 1e3
+    bound = "alu" if t_alu >= t_hbm else "hbm"
+    binary = 2.0 * Mg * Ng * kg * ab * wb
+    if bound == "alu":
+        achieved, peak, unit = binary / (ms * 1e-3) / 1e12, binary / (t_alu * 1e-3) / 1e12, "binary TOPS"
+    else:
+        achieved, peak, unit = nbytes / (ms * 1e-3) / 1e9, hbm_gbs, "GB/s"
+    return {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": max(t_alu, t_hbm) / ms,
+            "roofline_ms": max(t_alu, t_hbm), "popc_per_word": popc / (ab * wb * (kg / 32.0)), "alg_bytes": nbytes}
 
 
 def time_gemm(Mg, Ng, Kg, ab, wb, reps=5, warmup=3, sets=3, dev="cuda:0", seed=0):
@@ -116,6 +148,7 @@ def time_stack(net: str, batch: int, reps=3, warmup=2, dev="cuda:0", seed=0, lay
         enc_ms, conv_ms = statistics.median(t_enc), statistics.median(t_conv)
         macs = float(s.Mg) * s.Cout * s.Kg
         rows.append({"layer": s.name, "Mg": s.Mg, "Ng": s.Cout, "Kg": s.Kg, "ab": s.ab, "wb": s.wb,
+                     "R": s.R, "S": s.S, "C": s.C, "stride": s.stride, "in_rows": s.N * s.H * s.W,
                      "encode_ms": enc_ms, "conv_ms": conv_ms, "conv_encode_ms": statistics.median(t_fused),
                      "conv_binary_tops": 2 * macs * s.ab * s.wb / (conv_ms * 1e-3) / 1e12,
                      "conv_equiv_int_gops": 2 * macs / (conv_ms * 1e-3) / 1e9,

@@ -92,6 +92,35 @@ def test_argument_errors_are_reported_before_any_launch(qnn):
     assert lib.qnn_probe_copy(p, p, 24, None) == qnn.E_ARG
 
 
+def test_composite_calls_check_every_argument_before_their_first_copy_or_launch(qnn):
+    """qnn_fc_forward_host, its pipelined form and qnn_fc_forward_noalloc wrap a copy, the encoder and the contraction:
+    an argument that only the contraction would refuse (weight width, alpha, the int32 range, a misaligned blob)
+    must come back as an error with nothing enqueued.  On a machine without a GPU a copy or launch would answer
+    QNN_E_CUDA instead, so the exact codes below also show that nothing was attempted."""
+    lib = qnn.lib
+    buf = (ctypes.c_char * 4096)()
+    p = ctypes.c_void_p((ctypes.addressof(buf) + 255) // 256 * 256)      # aligned, never dereferenced by these calls
+    mis = ctypes.c_void_p(p.value + 4)
+    streams = (ctypes.c_void_p * 2)(None, None)
+    inf, nan = float("inf"), float("nan")
+
+    def host(wb=2, alpha=1.0, Kg=64, w=p, ab=2, scale=1.0, flags=0):
+        return lib.qnn_fc_forward_host(p, 4, Kg, ab, scale, flags, w, wb, 4, alpha, p, p, p, p, None)
+
+    def piped(wb=2, alpha=1.0, Kg=64, w=p, ab=2, scale=1.0, flags=0):
+        return lib.qnn_fc_forward_host_pipelined(p, 4, Kg, ab, scale, flags, w, wb, 4, alpha, p, p, p, p, 2, streams, 2)
+
+    def noalloc(wb=2, alpha=1.0, Kg=64, w=p, ab=2, scale=1.0, flags=0):
+        return lib.qnn_fc_forward_noalloc(p, 4, Kg, Kg, ab, scale, flags, w, wb, 4, alpha, p, 4, None)
+
+    for call in (host, piped, noalloc):
+        assert call(wb=0) == qnn.E_ARG and call(wb=9) == qnn.E_ARG
+        assert call(alpha=inf) == qnn.E_SCALE and call(alpha=nan) == qnn.E_SCALE
+        assert call(ab=8, wb=8, Kg=33026) == qnn.E_RANGE                  # 33026*255*255 >= 2^31
+        assert call(w=mis) == qnn.E_ALIGN
+        assert call(scale=0.0) == qnn.E_SCALE and call(flags=2) == qnn.E_ARG and call(ab=9) == qnn.E_ARG
+
+
 def test_importing_binding_without_library_fails_loudly(tmp_path, monkeypatch):
     import importlib.util
     src = (ROOT / "paper_2106_09886_b200" / "qnn.py").read_text()

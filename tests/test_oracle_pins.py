@@ -406,6 +406,56 @@ def test_mbit_encoder_forward_is_sign_of_sine_and_matches_the_lookup_encoder(bit
     assert np.all(cz[:, 0] == 0.0) and np.all(cz[0] == 0.0)
 
 
+@pytest.mark.parametrize("bits", range(1, 9))
+def test_mbit_encoder_forward_near_crossings_against_exact_rational_arithmetic(bits):
+    """Inside the band around the zero crossings, where a float64 sine cannot be trusted to decide the sign.
+    (a) Inputs x = n / 2^16: k_m * x = A * n / 2^(m+16) has at most 24 significant bits, so the binary32 product
+        of Eq. 10's argument is exact and sign(sin(pi * k_m * x)) is decided by integer arithmetic alone: 0 when
+        2^(m+16) divides A * n, else + on (2j, 2j+1) and - on (2j+1, 2j+2).  Every n in [-2^16, 2^16] is checked,
+        which includes each crossing that is a multiple of 2^-16 and its two neighbours on that grid.
+    (b) Arbitrary binary32 inputs within 1e-3 of a crossing (the band the float64 pin leaves out), including the
+        floats adjacent to each crossing: the argument is y = fl32(k_m * fl32(x / r)) (the reading of Eq. 10's
+        precision); numpy's IEEE binary32 operations give y, fractions.Fraction decides integer / parity exactly."""
+    from fractions import Fraction
+    A = 2 ** bits - 1
+    n = np.arange(-2 ** 16, 2 ** 16 + 1, dtype=np.int64)
+    x = (n.astype(np.float64) / 2.0 ** 16).astype(np.float32)
+    assert np.array_equal(x.astype(np.float64) * 2.0 ** 16, n.astype(np.float64))
+    c = oracle.mbit_encoder_forward(x, bits)
+    for m in range(1, bits + 1):
+        num, sh = A * n, m + 16                            # k_m * x = num / 2^sh exactly
+        integer = (num & ((1 << sh) - 1)) == 0
+        odd_floor = ((num >> sh) & 1) == 1                 # arithmetic shift = floor, also for negatives
+        want = np.where(integer, 0.0, np.where(odd_floor, -1.0, 1.0))
+        if m != bits:
+            want = -want
+        assert np.array_equal(c[m - 1], want.astype(np.float32)), (bits, m)
+        # the same through fractions.Fraction, literally, on a handful of points around crossings
+        for idx in (0, 1, 2 ** 16 - 1, 2 ** 16, 2 ** 16 + 1, 2 ** 17 - 1, 2 ** 17, 12345, 77777):
+            y = Fraction(A, 2 ** m) * Fraction(float(x[idx]))
+            fl = y.numerator // y.denominator
+            sg = 0.0 if y.denominator == 1 else (1.0 if fl % 2 == 0 else -1.0)
+            assert c[m - 1][idx] == (sg if m == bits else -sg)
+    # (b) floats in the band around crossings, several ranges r
+    rng = np.random.default_rng(500 + bits)
+    for r in (1.0, 3.0, 0.37):
+        r32 = np.float32(r)
+        cross = rng.integers(-A, A + 1, size=400).astype(np.float64) * 2.0 / A * r     # crossings of the lowest plane
+        xb = (cross + rng.uniform(-1e-3, 1e-3, size=cross.size) * 2.0 / A * r).astype(np.float32)
+        xc = cross.astype(np.float32)
+        xs = np.concatenate([xb, xc, np.nextafter(xc, np.float32(np.inf)), np.nextafter(xc, np.float32(-np.inf))])
+        cb = oracle.mbit_encoder_forward(xs, bits, r)
+        xn = xs / r32                                       # binary32 division
+        for m in range(1, bits + 1):
+            k32 = np.float32(A) / np.float32(2 ** m)       # exact
+            y32 = k32 * xn                                  # binary32 product (numpy: IEEE, not the oracle's C code)
+            for e in range(0, xs.size, 7):
+                y = Fraction(float(y32[e]))
+                fl = y.numerator // y.denominator
+                sg = 0.0 if y.denominator == 1 else (1.0 if fl % 2 == 0 else -1.0)
+                assert cb[m - 1][e] == (sg if m == bits else -sg), (bits, m, r, float(xs[e]))
+
+
 @pytest.mark.parametrize("bits", [1, 2, 3, 5, 8])
 def test_mbit_encoder_backward_is_the_derivative_of_the_sine_and_zero_outside(bits):
     """Eq. 12 is the derivative of the sine inside the sign (a straight-through estimate): compare with a central

@@ -4,8 +4,9 @@ Such a caller (a framework plug-in that must not allocate in its callback, a rea
 fixed at start-up, a bare C program) passes only its input, the packed weights and its output; the
 activation planes in between live in an array built into the library.  The check: through the C ABI, its
 output equals that of the ordinary two-call route (qnn_encode_pack into a caller-allocated buffer, then
-qnn_bgemm) on two calls in a row that share the built-in array -- the second with a different, smaller
-problem, so that planes left over from the first call would show up if they leaked.
+qnn_bgemm) and the CPU oracle's result for the same layer, on two calls in a row that share the built-in
+array -- the second with a different, smaller problem, so that planes left over from the first call would
+show up if they leaked.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run every other test.
 """
@@ -13,6 +14,8 @@ import ctypes
 
 import numpy as np
 import pytest
+
+from helpers import assert_fp32_close, oracle_fc
 
 pytestmark = pytest.mark.gpu
 
@@ -50,6 +53,9 @@ def test_noalloc_entry_matches_two_call_route_twice_in_a_row():
         got = out.cpu().numpy()
         assert np.all(np.abs(got.astype(np.float64) - want) <= 1e-6 * np.abs(want.astype(np.float64)))
         assert np.array_equal(got, want)                    # same kernels, same inputs: the same bits
+        # and against the independent CPU oracle, so that a mistake common to both GPU routes cannot pass
+        _, _, _, want_oracle = oracle_fc(x, w, False, ab, wb, sa, sw, alpha, relu=bool(flags & qnn.RELU))
+        assert_fp32_close(got, want_oracle)
 
 
 def test_noalloc_entry_refuses_what_does_not_fit():
