@@ -41,6 +41,9 @@ def _time_calls(fn, reps: int, warmup: int, flush: bool = False):
     for i in range(reps):
         if flush:
             flush_l2()
+        else:
+            torch.cuda._sleep(60000)      # keeps the GPU busy (~30 us) while the host enqueues, so that the event pair
+                                          # brackets the kernel and not the host's launch latency
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         fn(i)
