@@ -3,6 +3,7 @@
 #include "qnn_internal.cuh"
 #include "bgemm_tiled.cuh"
 #include "bconv_dense.cuh"
+#include "bconv_pointwise.cuh"
 
 namespace {
 
@@ -161,6 +162,12 @@ int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int kw = (int)qnn_row_words_i(Kg);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
+    if (!ne && qnn_pointwise::applicable(ab, wb, Kg, Ng)) {          // rows of at most four words per plane
+        qnn_pointwise::Params d = {};
+        d.a = a_planes; d.w = w; d.Mg = Mg; d.Ng = Ng; d.Kg = Kg; d.a_pitch = kw; d.w_pitch = kw;
+        d.alpha = alpha; d.out = out; d.ldo = ldo; d.acc = acc; d.conv = 0;
+        return qnn_pointwise::dispatch(ab, wb, d, st);
+    }
     qnn_tiled::Params p = {};
     p.a = a_planes; p.w = w; p.tapsum = nullptr;
     p.Mg = Mg; p.Ng = Ng;
@@ -207,6 +214,14 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
+    if (!ne && dil == 1 && !transposed && R == 1 && S == 1 && pad == 0 && C >= 32 && qnn_pointwise::applicable(ab, wb, C, Cout)) {
+        // 1x1 convolution on at most 128 channels (a residual network's projections): no border, whole reduction in registers
+        qnn_pointwise::Params d = {};
+        d.a = a_planes; d.w = w; d.Mg = Mg; d.Ng = Cout; d.Kg = C; d.a_pitch = g.a_pitch; d.w_pitch = g.w_pitch;
+        d.alpha = alpha; d.out = out; d.ldo = Cout; d.acc = acc;
+        d.conv = 1; d.H = H; d.W = W; d.Ho = g.Ho; d.Wo = g.Wo; d.stride = stride;
+        return qnn_pointwise::dispatch(ab, wb, d, st);
+    }
     if (dil == 1 && !transposed && qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout)) {
         qnn_dense::Params d = {};
         d.a = a_planes; d.w = w;
@@ -258,6 +273,8 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
 extern "C" int64_t qnn_popcounts_per_output(int ab, int wb, int is_conv, int R, int S, int C, int Cout) {
     if (!qnn_bits_ok(ab) || !qnn_bits_ok(wb) || R < 1 || S < 1 || C < 1 || Cout < 1 || (!is_conv && R * S != 1)) return 0;
     const int64_t cw = (C + 31) / 32, pairs = (int64_t)ab * wb;
+    if ((!is_conv || (R == 1 && S == 1 && C >= 32)) && qnn_pointwise::applicable(ab, wb, C, Cout))
+        return qnn_pointwise::weighted_count_popcounts(ab, wb, (int)cw);          // (1x1 convolutions: when pad = 0)
     if (is_conv && qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout))
         return (ab == 4 && wb == 4) ? 10 : ((ab == 3 && wb == 3) ? 7 : pairs);
     if (is_conv && R * S == 9 && cw <= 4 && ab <= 4 && wb <= 4) return pairs * cw * 4;      // 9-word groups
