@@ -241,11 +241,13 @@ int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_planes, size_t 
  *                                 and r) applies the encoder derivative of Eq. 12 as in qnn_bgemm_backward_data.
  *   qnn_bconv2d_backward_weights  GW[co][r][s][c] = alpha * sum over the output pixels of g[n][ho][wo][co] *
  *                                 qa[n][ho*stride - pad + r][wo*stride - pad + s][c]; g_{W^j} = 2^(j-1) * GW.
- * Both run the TF32 tensor-core contraction of the fully-connected case on an explicit patch matrix held in the
- * workspace: for the weights the im2col of the activation codes ([R*S*C][N*Ho*Wo] fp32), for the data the patch
- * gradients ([N*Ho*Wo][R*S*C] fp32), which a gather then sums onto the pixels in a fixed tap order.  Error bound as
- * for the fully-connected products with contraction lengths Cout (data; plus one fp32 addition per tap) and N*Ho*Wo
- * (weights); integer-valued g with small sums is contracted exactly.
+ * Both are TF32 tensor-core contractions like the fully-connected products.  The data gradient is an implicit GEMM over
+ * (tap, output feature): the kernel gathers its operand from g itself, one shifted box per tap, so no patch matrix is
+ * ever written and each result element is a single fp32 accumulation of R*S*Cout terms; the workspace only holds the
+ * unpacked weight codes (and a row-padded copy of g when Cout is not a multiple of 4).  The weight gradient contracts g
+ * with the im2col of the activation codes, which it stages in the workspace ([R*S*C][N*Ho*Wo] fp32).  Error bound as for
+ * the fully-connected products with contraction lengths R*S*Cout (data) and N*Ho*Wo (weights); integer-valued g with
+ * small sums is contracted exactly.
  *   w_packed  blob of qnn_pack_weights(n_out = Cout, taps = R*S, c_in = C, bits = wb); a_planes [N*H*W][ab][qnn_row_words(C)]
  *   g         device fp32, 16-byte aligned for backward_data (4-byte for backward_weights)
  *   out / gw  device fp32 [N][H][W][C] / [Cout][R][S][C]

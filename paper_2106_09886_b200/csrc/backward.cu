@@ -7,10 +7,10 @@
 // (tcgen05.mma, kind::tf32, accumulator in tensor memory), fed by TMA through a ring of mbarrier-guarded stages.
 // The integer codes (|q| <= 255) are exact in TF32; the gradient keeps 11 significant bits per element.
 // Bound: tensor pipe (2*M*N*K flop per call).
-// A convolution goes through the same GEMM on an explicit patch matrix: the weight gradient contracts g with the
-// im2col of the activation codes (unpacked straight from the planes into K-major order), the data gradient
-// multiplies g by the weight codes and gathers the patch gradients back onto the pixels (a gather, not a scatter
-// with atomics, so the fp32 sums have a fixed order).
+// A convolution goes through the same GEMM: the weight gradient contracts g with the im2col of the activation codes
+// (unpacked straight from the planes into K-major order); the data gradient is an implicit GEMM over (tap, output
+// feature) whose A operand the TMA unit gathers from g itself, one shifted 4-D box per tap (see ConvGather in
+// tc_gemm.cuh), so no patch matrix exists and every result pixel is one fp32 accumulation in tensor memory.
 #include "tc_gemm.cuh"
 
 namespace {
@@ -169,58 +169,6 @@ __global__ void __launch_bounds__(256) conv_weights_t_kernel(const uint32_t *__r
     }
 }
 
-// Gathers the patch gradients back onto the input pixels: out[n][h][w][c] = sum over the taps (r, s) and output pixels
-// (ho, wo) with ho*st - pad + r = h and wo*st - pad + s = w of dcol[(n, ho, wo)][(r*S + s)*C + c], taps in
-// increasing (r, s) order (a gather, so the sum has a fixed order).  BITS > 0: the encoder derivative of Eq. 12 is
-// applied to the sum (x = what the previous layer fed its encoder, as in qnn_bgemm_backward_data).
-// One thread per pixel and VEC consecutive channels (VEC = 4 when C is a multiple of 4: 16-byte accesses, a quarter of
-// the index arithmetic); the tap loops run in 32-bit arithmetic, only the row offset into dcol is 64-bit.
-template <int BITS, int VEC>
-__global__ void __launch_bounds__(256) conv_col2im_kernel(const float *__restrict__ dcol, ConvGeom g, const float *__restrict__ x,
-                                                         float r_range, MbitPlaneConsts enc, float *__restrict__ out) {
-    const int cv = g.C / VEC;                                          // channel groups per pixel
-    const long long total = (long long)g.N * g.H * g.W * cv;
-    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
-        const long long pix = i / cv;
-        const int c = (int)(i - pix * cv) * VEC;
-        const long long nh = pix / g.W;
-        const int w = (int)(pix - nh * g.W);
-        const long long n = nh / g.H;
-        const int h = (int)(nh - n * g.H);
-        float sum[VEC];
-#pragma unroll
-        for (int v = 0; v < VEC; ++v) sum[v] = 0.0f;
-        for (int r = 0; r < g.R; ++r) {
-            const int th = h + g.pad - r;
-            if (th < 0) break;                                         // larger r only moves further up
-            const int ho = th / g.stride;
-            if (ho * g.stride != th || ho >= g.Ho) continue;
-            const long long rowbase = (n * g.Ho + ho) * g.Wo;
-            for (int sx = 0; sx < g.S; ++sx) {
-                const int tw = w + g.pad - sx;
-                if (tw < 0) break;
-                const int wo = tw / g.stride;
-                if (wo * g.stride != tw || wo >= g.Wo) continue;
-                const float *src = dcol + (rowbase + wo) * g.Kg + (r * g.S + sx) * g.C + c;
-                if (VEC == 4) {
-                    const float4 d = __ldcs(reinterpret_cast<const float4 *>(src));
-                    sum[0] = __fadd_rn(sum[0], d.x); sum[1 % VEC] = __fadd_rn(sum[1 % VEC], d.y);
-                    sum[2 % VEC] = __fadd_rn(sum[2 % VEC], d.z); sum[3 % VEC] = __fadd_rn(sum[3 % VEC], d.w);
-                } else {
-                    sum[0] = __fadd_rn(sum[0], __ldcs(src));
-                }
-            }
-        }
-        const long long o = pix * g.C + c;
-        if constexpr (BITS > 0) {
-#pragma unroll
-            for (int v = 0; v < VEC; ++v) sum[v] = mbit_backward_shared<BITS>(__ldg(x + o + v), r_range, sum[v], enc);
-        }
-        if (VEC == 4) *reinterpret_cast<float4 *>(out + o) = make_float4(sum[0], sum[1 % VEC], sum[2 % VEC], sum[3 % VEC]);
-        else out[o] = sum[0];
-    }
-}
-
 bool conv_geom(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad, ConvGeom *g) {
     if (N < 1 || H < 1 || W < 1 || C < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0) return false;
     const long long Ho = ((long long)H + 2 * pad - R) / stride + 1, Wo = ((long long)W + 2 * pad - S) / stride + 1;
@@ -342,7 +290,7 @@ extern "C" size_t qnn_bconv2d_backward_data_workspace(int N, int H, int W, int C
     ConvGeom g;
     if (!conv_geom(N, H, W, C, Cout, R, S, stride, pad, &g) || !conv_backward_dims_ok(g)) return 0;
     const size_t ldn = (size_t)pad32(Cout);
-    return round256((size_t)g.Kg * ldn * 4) + (Cout % 4 ? round256((size_t)g.Mg * ldn * 4) : 0) + round256((size_t)g.Mg * g.Kg * 4);
+    return round256((size_t)g.Kg * ldn * 4) + (Cout % 4 ? round256((size_t)g.Mg * ldn * 4) : 0);
 }
 
 extern "C" int qnn_bconv2d_backward_data(const float *g, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
@@ -384,30 +332,14 @@ extern "C" int qnn_bconv2d_backward_data(const float *g, const void *w_packed, i
         a = gp;
         lda = ldn;
     }
-    float *dcol = reinterpret_cast<float *>(ws);                        // [Mg][Kg]: gradient of every patch element
     GemmParams p{};
-    p.M = (int)cg.Mg; p.N = (int)cg.Kg; p.K = Cout;
     p.alpha = alpha;
-    p.C = dcol; p.ldc = cg.Kg;
+    p.C = out; p.ldc = C;
+    p.x = x; p.ldx = C; p.bits = ab; p.r = r;
+    if (x) p.enc = mbit_plane_consts(ab);
     if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
-    if ((rc = run_gemm<TC_TF32>(a, lda, wqt, ldn, p, st)) != QNN_OK) return rc;
-    // 16-byte accesses need C % 4 == 0 (then every patch row, R*S*C floats, and every pixel start on 16-byte
-    // boundaries of the 256-byte aligned workspace) and a 16-byte aligned output
-    const bool vec4 = C % 4 == 0 && qnn_aligned(out, 16);
-    const long long total = (long long)N * H * W * (vec4 ? C / 4 : C);
-    const int blocks = (int)(qnn_ceil_div(total, 256) < 148 * 64 ? qnn_ceil_div(total, 256) : 148 * 64);
-    MbitPlaneConsts enc = x ? mbit_plane_consts(ab) : MbitPlaneConsts{};
-#define CONV_C2I_CASE(B)                                                                          \
-    case B:                                                                                       \
-        if (vec4) conv_col2im_kernel<B, 4><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out);     \
-        else conv_col2im_kernel<B, 1><<<blocks, 256, 0, st>>>(dcol, cg, x, r, enc, out);          \
-        break;
-    switch (x ? ab : 0) {
-        CONV_C2I_CASE(0) CONV_C2I_CASE(1) CONV_C2I_CASE(2) CONV_C2I_CASE(3) CONV_C2I_CASE(4) CONV_C2I_CASE(5) CONV_C2I_CASE(6)
-        CONV_C2I_CASE(7) CONV_C2I_CASE(8)
-    }
-#undef CONV_C2I_CASE
-    return qnn_launch_status();
+    // implicit gather: the tensor cores read shifted boxes of g and the tap's weight codes; no patch matrix
+    return run_conv_data_gradient(a, lda, wqt, ldn, N, H, W, C, Cout, R, S, stride, pad, cg.Ho, cg.Wo, p, st);
 }
 
 extern "C" size_t qnn_bconv2d_backward_weights_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride,

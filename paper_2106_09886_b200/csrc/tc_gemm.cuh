@@ -64,6 +64,19 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, u
         : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int x, int y, int z, int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -136,6 +149,22 @@ constexpr int MMA_K_BYTES = 32;         // bytes of K one instruction consumes (
 constexpr int EPI_WARPS = 8;            // two warps per quarter of the tensor-memory lanes, alternating 32-column chunks
 constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;   // warp 0: TMA producer, warp 1: MMA issuer + tensor-memory owner
 
+// Data gradient of a convolution as an implicit GEMM (no patch matrix in memory): result pixel (n, h, w) sums, over the
+// taps (r, s) that reach it and over the output features co, g[n][(h + pad - r)/st][(w + pad - s)/st][co] * qw[co][r][s][c].
+// Pixels are taken one stride class (h mod st, w mod st) at a time, because all pixels of a class are reached by the
+// same taps; the 128 rows of a tile are bn images x bh x bw pixels of the class (powers of two), so that the A operand of
+// one (tap, block of 32 features) is ONE 4-D box of g, shifted by the tap; the tensor map fills what lies outside g with
+// zeros, which is exactly the contribution of a tap that reaches no output.  B is the tap's weight codes [c][co].
+struct ConvGather {
+    int enabled;
+    int st, pad, R, S;
+    int H, W;                           // result (= layer input) image
+    int log_bw, log_bh, log_bn;         // tile = 2^log_bn images x 2^log_bh x 2^log_bw pixels of a class
+    int tiles_w, tiles_h, tiles_nb;     // tiles per class along w, h and the batch
+    int coblocks;                       // blocks of 32 output features (the contraction within a tap)
+    int n_images;
+};
+
 struct GemmParams {
     int M, N, K;                        // C[M][N] = alpha * sum_k A[M][K] * B[N][K]
     float alpha;
@@ -156,7 +185,49 @@ struct GemmParams {
     int ksplit, kb_per_split;
     long long split_stride;
     unsigned int wait_limit;            // polls after which a wait on an arrival gives up (0 = WAIT_LIMIT)
+    ConvGather conv;                    // enabled: A is gathered from the gradient image, rows of C are pixels (see above)
 };
+
+// floor(a / b) and whether b divides a, for b > 0 and any sign of a
+__device__ __forceinline__ bool exact_div(int a, int b, int &q) {
+    q = a >= 0 ? a / b : -((-a + b - 1) / b);
+    return q * b == a;
+}
+
+// One tile of the convolution's data gradient: stride class, first image / class row / class column, channel tile.
+struct ConvTile {
+    int ph, pw, n0, a0, b0, c0;
+    int nkb;                            // K blocks: (taps of the class) x coblocks
+};
+template <int BN>
+__device__ __forceinline__ ConvTile conv_tile(int tile, const GemmParams &p) {
+    const ConvGather &c = p.conv;
+    ConvTile t;
+    const int ct = tile % p.tiles_n;
+    int mt = tile / p.tiles_n;
+    t.c0 = ct * BN;
+    const int wb = mt % c.tiles_w; mt /= c.tiles_w;
+    const int hb = mt % c.tiles_h; mt /= c.tiles_h;
+    const int nb = mt % c.tiles_nb; mt /= c.tiles_nb;
+    t.pw = mt % c.st;
+    t.ph = mt / c.st;
+    t.b0 = wb << c.log_bw; t.a0 = hb << c.log_bh; t.n0 = nb << c.log_bn;
+    int th = 0, tw = 0, q;
+    for (int r = 0; r < c.R; ++r) th += exact_div(t.ph + c.pad - r, c.st, q) ? 1 : 0;
+    for (int s = 0; s < c.S; ++s) tw += exact_div(t.pw + c.pad - s, c.st, q) ? 1 : 0;
+    t.nkb = th * tw * c.coblocks;
+    return t;
+}
+// Offset (in rows of C / x) of tile row `row`, or -1 when the row lies outside the image or the batch.
+__device__ __forceinline__ long long conv_row(const ConvTile &t, int row, const GemmParams &p) {
+    const ConvGather &c = p.conv;
+    const int dw = row & ((1 << c.log_bw) - 1);
+    const int dh = (row >> c.log_bw) & ((1 << c.log_bh) - 1);
+    const int dn = row >> (c.log_bw + c.log_bh);
+    const int n = t.n0 + dn, h = (t.a0 + dh) * c.st + t.ph, w = (t.b0 + dw) * c.st + t.pw;
+    if (n >= c.n_images || h >= c.H || w >= c.W) return -1;
+    return ((long long)n * c.H + h) * c.W + w;
+}
 
 // One column of a 32 x 32 chunk (this lane's), rows_here rows: C = Eq. 12 applied to the staged products and x.
 // Four rows are in flight at a time; the element arithmetic has no branch, so their instructions interleave.
@@ -176,6 +247,20 @@ __device__ __forceinline__ void epilogue_encoder(float *cptr, long long ldc, con
     }
     for (; rr < rows_here; ++rr)
         cptr[(long long)rr * ldc] = mbit_backward_shared<BITS>(__ldcs(xptr + (long long)rr * ldx), r, stage_col[rr * 33], c);
+}
+
+// Convolution data gradient: one column (this lane's) of a 32 x 32 chunk whose rows are tile rows row0 .. row0 + 31;
+// BITS > 0 applies Eq. 12 with x read at the same pixel.
+template <int BITS>
+__device__ __forceinline__ void conv_epilogue_rows(const ConvTile &t, int row0, const GemmParams &p, int col, const float *stage_col) {
+#pragma unroll 4
+    for (int rr = 0; rr < 32; ++rr) {
+        const long long pix = conv_row(t, row0 + rr, p);
+        if (pix < 0) continue;
+        float v = t.nkb ? stage_col[rr * 33] : 0.0f;      // a stride class that no tap reaches: nothing was accumulated
+        if constexpr (BITS > 0) v = mbit_backward_shared<BITS>(__ldcs(p.x + pix * p.ldx + col), p.r, v, p.enc);
+        p.C[pix * p.ldc + col] = v;
+    }
 }
 
 // Work item w of a launch: whole tiles first; the tiles of a ragged last round (fewer than half as many as there are
@@ -256,34 +341,61 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
     if (warp == 0) {
         if (lane == 0) {
             long long it = 0;                                 // stage uses so far, over all tiles
+            int s = 0;                                        // ring position it % STAGES and parity of it / STAGES, kept
+            uint32_t ph = 0;                                  // incrementally (this one thread's instructions are the pace)
+            auto advance = [&]() {
+                ++it;
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            };
             for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x) {
+                if (KIND == TC_TF32 && p.conv.enabled) {
+                    // implicit gather: per tap of the tile's stride class and block of 32 output features, one 4-D box
+                    // of the gradient image shifted by the tap (zero outside it) and the tap's weight codes
+                    const ConvTile t = conv_tile<BN>(w, p);
+                    for (int r = 0; r < p.conv.R && !*abort_flag; ++r) {
+                        int dr, ds;
+                        if (!exact_div(t.ph + p.conv.pad - r, p.conv.st, dr)) continue;
+                        for (int sx = 0; sx < p.conv.S && !*abort_flag; ++sx) {
+                            if (!exact_div(t.pw + p.conv.pad - sx, p.conv.st, ds)) continue;
+                            const int tap = r * p.conv.S + sx, wx = t.b0 + ds, hy = t.a0 + dr;
+                            for (int cb = 0; cb < p.conv.coblocks; ++cb) {
+                                if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err, p.wait_limit)) break;
+                                mbar_expect_tx(&full[s], L::STAGE_BYTES);
+                                tma_load_4d(smem + s * L::STAGE_BYTES, &map_a, &full[s], cb * BK, wx, hy, t.n0);
+                                tma_load_3d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], cb * BK, t.c0, tap);
+                                advance();
+                            }
+                        }
+                    }
+                    continue;
+                }
                 const WorkItem wi = work_item<BN>(w, p, nkb);
                 const bool whole = wi.width == BN;
-                for (int kb = wi.kb0; kb < wi.kb1; ++kb, ++it) {
-                    const int s = (int)(it % STAGES);
-                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                for (int kb = wi.kb0; kb < wi.kb1; ++kb) {
                     if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err, p.wait_limit)) break;
                     mbar_expect_tx(&full[s], whole ? L::STAGE_BYTES : L::A_BYTES + L::B_BYTES / 2);
                     tma_load_2d(smem + s * L::STAGE_BYTES, &map_a, &full[s], kb * BK, wi.m0);
                     tma_load_2d(smem + s * L::STAGE_BYTES + L::A_BYTES, whole ? &map_b : &map_b_half, &full[s], kb * BK, wi.n0);
+                    advance();
                 }
             }
             if (*abort_flag) drain_copies_in_flight(full, it, STAGES, p.wait_limit);
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            long long it = 0;
+            int s = 0;                                        // ring position and phase, as in the producer
+            uint32_t ph = 0;
             int local = 0;
             for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x, ++local) {
-                const WorkItem wi = work_item<BN>(w, p, nkb);
+                WorkItem wi;
+                if (KIND == TC_TF32 && p.conv.enabled) wi = WorkItem{0, 0, BN, 0, conv_tile<BN>(w, p).nkb, 0};
+                else wi = work_item<BN>(w, p, nkb);
                 const uint32_t idesc = wi.width == BN ? idesc_kmajor<BN, KIND>() : idesc_kmajor<BN / 2, KIND>();
                 const int buf = local & 1;
                 if (!mbar_wait(&acc_empty[buf], ((uint32_t)(local >> 1) & 1u) ^ 1u, abort_flag, 3, p.err, p.wait_limit)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = wi.kb0; kb < wi.kb1; ++kb, ++it) {
-                    const int s = (int)(it % STAGES);
-                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                for (int kb = wi.kb0; kb < wi.kb1; ++kb) {
                     if (!mbar_wait(&full[s], ph, abort_flag, 1, p.err, p.wait_limit)) break;
                     tc_fence_after();
                     const uint64_t a_desc = smem_desc_k_sw128(smem_u32(smem + s * L::STAGE_BYTES));
@@ -292,6 +404,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     for (int j = 0; j < BK_BYTES / MMA_K_BYTES; ++j)   // 32 bytes along K per step = 2 descriptor address units
                         tc_mma<KIND>(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, ((kb - wi.kb0) | j) != 0 ? 1u : 0u);
                     tc_commit(&empty[s]);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 tc_commit(&acc_full[buf]);
                 committed = local + 1;
@@ -302,7 +415,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
         const int half = (warp - 2) >> 2;                  // which of the two warps of this quarter
         int local = 0;
         for (int w = blockIdx.x; w < p.items; w += gridDim.x, ++local) {
-            const WorkItem wi = work_item<BN>(w, p, nkb);
+            const bool conv = KIND == TC_TF32 && p.conv.enabled;
+            ConvTile ct = {};
+            WorkItem wi;
+            if (conv) {
+                ct = conv_tile<BN>(w, p);
+                wi = WorkItem{0, ct.c0, BN, 0, ct.nkb, 0};
+            } else {
+                wi = work_item<BN>(w, p, nkb);
+            }
             const int m0 = wi.m0, n0 = wi.n0;
             const int buf = local & 1;
             // every lane polls (each needs the barrier's acquire), but the warp must reach the warp-wide
@@ -338,7 +459,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
 #pragma unroll
                     for (int i = 0; i < 32; ++i) stage[lane * 33 + i] = __fmul_rn(__uint_as_float(v[i]), p.alpha);
                     __syncwarp();
-                    if (col < p.N) {
+                    if (conv) {
+                        // rows of the tile are pixels of a stride class: each row has its own place in the result
+                        if (col < p.N) {
+                            switch (p.x ? p.bits : 0) {
+                                case 0: conv_epilogue_rows<0>(ct, q * 32, p, col, stage + lane); break;
+                                case 1: conv_epilogue_rows<1>(ct, q * 32, p, col, stage + lane); break;
+                                case 2: conv_epilogue_rows<2>(ct, q * 32, p, col, stage + lane); break;
+                                case 3: conv_epilogue_rows<3>(ct, q * 32, p, col, stage + lane); break;
+                                case 4: conv_epilogue_rows<4>(ct, q * 32, p, col, stage + lane); break;
+                                case 5: conv_epilogue_rows<5>(ct, q * 32, p, col, stage + lane); break;
+                                case 6: conv_epilogue_rows<6>(ct, q * 32, p, col, stage + lane); break;
+                                case 7: conv_epilogue_rows<7>(ct, q * 32, p, col, stage + lane); break;
+                                default: conv_epilogue_rows<8>(ct, q * 32, p, col, stage + lane); break;
+                            }
+                        }
+                    } else if (col < p.N) {
                         float *cptr = p.C + (long long)wi.split * p.split_stride + (long long)(m0 + q * 32) * p.ldc + col;
                         if (p.x) {
                             const float *xptr = p.x + (long long)(m0 + q * 32) * p.ldx + col;
@@ -415,6 +551,25 @@ bool make_map(CUtensorMap *map, const void *base, long long rows, long long cols
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of an fp32 tensor of `rank` dimensions (innermost first): dims in elements, strides of dimensions 1.. in
+// elements, box = 32 elements (128 bytes) x box[1..], 128-byte swizzle, zero fill outside the tensor.
+bool make_map_nd(CUtensorMap *map, const void *base, int rank, const long long *dims, const long long *strides_elems,
+                 const int *box) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || rank < 2 || rank > 5) return false;
+    cuuint64_t d[5], st[4];
+    cuuint32_t b[5], es[5];
+    for (int i = 0; i < rank; ++i) {
+        d[i] = (cuuint64_t)dims[i];
+        b[i] = (cuuint32_t)box[i];
+        es[i] = 1;
+        if (i > 0) st[i - 1] = (cuuint64_t)strides_elems[i - 1] * 4u;
+    }
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<void *>(base), d, st, b, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 long long pad32(long long v) { return (v + 31) / 32 * 32; }
 
 template <int BN, int STAGES, int KIND>
@@ -438,7 +593,7 @@ int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtens
     } else {
         p.ksplit = 1;
         const int rem = p.tiles % grid;
-        const bool split = rem > 0 && 2 * rem <= grid;
+        const bool split = !p.conv.enabled && rem > 0 && 2 * rem <= grid;
         p.whole_items = split ? p.tiles - rem : p.tiles;
         p.items = split ? p.tiles + rem : p.tiles;
     }
@@ -472,6 +627,60 @@ int run_gemm(const void *A, long long lda, const void *B, long long ldb, GemmPar
         return QNN_E_CUDA;
     return wide ? launch_gemm<256, 4, KIND>(map_a, map_b, map_b_half, p, sms, st)
                 : launch_gemm<128, 6, KIND>(map_a, map_b, map_b_half, p, sms, st);
+}
+
+int ceil_log2(long long v) {
+    int l = 0;
+    while ((1ll << l) < v) ++l;
+    return l;
+}
+
+// Data gradient of a convolution (see ConvGather): result[n][h][w][c] = alpha * sum over taps and co of
+// g[n][(h + pad - r)/st][(w + pad - s)/st][co] * wq[r*S + s][c][co], optionally through Eq. 12 (p.x, p.bits, p.r, p.enc).
+//   g    fp32 [N][Ho][Wo][ldg] (ldg >= Cout, a multiple of 4), 16-byte aligned
+//   wq   fp32 [R*S][C][ldw]    (ldw >= Cout, a multiple of 4), 16-byte aligned: the weight codes, tap-major
+// p carries alpha, C (the result, ldc), x / ldx / bits / r / enc and err; the rest is filled in here.
+int run_conv_data_gradient(const float *g, long long ldg, const float *wq, long long ldw, int N, int H, int W, int C, int Cout,
+                           int R, int S, int stride, int pad, int Ho, int Wo, GemmParams p, cudaStream_t st) {
+    if (!p.err || !qnn_aligned(g, 16) || !qnn_aligned(wq, 16) || ldg % 4 || ldw % 4) return QNN_E_ALIGN;
+    const int sms = sm_count();
+    if (sms <= 0) return QNN_E_CUDA;
+    // tile = 2^bn images x 2^bh x 2^bw pixels of one stride class (128 rows): the shape that wastes the fewest rows,
+    // among equals the one with the longest runs along w, then h (measured: the shape itself does not change the time)
+    const long long Wa = (W + stride - 1) / stride, Ha = (H + stride - 1) / stride;
+    int best_bw = 0, best_bh = 0;
+    double best = -1.0;
+    for (int lw = 7; lw >= 0; --lw)
+        for (int lh = 7 - lw; lh >= 0; --lh) {
+            const int ln = 7 - lw - lh;
+            const double e = (double)Wa / (double)(((Wa + (1 << lw) - 1) >> lw) << lw) *
+                             (double)Ha / (double)(((Ha + (1 << lh) - 1) >> lh) << lh) *
+                             (double)N / (double)((((long long)N + (1 << ln) - 1) >> ln) << ln);
+            if (e > best + 1e-9) { best = e; best_bw = lw; best_bh = lh; }
+        }
+    ConvGather &c = p.conv;
+    c.enabled = 1; c.st = stride; c.pad = pad; c.R = R; c.S = S; c.H = H; c.W = W; c.n_images = N;
+    c.log_bw = best_bw; c.log_bh = best_bh; c.log_bn = 7 - best_bw - best_bh;
+    c.tiles_w = (int)((Wa + (1 << c.log_bw) - 1) >> c.log_bw);
+    c.tiles_h = (int)((Ha + (1 << c.log_bh) - 1) >> c.log_bh);
+    c.tiles_nb = (int)(((long long)N + (1 << c.log_bn) - 1) >> c.log_bn);
+    c.coblocks = (Cout + 31) / 32;
+    const long long mtiles = (long long)stride * stride * c.tiles_nb * c.tiles_h * c.tiles_w;
+    if (mtiles * BM > 0x7FFFFFFFll) return QNN_E_RANGE;
+    p.M = (int)(mtiles * BM); p.N = C; p.K = 0;
+    p.ksplit = 1;
+    // tile width: the narrowest of 64 / 128 / 256 channels that covers C (256 only when that still gives every SM a
+    // tile); columns beyond C would be multiplied for nothing
+    const int bn = C <= 64 ? 64 : ((C <= 128 || mtiles * ((C + 255) / 256) < sms) ? 128 : 256);
+    const long long gdims[4] = {Cout, Wo, Ho, N}, gstr[3] = {ldg, (long long)Wo * ldg, (long long)Ho * Wo * ldg};
+    const int gbox[4] = {32, 1 << c.log_bw, 1 << c.log_bh, 1 << c.log_bn};
+    const long long wdims[3] = {Cout, C, (long long)R * S}, wstr[2] = {ldw, (long long)C * ldw};
+    const int wbox[3] = {32, bn, 1};
+    CUtensorMap map_a, map_b;
+    if (!make_map_nd(&map_a, g, 4, gdims, gstr, gbox) || !make_map_nd(&map_b, wq, 3, wdims, wstr, wbox)) return QNN_E_CUDA;
+    return bn == 256 ? launch_gemm<256, 4, TC_TF32>(map_a, map_b, map_b, p, sms, st)
+         : bn == 128 ? launch_gemm<128, 6, TC_TF32>(map_a, map_b, map_b, p, sms, st)
+                     : launch_gemm<64, 8, TC_TF32>(map_a, map_b, map_b, p, sms, st);
 }
 
 // C[i][j] = sum over s (in increasing order: a fixed summation order) of part[s][i][j]; dense partial buffers [M][N].

@@ -1,12 +1,14 @@
-"""GPU parity of the backward products of a convolution layer (Algorithm 1 backward; TF32 tensor-core contractions
-on an explicit patch matrix) against the CPU oracle.
+"""GPU parity of the backward products of a convolution layer (Algorithm 1 backward; TF32 tensor-core contractions:
+the data gradient as an implicit GEMM whose operand the TMA unit gathers from the gradient image, the weight gradient
+on staged activation codes) against the CPU oracle.
 
 Tolerance, element by element, as for the fully-connected products:
-    |got - want| <= alpha * sum |g| * |q| * (2^-10 + (L + T) * 2^-24)
-over the terms of that element's sum, with L the contraction length on the tensor cores (Cout for the data gradient,
-N*Ho*Wo for the weight gradient) and T = R*S the fp32 additions of the gather that follows (data gradient only).
+    |got - want| <= alpha * sum |g| * |q| * (2^-10 + L * 2^-24)
+over the terms of that element's sum, with L the contraction length on the tensor cores (R*S*Cout for the data
+gradient: taps and output features are one accumulation; N*Ho*Wo for the weight gradient).
 Integer-valued g with alpha a power of two is contracted exactly and compared with ==, which pins every index of the
-patch staging, the tap-major weight layout and the gather independently of rounding."""
+gather (stride classes, tap shifts, zero fill outside the gradient image), of the tap-major weight layout and of the
+tile-row-to-pixel mapping independently of rounding."""
 import numpy as np
 import pytest
 
@@ -17,7 +19,10 @@ pytestmark = pytest.mark.gpu
 
 # (N, H, W, C, Cout, R, S, stride, pad): ragged channel counts, strides, 1x1, a 5x5, Cout % 4 != 0 (padded copy of g)
 GEOMS = [(2, 6, 5, 3, 4, 3, 3, 1, 1), (1, 9, 9, 40, 6, 3, 3, 2, 1), (3, 8, 8, 64, 16, 1, 1, 2, 0), (2, 7, 6, 33, 5, 5, 5, 1, 2),
-         (2, 14, 14, 128, 32, 3, 3, 1, 1), (1, 5, 4, 70, 130, 3, 2, 1, 0), (5, 12, 12, 16, 24, 3, 3, 2, 2)]
+         (2, 14, 14, 128, 32, 3, 3, 1, 1), (1, 5, 4, 70, 130, 3, 2, 1, 0), (5, 12, 12, 16, 24, 3, 3, 2, 2),
+         # stride 3 with a 5 x 4 kernel (nine stride classes with different tap sets), a wide image (several tiles along
+         # w), many images of 7 x 7 (tiles that span images), more than 256 channels (several channel tiles)
+         (2, 11, 10, 8, 12, 5, 4, 3, 2), (1, 3, 150, 16, 8, 3, 3, 1, 1), (37, 7, 7, 24, 40, 3, 3, 1, 1), (2, 6, 6, 300, 20, 3, 3, 2, 1)]
 
 
 def _codes(rng, shape, bits):
@@ -114,7 +119,7 @@ def test_conv_backward_within_tf32_bound(geom, ab, wb):
     Mg = g.shape[0] * g.shape[1] * g.shape[2]
     mag_d = oracle.conv_backward_data(np.abs(g), np.full_like(qw, 2 ** wb - 1), (H, W), stride, pad, 1, wb, alpha)[0]
     mag_w = oracle.conv_backward_weights(np.abs(g), np.full_like(qa, 2 ** ab - 1), (R, S), stride, pad, ab, 1, alpha)[0]
-    bd = mag_d * (2.0 ** -10 + (Cout + R * S) * 2.0 ** -24)
+    bd = mag_d * (2.0 ** -10 + Cout * R * S * 2.0 ** -24)
     bw = mag_w * (2.0 ** -10 + Mg * 2.0 ** -24)
     for p in range(ab):
         assert np.all(np.abs(2.0 ** p * G.astype(np.float64) - ga[p]) <= 2.0 ** p * bd * (1 + 2.0 ** -20) + 1e-30)
