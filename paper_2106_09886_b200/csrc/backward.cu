@@ -169,6 +169,63 @@ __global__ void __launch_bounds__(256) conv_weights_t_kernel(const uint32_t *__r
     }
 }
 
+// Gradient image g[n][ho][wo][co] -> gt[co][n][ho][wp] (pixel-contiguous, rows padded with zeros from Wo to Wp columns):
+// the K-major A operand of the implicit weight gradient.  One block = 32 features x 32 columns of one image row, through
+// a 32 x 33 shared tile (both sides coalesced).
+__global__ void __launch_bounds__(256) conv_g_t_kernel(const float *__restrict__ g, int Cout, int Wo, long long Wp,
+                                                      long long rows /* N*Ho */, float *__restrict__ gt) {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const long long row = blockIdx.x;
+    const int c0 = blockIdx.y * 32, w0 = blockIdx.z * 32;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int wo = w0 + ty + 8 * i, co = c0 + tx;
+        tile[ty + 8 * i][tx] = (wo < Wo && co < Cout) ? g[(row * Wo + wo) * Cout + co] : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int co = c0 + ty + 8 * i;
+        const long long wp = w0 + tx;
+        if (co < Cout && wp < Wp) gt[((long long)co * rows + row) * Wp + wp] = tile[tx][ty + 8 * i];
+    }
+}
+
+// Activation planes -> S shifted copies of the transposed codes with the padding rows in place:
+// qas[s][c][n][hq][j] = qa[n][hq - pad][j - pad + s][c] for hq - pad inside the image, j < Wo and a column inside the
+// image, else 0; hq = 0 .. Hq - 1 = H + 2*pad - 1, j = 0 .. Wq - 1 (the B operand of the implicit weight gradient of a
+// stride-1 convolution).  One thread per (n, hq, j) and (s, channel word): consecutive threads write consecutive j.
+template <int BITS>
+__global__ void __launch_bounds__(256) conv_codes_shift_kernel(const uint32_t *__restrict__ planes, long long a_pitch, ConvGeom g,
+                                                              int Hq, int Wq, float *__restrict__ qas) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long rows_total = (long long)g.N * Hq;
+    if (idx >= rows_total * Wq) return;
+    const long long row = idx / Wq;                       // (n, hq)
+    const int j = (int)(idx - row * Wq);
+    const long long n = row / Hq;
+    const int h = (int)(row - n * Hq) - g.pad;
+    const int s = blockIdx.y / g.cw, cwi = blockIdx.y % g.cw;
+    const int wi = j - g.pad + s;
+    const bool inside = h >= 0 && h < g.H && j < g.Wo && wi >= 0 && wi < g.W;
+    uint32_t w[BITS];
+#pragma unroll
+    for (int b = 0; b < BITS; ++b)
+        w[b] = inside ? __ldg(planes + (((n * g.H + h) * g.W + wi) * BITS + b) * a_pitch + cwi) : 0u;
+    const float amax = (float)((1 << BITS) - 1);
+    const int ncol = min(32, g.C - cwi * 32);
+    const long long cstride = rows_total * Wq;
+    float *o = qas + ((long long)s * g.C + cwi * 32) * cstride + idx;
+#pragma unroll 8
+    for (int c = 0; c < 32; ++c) {
+        int t = 0;
+#pragma unroll
+        for (int b = 0; b < BITS; ++b) t |= (int)((w[b] >> c) & 1u) << b;
+        if (c < ncol) o[c * cstride] = inside ? (float)(2 * t) - amax : 0.0f;
+    }
+}
+
 bool conv_geom(int N, int H, int W, int C, int Cout, int R, int S, int stride, int pad, ConvGeom *g) {
     if (N < 1 || H < 1 || W < 1 || C < 1 || Cout < 1 || R < 1 || S < 1 || stride < 1 || pad < 0) return false;
     const long long Ho = ((long long)H + 2 * pad - R) / stride + 1, Wo = ((long long)W + 2 * pad - S) / stride + 1;
@@ -342,10 +399,25 @@ extern "C" int qnn_bconv2d_backward_data(const float *g, const void *w_packed, i
     return run_conv_data_gradient(a, lda, wqt, ldn, N, H, W, C, Cout, R, S, stride, pad, cg.Ho, cg.Wo, p, st);
 }
 
+// The weight gradient of a stride-1 convolution runs as an implicit GEMM on the transposed gradient and S shifted copies
+// of the transposed codes (about 1 + S times the size of the layer's tensors instead of R*S times); other strides stage
+// the whole patch matrix.
+static bool wgrad_implicit(const ConvGeom &g) {
+    const long long Wq = ((long long)g.Wo + 3) / 4 * 4, Hq = (long long)g.H + 2 * g.pad;
+    return g.stride == 1 && (long long)g.N * g.Ho <= 0x7FFFFFFFll && Wq <= 65535 * 32 && (long long)g.S * g.cw <= 65535 &&
+           (long long)g.N * Hq * Wq <= (1ll << 36) && Wq * Hq * g.N * (long long)g.C < (1ll << 36) &&
+           Wq * g.Ho * g.N * (long long)g.Cout < (1ll << 36);
+}
+
 extern "C" size_t qnn_bconv2d_backward_weights_workspace(int N, int H, int W, int C, int Cout, int R, int S, int stride,
                                                          int pad) {
     ConvGeom g;
     if (!conv_geom(N, H, W, C, Cout, R, S, stride, pad, &g) || !conv_backward_dims_ok(g)) return 0;
+    if (wgrad_implicit(g)) {
+        const size_t Wq = ((size_t)g.Wo + 3) / 4 * 4, Hq = (size_t)H + 2 * (size_t)pad;
+        return round256((size_t)Cout * N * g.Ho * Wq * 4) + round256((size_t)S * C * N * Hq * Wq * 4) +
+               round256(conv_wgrad_split_workspace(N, H, C, Cout, R, S, pad, g.Ho, g.Wo));
+    }
     const size_t ldm = (size_t)pad32(g.Mg);
     return round256((size_t)Cout * ldm * 4) + round256((size_t)g.Kg * ldm * 4) + round256(gemm_split_workspace(Cout, g.Kg, g.Mg));
 }
@@ -362,6 +434,30 @@ extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_pl
     if (!qnn_aligned(g, 4) || !qnn_aligned(a_planes, 16) || !qnn_aligned(workspace, 256) || !qnn_aligned(gw, 4))
         return QNN_E_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (wgrad_implicit(cg)) {
+        const long long Wq = ((long long)cg.Wo + 3) / 4 * 4, Hq = (long long)H + 2 * pad, rows = (long long)N * cg.Ho;
+        float *gt = static_cast<float *>(workspace);                    // [Cout][N][Ho][Wq]
+        float *qas = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)Cout * rows * Wq * 4));   // [S][C][N][Hq][Wq]
+        void *split_ws = reinterpret_cast<char *>(qas) + round256((size_t)S * C * N * Hq * Wq * 4);
+        const dim3 ggrid((unsigned)rows, (unsigned)qnn_ceil_div(Cout, 32), (unsigned)qnn_ceil_div(Wq, 32));
+        conv_g_t_kernel<<<ggrid, 256, 0, st>>>(g, Cout, cg.Wo, Wq, rows, gt);
+        int rc = qnn_launch_status();
+        if (rc != QNN_OK) return rc;
+        const dim3 sgrid((unsigned)qnn_ceil_div((long long)N * Hq * Wq, 256), (unsigned)(S * cg.cw));
+        const long long a_pitch = qnn_row_words_i(C);
+#define CONV_S_CASE(B) case B: conv_codes_shift_kernel<B><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, qas); break;
+        switch (ab) {
+            CONV_S_CASE(1) CONV_S_CASE(2) CONV_S_CASE(3) CONV_S_CASE(4) CONV_S_CASE(5) CONV_S_CASE(6) CONV_S_CASE(7)
+            default: conv_codes_shift_kernel<8><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, qas); break;
+        }
+#undef CONV_S_CASE
+        if ((rc = qnn_launch_status()) != QNN_OK) return rc;
+        GemmParams p{};
+        p.alpha = alpha;
+        p.C = gw; p.ldc = cg.Kg;
+        if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
+        return run_conv_weight_gradient(gt, qas, N, H, C, Cout, R, S, pad, cg.Ho, cg.Wo, p, split_ws, st);
+    }
     const long long ldm = pad32(cg.Mg);
     float *gt = static_cast<float *>(workspace);                        // [Cout][ldm]: gt[co][m] = g[m][co]
     float *colt = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)Cout * ldm * 4));   // [Kg][ldm]

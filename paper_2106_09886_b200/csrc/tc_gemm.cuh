@@ -165,6 +165,23 @@ struct ConvGather {
     int n_images;
 };
 
+// Weight gradient of a stride-1 convolution as an implicit GEMM: GW[co][(r, s), c] = sum over output pixels (n, ho, wo) of
+// g[n][ho][wo][co] * qa[n][ho - pad + r][wo - pad + s][c].  The contraction runs over pixels, so both operands are read
+// pixel-contiguous: A from the transposed gradient gt[co][n][ho][j] and B from S copies of the transposed activation
+// codes, qas[s][c][n][h'][j] = qa[n][h' - pad][j - pad + s][c] (zero outside the image; h' = 0 .. H + 2*pad - 1, so the
+// padding rows exist as zeros).  Rows of both hold Wq >= Wo columns (Wo rounded up to 4, the extra columns of gt zero),
+// and (row, column) is ONE index p = row*Wq + j: a block of the contraction is 32 consecutive p of one image, and tap
+// (r, s) is copy s read at p + r*Wq -- a multiple of 4 elements, as the 16-byte rule for the start of a TMA box along its
+// innermost dimension demands (which is also why the shift along w is baked into the copies instead).
+// A tile of the result = 128 output features x up to BN channels of ONE tap.
+struct ConvWeightGather {
+    int enabled;
+    int C, S;
+    int tiles_c;                        // channel tiles per tap
+    int Wq;                             // columns per stored row
+    int kb_per_image;                   // blocks of the contraction per image: ceil(Ho*Wq / 32)
+};
+
 struct GemmParams {
     int M, N, K;                        // C[M][N] = alpha * sum_k A[M][K] * B[N][K]
     float alpha;
@@ -186,6 +203,7 @@ struct GemmParams {
     long long split_stride;
     unsigned int wait_limit;            // polls after which a wait on an arrival gives up (0 = WAIT_LIMIT)
     ConvGather conv;                    // enabled: A is gathered from the gradient image, rows of C are pixels (see above)
+    ConvWeightGather wconv;             // enabled: the contraction runs over the pixels of a convolution (see above)
 };
 
 // floor(a / b) and whether b divides a, for b > 0 and any sign of a
@@ -268,6 +286,7 @@ __device__ __forceinline__ void conv_epilogue_rows(const ConvTile &t, int row0, 
 struct WorkItem {
     int m0, n0, width;
     int kb0, kb1, split;                // K blocks [kb0, kb1) of this item; index of its partial buffer
+    int n_end;                          // columns of C from here on are not this tile's
 };
 template <int BN>
 __device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p, int nkb) {
@@ -276,7 +295,18 @@ __device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p, int nk
         tile = w / p.ksplit;
         const int sp = w - tile * p.ksplit;
         const int kb0 = sp * p.kb_per_split;
-        return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN, BN, kb0, min(nkb, kb0 + p.kb_per_split), sp};
+        const int nt = tile % p.tiles_n;
+        if (p.wconv.enabled) {                                      // column tile nt = (tap, channel tile)
+            const int tap = nt / p.wconv.tiles_c, c0 = (nt - tap * p.wconv.tiles_c) * BN;
+            return {(tile / p.tiles_n) * BM, tap * p.wconv.C + c0, BN, kb0, min(nkb, kb0 + p.kb_per_split), sp,
+                    tap * p.wconv.C + min(p.wconv.C, c0 + BN)};
+        }
+        return {(tile / p.tiles_n) * BM, nt * BN, BN, kb0, min(nkb, kb0 + p.kb_per_split), sp, p.N};
+    }
+    if (p.wconv.enabled) {
+        const int nt = tile % p.tiles_n;
+        const int tap = nt / p.wconv.tiles_c, c0 = (nt - tap * p.wconv.tiles_c) * BN;
+        return {(tile / p.tiles_n) * BM, tap * p.wconv.C + c0, BN, 0, nkb, 0, tap * p.wconv.C + min(p.wconv.C, c0 + BN)};
     }
     if (w >= p.whole_items) {
         const int r = w - p.whole_items;
@@ -284,7 +314,7 @@ __device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p, int nk
         off = (r & 1) * (BN / 2);
         width = BN / 2;
     }
-    return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN + off, width, 0, nkb, 0};
+    return {(tile / p.tiles_n) * BM, (tile % p.tiles_n) * BN + off, width, 0, nkb, 0, p.N};
 }
 
 template <int BN, int STAGES>
@@ -370,6 +400,22 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     continue;
                 }
                 const WorkItem wi = work_item<BN>(w, p, nkb);
+                if (KIND == TC_TF32 && p.wconv.enabled) {
+                    // block kb of the contraction = (image n, block pb of its pixels), walked incrementally
+                    const ConvWeightGather &c = p.wconv;
+                    const int tap = wi.n0 / c.C, cbase = wi.n0 - tap * c.C;
+                    const int r = tap / c.S, sx = tap - r * c.S;
+                    int n = wi.kb0 / c.kb_per_image, pb = wi.kb0 - n * c.kb_per_image;
+                    for (int kb = wi.kb0; kb < wi.kb1; ++kb) {
+                        if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err, p.wait_limit)) break;
+                        mbar_expect_tx(&full[s], L::STAGE_BYTES);
+                        tma_load_3d(smem + s * L::STAGE_BYTES, &map_a, &full[s], pb * BK, n, wi.m0);
+                        tma_load_4d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], pb * BK + r * c.Wq, n, cbase, sx);
+                        advance();
+                        if (++pb == c.kb_per_image) { pb = 0; ++n; }
+                    }
+                    continue;
+                }
                 const bool whole = wi.width == BN;
                 for (int kb = wi.kb0; kb < wi.kb1; ++kb) {
                     if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err, p.wait_limit)) break;
@@ -388,7 +434,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             int local = 0;
             for (int w = blockIdx.x; w < p.items && !*abort_flag; w += gridDim.x, ++local) {
                 WorkItem wi;
-                if (KIND == TC_TF32 && p.conv.enabled) wi = WorkItem{0, 0, BN, 0, conv_tile<BN>(w, p).nkb, 0};
+                if (KIND == TC_TF32 && p.conv.enabled) wi = WorkItem{0, 0, BN, 0, conv_tile<BN>(w, p).nkb, 0, p.N};
                 else wi = work_item<BN>(w, p, nkb);
                 const uint32_t idesc = wi.width == BN ? idesc_kmajor<BN, KIND>() : idesc_kmajor<BN / 2, KIND>();
                 const int buf = local & 1;
@@ -420,7 +466,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             WorkItem wi;
             if (conv) {
                 ct = conv_tile<BN>(w, p);
-                wi = WorkItem{0, ct.c0, BN, 0, ct.nkb, 0};
+                wi = WorkItem{0, ct.c0, BN, 0, ct.nkb, 0, p.N};
             } else {
                 wi = work_item<BN>(w, p, nkb);
             }
@@ -436,7 +482,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
             float *stage = reinterpret_cast<float *>(smem + L::EPI_OFFSET) + (warp - 2) * (32 * 33);
 #pragma unroll 1
             for (int c0 = half * 32; c0 < wi.width; c0 += 64) {
-                if (n0 + c0 >= p.N) break;                 // uniform over the warp
+                if (n0 + c0 >= wi.n_end) break;            // uniform over the warp
                 uint32_t v[32];
                 tmem_load_32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), v);
                 const int col = n0 + c0 + lane;
@@ -446,7 +492,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
 #pragma unroll
                     for (int i = 0; i < 32; ++i) istage[lane * 33 + i] = (int)v[i];
                     __syncwarp();
-                    if (col < p.N) {
+                    if (col < wi.n_end) {
                         const long long off = (long long)(m0 + q * 32) * p.ldc + col;
 #pragma unroll 8
                         for (int rr = 0; rr < rows_here; ++rr) {
@@ -461,7 +507,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     __syncwarp();
                     if (conv) {
                         // rows of the tile are pixels of a stride class: each row has its own place in the result
-                        if (col < p.N) {
+                        if (col < wi.n_end) {
                             switch (p.x ? p.bits : 0) {
                                 case 0: conv_epilogue_rows<0>(ct, q * 32, p, col, stage + lane); break;
                                 case 1: conv_epilogue_rows<1>(ct, q * 32, p, col, stage + lane); break;
@@ -474,7 +520,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                                 default: conv_epilogue_rows<8>(ct, q * 32, p, col, stage + lane); break;
                             }
                         }
-                    } else if (col < p.N) {
+                    } else if (col < wi.n_end) {
                         float *cptr = p.C + (long long)wi.split * p.split_stride + (long long)(m0 + q * 32) * p.ldc + col;
                         if (p.x) {
                             const float *xptr = p.x + (long long)(m0 + q * 32) * p.ldx + col;
@@ -581,7 +627,8 @@ int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtens
         cudaSuccess)
         return QNN_E_CUDA;
     if (p.wait_limit == 0) p.wait_limit = WAIT_LIMIT;
-    const long long tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const long long tiles_m = (p.M + BM - 1) / BM;
+    const long long tiles_n = p.wconv.enabled ? p.tiles_n : (p.N + BN - 1) / BN;   // (taps x channel tiles, set by the caller)
     if (tiles_m * tiles_n > 0x7FFFFFFFll) return QNN_E_ARG;
     p.tiles_n = (int)tiles_n;
     p.tiles = (int)(tiles_m * tiles_n);
@@ -593,7 +640,7 @@ int launch_gemm(const CUtensorMap &map_a, const CUtensorMap &map_b, const CUtens
     } else {
         p.ksplit = 1;
         const int rem = p.tiles % grid;
-        const bool split = !p.conv.enabled && rem > 0 && 2 * rem <= grid;
+        const bool split = !p.conv.enabled && !p.wconv.enabled && rem > 0 && 2 * rem <= grid;
         p.whole_items = split ? p.tiles - rem : p.tiles;
         p.items = split ? p.tiles + rem : p.tiles;
     }
@@ -683,6 +730,41 @@ int run_conv_data_gradient(const float *g, long long ldg, const float *wq, long 
                      : launch_gemm<64, 8, TC_TF32>(map_a, map_b, map_b, p, sms, st);
 }
 
+// Weight gradient of a stride-1 convolution (see ConvWeightGather): gw[co][(r*S + s)*C + c] = alpha * sum over output
+// pixels of gt[co][n][ho][wo] * qas[s][c][n][ho - pad + r][wo] (copy s already shifted by s - pad along w).
+//   gt   fp32 [Cout][N][Ho][Wp], qas fp32 [S][C][N][H][Wp], Wp = Wo rounded up to 4, padding columns zero; 16-byte aligned
+//   split_ws: partial products when the contraction is split over the CTAs (conv_wgrad_split_workspace bytes)
+struct ConvWgradPlan {
+    int Wq, Hq, kb_per_image, bn, tiles_c, ksplit, kb_per_split;
+    long long nkb;
+};
+ConvWgradPlan conv_wgrad_plan(int N, int H, int C, int Cout, int R, int S, int pad, int Ho, int Wo) {
+    ConvWgradPlan pl;
+    pl.Wq = (Wo + 3) / 4 * 4;
+    pl.Hq = H + 2 * pad;
+    pl.kb_per_image = (int)(((long long)Ho * pl.Wq + 31) / 32);
+    pl.nkb = (long long)N * pl.kb_per_image;
+    pl.bn = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
+    pl.tiles_c = (C + pl.bn - 1) / pl.bn;
+    // about two work items per SM (sized for 148 SMs so that workspace queries and calls agree), at least four blocks each
+    const long long tiles = (((long long)Cout + BM - 1) / BM) * R * S * pl.tiles_c;
+    long long want = (2 * 148) / tiles;
+    if (want > pl.nkb / 4) want = pl.nkb / 4;
+    if (want > 64) want = 64;
+    if (want < 2) {
+        pl.ksplit = 1; pl.kb_per_split = (int)pl.nkb;
+    } else {
+        const long long per = (pl.nkb + want - 1) / want;
+        pl.kb_per_split = (int)per;
+        pl.ksplit = (int)((pl.nkb + per - 1) / per);
+    }
+    return pl;
+}
+size_t conv_wgrad_split_workspace(int N, int H, int C, int Cout, int R, int S, int pad, int Ho, int Wo) {
+    const ConvWgradPlan pl = conv_wgrad_plan(N, H, C, Cout, R, S, pad, Ho, Wo);
+    return pl.ksplit > 1 ? (size_t)pl.ksplit * (size_t)Cout * (size_t)R * S * C * sizeof(float) : 0;
+}
+
 // C[i][j] = sum over s (in increasing order: a fixed summation order) of part[s][i][j]; dense partial buffers [M][N].
 __global__ void __launch_bounds__(256) sum_partials_kernel(const float *__restrict__ part, int ksplit, long long stride,
                                                           long long M, long long N, float *__restrict__ C, long long ldc) {
@@ -731,6 +813,39 @@ int run_gemm_tf32_split(const void *A, long long lda, const void *B, long long l
     const long long total = (long long)p.M * p.N;
     const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
     sum_partials_kernel<<<blocks, 256, 0, st>>>(p.C, ks, p.split_stride, p.M, p.N, C, ldc);
+    return qnn_launch_status();
+}
+
+int run_conv_weight_gradient(const float *gt, const float *qas, int N, int H, int C, int Cout, int R, int S, int pad, int Ho,
+                             int Wo, GemmParams p, void *split_ws, cudaStream_t st) {
+    if (!p.err || !qnn_aligned(gt, 16) || !qnn_aligned(qas, 16)) return QNN_E_ALIGN;
+    const int sms = sm_count();
+    if (sms <= 0) return QNN_E_CUDA;
+    const ConvWgradPlan pl = conv_wgrad_plan(N, H, C, Cout, R, S, pad, Ho, Wo);
+    if (pl.nkb * 32 > 0x7FFFFFFFll) return QNN_E_RANGE;
+    const long long Kg = (long long)R * S * C;
+    ConvWeightGather &c = p.wconv;
+    c.enabled = 1; c.C = C; c.S = S; c.tiles_c = pl.tiles_c; c.Wq = pl.Wq; c.kb_per_image = pl.kb_per_image;
+    p.M = Cout; p.N = (int)Kg; p.K = (int)(pl.nkb * 32);
+    p.tiles_n = R * S * pl.tiles_c;
+    float *C_out = p.C;
+    const long long ldc = p.ldc;
+    p.ksplit = pl.ksplit; p.kb_per_split = pl.kb_per_split;
+    if (pl.ksplit > 1) { p.C = static_cast<float *>(split_ws); p.ldc = Kg; p.split_stride = (long long)Cout * Kg; }
+    const long long pa = (long long)Ho * pl.Wq, pb = (long long)pl.Hq * pl.Wq;       // pixels per image in gt / in a copy
+    const long long adims[3] = {pa, N, Cout}, astr[2] = {pa, pa * N};
+    const int abox[3] = {32, 1, BM};
+    const long long bdims[4] = {pb, N, C, S}, bstr[3] = {pb, pb * N, pb * N * C};
+    const int bbox[4] = {32, 1, pl.bn, 1};
+    CUtensorMap map_a, map_b;
+    if (!make_map_nd(&map_a, gt, 3, adims, astr, abox) || !make_map_nd(&map_b, qas, 4, bdims, bstr, bbox)) return QNN_E_CUDA;
+    const int rc = pl.bn == 256 ? launch_gemm<256, 4, TC_TF32>(map_a, map_b, map_b, p, sms, st)
+                 : pl.bn == 128 ? launch_gemm<128, 6, TC_TF32>(map_a, map_b, map_b, p, sms, st)
+                                : launch_gemm<64, 8, TC_TF32>(map_a, map_b, map_b, p, sms, st);
+    if (rc != QNN_OK || pl.ksplit <= 1) return rc;
+    const long long total = (long long)Cout * Kg;
+    const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+    sum_partials_kernel<<<blocks, 256, 0, st>>>(static_cast<const float *>(split_ws), pl.ksplit, p.split_stride, Cout, Kg, C_out, ldc);
     return qnn_launch_status();
 }
 
