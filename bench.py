@@ -333,6 +333,15 @@ def training_side_leg(torch, qnn, dev, planes, packed, mp, mp_kind):
         status = qnn.tensor_path_status()
         flop = 2.0 * m * n * k
         peak = mp["bf16_tflops"] * (1.1 / 2.25)
+        # the same for convolution layers: the single-convolution configuration's layer and a mid-sized one
+        from paper_2106_09886_b200 import run_case as rc
+        conv = []
+        for (cn, ch, cc, cco) in ((32, 14, 256, 256), (16, 56, 256, 256)):
+            r = rc.time_backward_conv(cn, ch, ch, cc, cco, 3, 3, 1, 1, AB, WB, reps=10, warmup=3)
+            conv.append({"layer": f"conv3x3 {cc}->{cco}, {ch}x{ch}, batch {cn}, stride 1, pad 1", "data_ms": r["data_ms"],
+                         "weights_ms": r["weights_ms"], "data_tflops": r["data_tflops"], "weights_tflops": r["weights_tflops"],
+                         "data_frac_of_tf32_peak": r["data_tflops"] / peak, "weights_frac_of_tf32_peak": r["weights_tflops"] / peak,
+                         "workspace_mb": r["workspace_mb"], "tensor_path_status": r["status"]})
         return {"what": "Algorithm 1 backward of the benchmarked layer: whole calls (code unpack / transpose + TF32 tcgen05 GEMM), CUDA events",
                 "workload": f"fc {m}x{n}x{k}, w{WB}a{AB}", "dtype": "tf32 x exact codes, fp32 accumulate",
                 "backward_data_ms": t_data, "backward_data_with_encoder_derivative_ms": t_enc, "backward_weights_ms": t_w,
@@ -340,7 +349,8 @@ def training_side_leg(torch, qnn, dev, planes, packed, mp, mp_kind):
                 "roofline": {"bound": "tensor", "achieved": flop / (t_data * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                              "frac": flop / (t_data * 1e-3) / 1e12 / peak,
                              "peak_kind": f"{mp_kind} bf16 burst x 1.1/2.25 (nominal TF32:bf16)"},
-                "mbit_encoder_backward_gbs": m * k * 4.0 * (2 + AB) / (t_mb * 1e-3) / 1e9, "tensor_path_status": status}
+                "mbit_encoder_backward_gbs": m * k * 4.0 * (2 + AB) / (t_mb * 1e-3) / 1e9, "tensor_path_status": status,
+                "convolution_backward": conv}
     except Exception as exc:   # reported beside the benchmark, never fails it
         return {"what": "Algorithm 1 backward", "unavailable": f"{type(exc).__name__}: {exc}"[:200]}
 

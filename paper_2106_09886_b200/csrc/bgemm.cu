@@ -92,6 +92,19 @@ void fill_next(qnn_tiled::Params &p, const NextEnc *ne, int Ng) {
     qnn_clamp_bounds(ne->bits, ne->scale, (ne->flags & QNN_RELU) != 0, &p.next_lo, &p.next_hi);
 }
 
+void fill_next(qnn_pointwise::Params &p, const NextEnc *ne, int Ng) {
+    if (!ne) return;
+    p.ch_gamma = ne->gamma;
+    p.ch_beta = ne->beta;
+    if (!ne->planes) return;
+    p.next_planes = ne->planes;
+    p.next_bits = ne->bits;
+    p.next_kw = (int)qnn_row_words_i(Ng);
+    p.next_inv2s = 1.0f / (2.0f * ne->scale);
+    p.next_half = (float)(1 << (ne->bits - 1));
+    qnn_clamp_bounds(ne->bits, ne->scale, (ne->flags & QNN_RELU) != 0, &p.next_lo, &p.next_hi);
+}
+
 int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int64_t Mg, int Ng, int Kg, float alpha,
                float *out, int64_t ldo, int32_t *acc, const NextEnc *ne, void *stream);
 int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, int N, int H, int W, int C, int Cout,
@@ -162,10 +175,11 @@ int bgemm_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int kw = (int)qnn_row_words_i(Kg);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    if (!ne && qnn_pointwise::applicable(ab, wb, Kg, Ng)) {          // rows of at most four words per plane
+    if (qnn_pointwise::applicable(ab, wb, Kg, Ng)) {                 // rows of at most four words per plane
         qnn_pointwise::Params d = {};
         d.a = a_planes; d.w = w; d.Mg = Mg; d.Ng = Ng; d.Kg = Kg; d.a_pitch = kw; d.w_pitch = kw;
         d.alpha = alpha; d.out = out; d.ldo = ldo; d.acc = acc; d.conv = 0;
+        fill_next(d, ne, Ng);
         return qnn_pointwise::dispatch(ab, wb, d, st);
     }
     qnn_tiled::Params p = {};
@@ -214,12 +228,13 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
     if (Mg > ((int64_t)1 << 31) - 1 || (int64_t)N * H * W > ((int64_t)1 << 31) - 1) return QNN_E_RANGE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t *w = static_cast<const uint32_t *>(w_packed);
-    if (!ne && dil == 1 && !transposed && R == 1 && S == 1 && pad == 0 && C >= 32 && qnn_pointwise::applicable(ab, wb, C, Cout)) {
+    if (dil == 1 && !transposed && R == 1 && S == 1 && pad == 0 && C >= 32 && qnn_pointwise::applicable(ab, wb, C, Cout)) {
         // 1x1 convolution on at most 128 channels (a residual network's projections): no border, whole reduction in registers
         qnn_pointwise::Params d = {};
         d.a = a_planes; d.w = w; d.Mg = Mg; d.Ng = Cout; d.Kg = C; d.a_pitch = g.a_pitch; d.w_pitch = g.w_pitch;
         d.alpha = alpha; d.out = out; d.ldo = Cout; d.acc = acc;
         d.conv = 1; d.H = H; d.W = W; d.Ho = g.Ho; d.Wo = g.Wo; d.stride = stride;
+        fill_next(d, ne, Cout);
         return qnn_pointwise::dispatch(ab, wb, d, st);
     }
     if (dil == 1 && !transposed && qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout)) {
