@@ -79,7 +79,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -663,10 +663,14 @@ def run_gpu(args):
         if world == 1:
             line["training_side"] = training_side_leg(torch, qnn, dev, planes[0], packed, mp, mp_kind)
         if world == 1 and not args.no_configs:
+            sampler2 = ClockSampler(local)                # the per-configuration table runs for seconds: its own clock record
+            sampler2.start()
+            t_c0 = time.time()
             try:
                 line["configs"] = configs_leg(torch, qnn, dev, peaks, mp, mp_kind)
             except Exception as exc:   # reported beside the benchmark, never fails it
                 line["configs"] = {"unavailable": f"{type(exc).__name__}: {exc}"[:300]}
+            line["configs"]["clocks"] = sampler2.stop(t_c0, time.time())
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg()
         print(json.dumps(line), flush=True)
