@@ -45,9 +45,9 @@ E2E_CHUNK_ROWS, E2E_STREAMS = 1024, 8   # measured best of a sweep (256..2048 ro
 POPC_PER_WORD = 0.5   # popcounts the tiled kernel issues per 32-bit xor word (7:3 bit-column counters)
 
 
-# DRAM read+write of one qnn_bgemm 4096^3 w2a2 launch from the ncu capture summarised in
-# profiles/bgemm_tiled_4096_w2a2.md, valid for the kernel source with this digest only.
-NCU_TRAFFIC = {"bytes": 21984512, "kernel_sha256": "b2443eaa82d807659cb48d991bfa180ce6bff5fbc3ada2d809593e9c98ab244d"}
+# DRAM read+write of one qnn_bgemm 4096^3 w2a2 launch (launch 0 of the metrics-only ncu pass whose command
+# profiles/bgemm_tiled_4096_w2a2.md lists), valid for the kernel source with this digest only.
+NCU_TRAFFIC = {"bytes": 21963776, "kernel_sha256": "1817527ec71354dd1cd3132cd1145968ef114ae348f981339b8a385b9535a865"}
 
 
 def ncu_traffic_bytes():

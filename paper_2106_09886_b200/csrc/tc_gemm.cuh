@@ -292,8 +292,10 @@ template <int BN>
 __device__ __forceinline__ WorkItem work_item(int w, const GemmParams &p, int nkb) {
     int tile = w, off = 0, width = BN;
     if (p.ksplit > 1) {
-        tile = w / p.ksplit;
-        const int sp = w - tile * p.ksplit;
+        // items that contract the same range of K blocks are neighbours (they run at the same time and read the same
+        // slices of both operands through L2)
+        const int sp = w / p.tiles;
+        tile = w - sp * p.tiles;
         const int kb0 = sp * p.kb_per_split;
         const int nt = tile % p.tiles_n;
         if (p.wconv.enabled) {                                      // column tile nt = (tap, channel tile)
