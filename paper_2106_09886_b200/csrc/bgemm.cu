@@ -268,7 +268,7 @@ int bconv_impl(const uint32_t *a_planes, int ab, const void *w_packed, int wb, i
         int kind = (dil != 1 || transposed) ? 2 : 1;
         // nine taps and at most 4 channel words: 9-word groups leave no reduction tail (9% faster at C = 64, 128);
         // for more channels the tail is negligible and the 16-byte copies of the 8-word path win
-        if (kind == 1 && R * S == 9 && g.cw <= 4 && ab <= 4 && wb <= 4) kind = 3;
+        if (kind == 1 && R == 3 && S == 3 && g.cw <= 4 && ab <= 4 && wb <= 4) kind = 3;
         return qnn_tiled::dispatch_tiled(kind, ab, wb, p, st);
     }
     if (dil != 1 || transposed) return QNN_E_RANGE;      // the fallback kernel knows plain convolutions only
@@ -292,7 +292,7 @@ extern "C" int64_t qnn_popcounts_per_output(int ab, int wb, int is_conv, int R, 
         return qnn_pointwise::weighted_count_popcounts(ab, wb, (int)cw);          // (1x1 convolutions: when pad = 0)
     if (is_conv && qnn_dense::dense1_applicable(ab, wb, R, S, C, Cout))
         return (ab == 4 && wb == 4) ? 10 : ((ab == 3 && wb == 3) ? 7 : pairs);
-    if (is_conv && R * S == 9 && cw <= 4 && ab <= 4 && wb <= 4) return pairs * cw * 4;      // 9-word groups
+    if (is_conv && R == 3 && S == 3 && cw <= 4 && ab <= 4 && wb <= 4) return pairs * cw * 4;    // 9-word groups
     qnn_tiled::Params p = {};
     p.kwords = is_conv ? (int)(R * S * cw) : (int)qnn_row_words_i(C);
     qnn_tiled::set_k_split(p);

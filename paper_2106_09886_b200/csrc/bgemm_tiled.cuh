@@ -263,12 +263,22 @@ __global__ void __launch_bounds__(kThreads, (TM == 1 && AB == 4 && (KIND == 0 ||
             if (a_unit) {
                 const int gi = stage * kStageChunks + a_ch;
                 if (gi < p.nfull) {
+                    // a 3 x 3 window: tap = 3*r + sx at compile time; the window's top-left word once, the taps as
+                    // row / pixel steps from it, the border tests once per row and column of the window
+                    const int pix_step = AB * p.a_pitch;
+                    const int64_t row_step = (int64_t)p.W * pix_step;
+                    const uint32_t *base = p.a + ((t.pixbase + (int64_t)t.h0 * p.W + t.w0) * AB + a_plane) * p.a_pitch + gi;
+                    bool okh[3], okw[3];
+#pragma unroll
+                    for (int d = 0; d < 3; ++d) {
+                        okh[d] = t.a_ok && t.h0 + d >= 0 && t.h0 + d < p.H;
+                        okw[d] = t.w0 + d >= 0 && t.w0 + d < p.W;
+                    }
 #pragma unroll
                     for (int tap = 0; tap < 9; ++tap) {
-                        const int r = (int)(((uint32_t)tap * p.s_magic) >> 20), sx = tap - r * p.S;
-                        const int hi = t.h0 + r, wi = t.w0 + sx;
-                        const bool ok = t.a_ok && hi >= 0 && hi < p.H && wi >= 0 && wi < p.W;
-                        const uint32_t *src = p.a + ((t.pixbase + (int64_t)hi * p.W + wi) * AB + a_plane) * p.a_pitch + gi;
+                        constexpr int kR[9] = {0, 0, 0, 1, 1, 1, 2, 2, 2}, kS[9] = {0, 1, 2, 0, 1, 2, 0, 1, 2};
+                        const bool ok = okh[kR[tap]] && okw[kS[tap]];
+                        const uint32_t *src = base + kR[tap] * row_step + kS[tap] * pix_step;
                         const uint32_t dst = tap < 8 ? a_smem + a_dst0 + (uint32_t)((tap >> 2) * AB * kBM * 16 + (tap & 3) * 4)
                                                      : a_ext + (uint32_t)(((a_ch * AB + a_plane) * kBM + srow) * 4);
                         cp_async(dst, ok ? (const void *)src : (const void *)p.a, 4, ok);
