@@ -245,10 +245,11 @@ int qnn_bgemm_backward_weights(const float *g, const uint32_t *a_planes, size_t 
  * (tap, output feature): the kernel gathers its operand from g itself, one shifted box per tap, so no patch matrix is
  * ever written and each result element is a single fp32 accumulation of R*S*Cout terms; the workspace only holds the
  * unpacked weight codes (and a row-padded copy of g when Cout is not a multiple of 4).  The weight gradient contracts
- * over the output pixels; for stride 1 it too is an implicit GEMM, on the transposed gradient and S copies of the
- * transposed activation codes shifted along w (tap rows are shifts of the box that the kernel reads), which the call
- * stages in the workspace (about 1 + S times the layer's tensors in fp32); for other strides it stages the whole im2col
- * of the codes ([R*S*C][N*Ho*Wo] fp32).  Error bound as for the fully-connected products with contraction lengths
+ * over the output pixels; it too is an implicit GEMM, on the transposed gradient and S*stride copies of the transposed
+ * activation codes with the stride and the shift along w baked in (tap rows are shifts of the box that the kernel
+ * reads), which the call stages in the workspace (at stride 1 about 1 + S times the layer's tensors in fp32); where those
+ * copies would not be clearly smaller than the im2col of the codes ([R*S*C][N*Ho*Wo] fp32; e.g. 3 x 3 at stride 2) it
+ * stages that instead.  Error bound as for the fully-connected products with contraction lengths
  * R*S*Cout (data) and N*Ho*Wo (weights, plus the columns that pad each image row to a multiple of 4, which add exact
  * zeros); integer-valued g with small sums is contracted exactly.
  *   w_packed  blob of qnn_pack_weights(n_out = Cout, taps = R*S, c_in = C, bits = wb); a_planes [N*H*W][ab][qnn_row_words(C)]

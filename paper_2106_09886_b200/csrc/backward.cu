@@ -192,22 +192,23 @@ __global__ void __launch_bounds__(256) conv_g_t_kernel(const float *__restrict__
     }
 }
 
-// Activation planes -> S shifted copies of the transposed codes with the padding rows in place:
-// qas[s][c][n][hq][j] = qa[n][hq - pad][j - pad + s][c] for hq - pad inside the image, j < Wo and a column inside the
-// image, else 0; hq = 0 .. Hq - 1 = H + 2*pad - 1, j = 0 .. Wq - 1 (the B operand of the implicit weight gradient of a
-// stride-1 convolution).  One thread per (n, hq, j) and (s, channel word): consecutive threads write consecutive j.
+// Activation planes -> the copies of the transposed codes that the implicit weight gradient reads (ConvWeightGather):
+// qas[s*st + rho][c][n][a'][j] = qa[n][(a' + qmin)*st + rho][j*st - pad + s][c] where that pixel is inside the image and
+// j < Wo, else 0; a' = 0 .. Hq - 1, j = 0 .. Wq - 1.  One thread per (n, a', j) and (copy, channel word): consecutive
+// threads write consecutive j.
 template <int BITS>
 __global__ void __launch_bounds__(256) conv_codes_shift_kernel(const uint32_t *__restrict__ planes, long long a_pitch, ConvGeom g,
-                                                              int Hq, int Wq, float *__restrict__ qas) {
+                                                              int Hq, int Wq, int qmin, float *__restrict__ qas) {
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     const long long rows_total = (long long)g.N * Hq;
     if (idx >= rows_total * Wq) return;
-    const long long row = idx / Wq;                       // (n, hq)
+    const long long row = idx / Wq;                       // (n, a')
     const int j = (int)(idx - row * Wq);
     const long long n = row / Hq;
-    const int h = (int)(row - n * Hq) - g.pad;
-    const int s = blockIdx.y / g.cw, cwi = blockIdx.y % g.cw;
-    const int wi = j - g.pad + s;
+    const int copy = blockIdx.y / g.cw, cwi = blockIdx.y % g.cw;
+    const int s = copy / g.stride, rho = copy - s * g.stride;
+    const int h = ((int)(row - n * Hq) + qmin) * g.stride + rho;
+    const int wi = j * g.stride - g.pad + s;
     const bool inside = h >= 0 && h < g.H && j < g.Wo && wi >= 0 && wi < g.W;
     uint32_t w[BITS];
 #pragma unroll
@@ -216,7 +217,7 @@ __global__ void __launch_bounds__(256) conv_codes_shift_kernel(const uint32_t *_
     const float amax = (float)((1 << BITS) - 1);
     const int ncol = min(32, g.C - cwi * 32);
     const long long cstride = rows_total * Wq;
-    float *o = qas + ((long long)s * g.C + cwi * 32) * cstride + idx;
+    float *o = qas + ((long long)copy * g.C + cwi * 32) * cstride + idx;
 #pragma unroll 8
     for (int c = 0; c < 32; ++c) {
         int t = 0;
@@ -399,13 +400,17 @@ extern "C" int qnn_bconv2d_backward_data(const float *g, const void *w_packed, i
     return run_conv_data_gradient(a, lda, wqt, ldn, N, H, W, C, Cout, R, S, stride, pad, cg.Ho, cg.Wo, p, st);
 }
 
-// The weight gradient of a stride-1 convolution runs as an implicit GEMM on the transposed gradient and S shifted copies
-// of the transposed codes (about 1 + S times the size of the layer's tensors instead of R*S times); other strides stage
-// the whole patch matrix.
+// The weight gradient runs as an implicit GEMM on the transposed gradient and S*stride copies of the transposed codes
+// (ConvWeightGather) where those copies are clearly smaller than the R*S-fold patch matrix; otherwise, and for
+// geometries beyond the index ranges below, it stages the whole patch matrix.
 static bool wgrad_implicit(const ConvGeom &g) {
-    const long long Wq = ((long long)g.Wo + 3) / 4 * 4, Hq = (long long)g.H + 2 * g.pad;
-    return g.stride == 1 && (long long)g.N * g.Ho <= 0x7FFFFFFFll && Wq <= 65535 * 32 && (long long)g.S * g.cw <= 65535 &&
-           (long long)g.N * Hq * Wq <= (1ll << 36) && Wq * Hq * g.N * (long long)g.C < (1ll << 36) &&
+    const ConvWgradPlan pl = conv_wgrad_plan(g.N, g.C, g.Cout, g.R, g.S, g.stride, g.pad, g.Ho, g.Wo);
+    const long long Wq = pl.Wq, Hq = pl.Hq, copies = (long long)g.S * g.stride;
+    // worth it when the copies are clearly smaller than the patch matrix: always at stride 1 (3 x 3: 0.4 of it); at
+    // stride 2 a 3 x 3 kernel's six half-height copies are 0.8 of it and measured 12% slower, so those stay explicit
+    if (4 * copies * Hq * Wq > 3ll * g.R * g.S * g.Ho * g.Wo) return false;
+    return g.stride <= 16 && (long long)g.N * g.Ho <= 0x7FFFFFFFll && Wq <= 65535 * 32 && copies * g.cw <= 65535 &&
+           (long long)g.N * Hq * Wq <= (1ll << 36) && Wq * Hq * g.N * (long long)g.C * copies < (1ll << 37) &&
            Wq * g.Ho * g.N * (long long)g.Cout < (1ll << 36);
 }
 
@@ -414,9 +419,9 @@ extern "C" size_t qnn_bconv2d_backward_weights_workspace(int N, int H, int W, in
     ConvGeom g;
     if (!conv_geom(N, H, W, C, Cout, R, S, stride, pad, &g) || !conv_backward_dims_ok(g)) return 0;
     if (wgrad_implicit(g)) {
-        const size_t Wq = ((size_t)g.Wo + 3) / 4 * 4, Hq = (size_t)H + 2 * (size_t)pad;
-        return round256((size_t)Cout * N * g.Ho * Wq * 4) + round256((size_t)S * C * N * Hq * Wq * 4) +
-               round256(conv_wgrad_split_workspace(N, H, C, Cout, R, S, pad, g.Ho, g.Wo));
+        const ConvWgradPlan pl = conv_wgrad_plan(N, C, Cout, R, S, stride, pad, g.Ho, g.Wo);
+        return round256((size_t)Cout * N * g.Ho * pl.Wq * 4) + round256((size_t)S * stride * C * N * pl.Hq * pl.Wq * 4) +
+               round256(conv_wgrad_split_workspace(N, C, Cout, R, S, stride, pad, g.Ho, g.Wo));
     }
     const size_t ldm = (size_t)pad32(g.Mg);
     return round256((size_t)Cout * ldm * 4) + round256((size_t)g.Kg * ldm * 4) + round256(gemm_split_workspace(Cout, g.Kg, g.Mg));
@@ -435,20 +440,21 @@ extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_pl
         return QNN_E_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (wgrad_implicit(cg)) {
-        const long long Wq = ((long long)cg.Wo + 3) / 4 * 4, Hq = (long long)H + 2 * pad, rows = (long long)N * cg.Ho;
+        const ConvWgradPlan pl = conv_wgrad_plan(N, C, Cout, R, S, stride, pad, cg.Ho, cg.Wo);
+        const long long Wq = pl.Wq, Hq = pl.Hq, rows = (long long)N * cg.Ho, copies = (long long)S * stride;
         float *gt = static_cast<float *>(workspace);                    // [Cout][N][Ho][Wq]
-        float *qas = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)Cout * rows * Wq * 4));   // [S][C][N][Hq][Wq]
-        void *split_ws = reinterpret_cast<char *>(qas) + round256((size_t)S * C * N * Hq * Wq * 4);
+        float *qas = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)Cout * rows * Wq * 4));   // [S*stride][C][N][Hq][Wq]
+        void *split_ws = reinterpret_cast<char *>(qas) + round256((size_t)copies * C * N * Hq * Wq * 4);
         const dim3 ggrid((unsigned)rows, (unsigned)qnn_ceil_div(Cout, 32), (unsigned)qnn_ceil_div(Wq, 32));
         conv_g_t_kernel<<<ggrid, 256, 0, st>>>(g, Cout, cg.Wo, Wq, rows, gt);
         int rc = qnn_launch_status();
         if (rc != QNN_OK) return rc;
-        const dim3 sgrid((unsigned)qnn_ceil_div((long long)N * Hq * Wq, 256), (unsigned)(S * cg.cw));
+        const dim3 sgrid((unsigned)qnn_ceil_div((long long)N * Hq * Wq, 256), (unsigned)(copies * cg.cw));
         const long long a_pitch = qnn_row_words_i(C);
-#define CONV_S_CASE(B) case B: conv_codes_shift_kernel<B><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, qas); break;
+#define CONV_S_CASE(B) case B: conv_codes_shift_kernel<B><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, pl.qmin, qas); break;
         switch (ab) {
             CONV_S_CASE(1) CONV_S_CASE(2) CONV_S_CASE(3) CONV_S_CASE(4) CONV_S_CASE(5) CONV_S_CASE(6) CONV_S_CASE(7)
-            default: conv_codes_shift_kernel<8><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, qas); break;
+            default: conv_codes_shift_kernel<8><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, pl.qmin, qas); break;
         }
 #undef CONV_S_CASE
         if ((rc = qnn_launch_status()) != QNN_OK) return rc;
@@ -456,7 +462,7 @@ extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_pl
         p.alpha = alpha;
         p.C = gw; p.ldc = cg.Kg;
         if (!(p.err = qnn_tc_error_word())) return QNN_E_CUDA;
-        return run_conv_weight_gradient(gt, qas, N, H, C, Cout, R, S, pad, cg.Ho, cg.Wo, p, split_ws, st);
+        return run_conv_weight_gradient(gt, qas, N, C, Cout, R, S, stride, pad, cg.Ho, cg.Wo, p, split_ws, st);
     }
     const long long ldm = pad32(cg.Mg);
     float *gt = static_cast<float *>(workspace);                        // [Cout][ldm]: gt[co][m] = g[m][co]

@@ -165,18 +165,21 @@ struct ConvGather {
     int n_images;
 };
 
-// Weight gradient of a stride-1 convolution as an implicit GEMM: GW[co][(r, s), c] = sum over output pixels (n, ho, wo) of
-// g[n][ho][wo][co] * qa[n][ho - pad + r][wo - pad + s][c].  The contraction runs over pixels, so both operands are read
-// pixel-contiguous: A from the transposed gradient gt[co][n][ho][j] and B from S copies of the transposed activation
-// codes, qas[s][c][n][h'][j] = qa[n][h' - pad][j - pad + s][c] (zero outside the image; h' = 0 .. H + 2*pad - 1, so the
-// padding rows exist as zeros).  Rows of both hold Wq >= Wo columns (Wo rounded up to 4, the extra columns of gt zero),
-// and (row, column) is ONE index p = row*Wq + j: a block of the contraction is 32 consecutive p of one image, and tap
-// (r, s) is copy s read at p + r*Wq -- a multiple of 4 elements, as the 16-byte rule for the start of a TMA box along its
-// innermost dimension demands (which is also why the shift along w is baked into the copies instead).
-// A tile of the result = 128 output features x up to BN channels of ONE tap.
+// Weight gradient of a convolution as an implicit GEMM: GW[co][(r, s), c] = sum over output pixels (n, ho, wo) of
+// g[n][ho][wo][co] * qa[n][ho*st - pad + r][wo*st - pad + s][c].  The contraction runs over pixels, so both operands are
+// read pixel-contiguous: A from the transposed gradient gt[co][n][ho][j] and B from copies of the transposed activation
+// codes in which the stride and the shift along w are baked in: with r - pad = rho + st*q (0 <= rho < st), input row
+// ho*st - pad + r = (ho + q)*st + rho, so copy (s, rho) holds, for a' = 0 .. Hq - 1 and j = 0 .. Wq - 1,
+//   qas[s*st + rho][c][n][a'][j] = qa[n][(a' + qmin)*st + rho][j*st - pad + s][c]      (zero outside the image),
+// qmin = floor(-pad / st), Hq = Ho + floor((R - 1 - pad) / st) - qmin.  Rows of both operands hold Wq >= Wo columns (Wo
+// rounded up to 4, the extra columns of gt zero), and (row, column) is ONE index p = row*Wq + j: a block of the
+// contraction is 32 consecutive p of one image, and tap (r, s) is copy (s, rho) read at p + (q - qmin)*Wq -- a multiple
+// of 4 elements, as the 16-byte rule for the start of a TMA box along its innermost dimension demands (which is why
+// the shift along w lives in the copies while the shift along h is free).  For stride 1 there are S copies of the
+// padded image.  A tile of the result = 128 output features x up to BN channels of ONE tap.
 struct ConvWeightGather {
     int enabled;
-    int C, S;
+    int C, S, st, pad, qmin;
     int tiles_c;                        // channel tiles per tap
     int Wq;                             // columns per stored row
     int kb_per_image;                   // blocks of the contraction per image: ceil(Ho*Wq / 32)
@@ -407,12 +410,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) tc_gemm_kernel(const __grid_c
                     const ConvWeightGather &c = p.wconv;
                     const int tap = wi.n0 / c.C, cbase = wi.n0 - tap * c.C;
                     const int r = tap / c.S, sx = tap - r * c.S;
+                    int q;                                                        // r - pad = rho + st*q
+                    exact_div(r - c.pad, c.st, q);
+                    const int rho = r - c.pad - q * c.st;
+                    const int shift = (q - c.qmin) * c.Wq, copy = sx * c.st + rho;
                     int n = wi.kb0 / c.kb_per_image, pb = wi.kb0 - n * c.kb_per_image;
                     for (int kb = wi.kb0; kb < wi.kb1; ++kb) {
                         if (!mbar_wait(&empty[s], ph ^ 1u, abort_flag, 0, p.err, p.wait_limit)) break;
                         mbar_expect_tx(&full[s], L::STAGE_BYTES);
                         tma_load_3d(smem + s * L::STAGE_BYTES, &map_a, &full[s], pb * BK, n, wi.m0);
-                        tma_load_4d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], pb * BK + r * c.Wq, n, cbase, sx);
+                        tma_load_4d(smem + s * L::STAGE_BYTES + L::A_BYTES, &map_b, &full[s], pb * BK + shift, n, cbase, copy);
                         advance();
                         if (++pb == c.kb_per_image) { pb = 0; ++n; }
                     }
@@ -732,18 +739,21 @@ int run_conv_data_gradient(const float *g, long long ldg, const float *wq, long 
                      : launch_gemm<64, 8, TC_TF32>(map_a, map_b, map_b, p, sms, st);
 }
 
-// Weight gradient of a stride-1 convolution (see ConvWeightGather): gw[co][(r*S + s)*C + c] = alpha * sum over output
-// pixels of gt[co][n][ho][wo] * qas[s][c][n][ho - pad + r][wo] (copy s already shifted by s - pad along w).
-//   gt   fp32 [Cout][N][Ho][Wp], qas fp32 [S][C][N][H][Wp], Wp = Wo rounded up to 4, padding columns zero; 16-byte aligned
+// Weight gradient of a convolution (see ConvWeightGather): gw[co][(r*S + s)*C + c] = alpha * sum over output pixels of
+// gt[co][n][ho][j] * (copy (s, rho(r)) of the codes read (q(r) - qmin) rows further down).
+//   gt   fp32 [Cout][N][Ho][Wq], qas fp32 [S*stride][C][N][Hq][Wq] (conv_wgrad_plan), padding columns zero; 16-byte aligned
 //   split_ws: partial products when the contraction is split over the CTAs (conv_wgrad_split_workspace bytes)
 struct ConvWgradPlan {
-    int Wq, Hq, kb_per_image, bn, tiles_c, ksplit, kb_per_split;
+    int Wq, Hq, qmin, kb_per_image, bn, tiles_c, ksplit, kb_per_split;
     long long nkb;
 };
-ConvWgradPlan conv_wgrad_plan(int N, int H, int C, int Cout, int R, int S, int pad, int Ho, int Wo) {
+int floor_div(int a, int b) { return a >= 0 ? a / b : -((-a + b - 1) / b); }
+
+ConvWgradPlan conv_wgrad_plan(int N, int C, int Cout, int R, int S, int stride, int pad, int Ho, int Wo) {
     ConvWgradPlan pl;
     pl.Wq = (Wo + 3) / 4 * 4;
-    pl.Hq = H + 2 * pad;
+    pl.qmin = floor_div(-pad, stride);
+    pl.Hq = Ho + floor_div(R - 1 - pad, stride) - pl.qmin;
     pl.kb_per_image = (int)(((long long)Ho * pl.Wq + 31) / 32);
     pl.nkb = (long long)N * pl.kb_per_image;
     pl.bn = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
@@ -762,8 +772,8 @@ ConvWgradPlan conv_wgrad_plan(int N, int H, int C, int Cout, int R, int S, int p
     }
     return pl;
 }
-size_t conv_wgrad_split_workspace(int N, int H, int C, int Cout, int R, int S, int pad, int Ho, int Wo) {
-    const ConvWgradPlan pl = conv_wgrad_plan(N, H, C, Cout, R, S, pad, Ho, Wo);
+size_t conv_wgrad_split_workspace(int N, int C, int Cout, int R, int S, int stride, int pad, int Ho, int Wo) {
+    const ConvWgradPlan pl = conv_wgrad_plan(N, C, Cout, R, S, stride, pad, Ho, Wo);
     return pl.ksplit > 1 ? (size_t)pl.ksplit * (size_t)Cout * (size_t)R * S * C * sizeof(float) : 0;
 }
 
@@ -818,16 +828,17 @@ int run_gemm_tf32_split(const void *A, long long lda, const void *B, long long l
     return qnn_launch_status();
 }
 
-int run_conv_weight_gradient(const float *gt, const float *qas, int N, int H, int C, int Cout, int R, int S, int pad, int Ho,
-                             int Wo, GemmParams p, void *split_ws, cudaStream_t st) {
+int run_conv_weight_gradient(const float *gt, const float *qas, int N, int C, int Cout, int R, int S, int stride, int pad,
+                             int Ho, int Wo, GemmParams p, void *split_ws, cudaStream_t st) {
     if (!p.err || !qnn_aligned(gt, 16) || !qnn_aligned(qas, 16)) return QNN_E_ALIGN;
     const int sms = sm_count();
     if (sms <= 0) return QNN_E_CUDA;
-    const ConvWgradPlan pl = conv_wgrad_plan(N, H, C, Cout, R, S, pad, Ho, Wo);
+    const ConvWgradPlan pl = conv_wgrad_plan(N, C, Cout, R, S, stride, pad, Ho, Wo);
     if (pl.nkb * 32 > 0x7FFFFFFFll) return QNN_E_RANGE;
     const long long Kg = (long long)R * S * C;
     ConvWeightGather &c = p.wconv;
-    c.enabled = 1; c.C = C; c.S = S; c.tiles_c = pl.tiles_c; c.Wq = pl.Wq; c.kb_per_image = pl.kb_per_image;
+    c.enabled = 1; c.C = C; c.S = S; c.st = stride; c.pad = pad; c.qmin = pl.qmin;
+    c.tiles_c = pl.tiles_c; c.Wq = pl.Wq; c.kb_per_image = pl.kb_per_image;
     p.M = Cout; p.N = (int)Kg; p.K = (int)(pl.nkb * 32);
     p.tiles_n = R * S * pl.tiles_c;
     float *C_out = p.C;
@@ -837,7 +848,7 @@ int run_conv_weight_gradient(const float *gt, const float *qas, int N, int H, in
     const long long pa = (long long)Ho * pl.Wq, pb = (long long)pl.Hq * pl.Wq;       // pixels per image in gt / in a copy
     const long long adims[3] = {pa, N, Cout}, astr[2] = {pa, pa * N};
     const int abox[3] = {32, 1, BM};
-    const long long bdims[4] = {pb, N, C, S}, bstr[3] = {pb, pb * N, pb * N * C};
+    const long long bdims[4] = {pb, N, C, (long long)S * stride}, bstr[3] = {pb, pb * N, pb * N * C};
     const int bbox[4] = {32, 1, pl.bn, 1};
     CUtensorMap map_a, map_b;
     if (!make_map_nd(&map_a, gt, 3, adims, astr, abox) || !make_map_nd(&map_b, qas, 4, bdims, bstr, bbox)) return QNN_E_CUDA;

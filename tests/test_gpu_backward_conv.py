@@ -22,7 +22,9 @@ GEOMS = [(2, 6, 5, 3, 4, 3, 3, 1, 1), (1, 9, 9, 40, 6, 3, 3, 2, 1), (3, 8, 8, 64
          (2, 14, 14, 128, 32, 3, 3, 1, 1), (1, 5, 4, 70, 130, 3, 2, 1, 0), (5, 12, 12, 16, 24, 3, 3, 2, 2),
          # stride 3 with a 5 x 4 kernel (nine stride classes with different tap sets), a wide image (several tiles along
          # w), many images of 7 x 7 (tiles that span images), more than 256 channels (several channel tiles)
-         (2, 11, 10, 8, 12, 5, 4, 3, 2), (1, 3, 150, 16, 8, 3, 3, 1, 1), (37, 7, 7, 24, 40, 3, 3, 1, 1), (2, 6, 6, 300, 20, 3, 3, 2, 1)]
+         (2, 11, 10, 8, 12, 5, 4, 3, 2), (1, 3, 150, 16, 8, 3, 3, 1, 1), (37, 7, 7, 24, 40, 3, 3, 1, 1), (2, 6, 6, 300, 20, 3, 3, 2, 1),
+         # a 7 x 7 kernel at stride 2 (a network's stem): the weight gradient's strided copies of the codes, two row parities
+         (2, 16, 16, 8, 12, 7, 7, 2, 3)]
 
 
 def _codes(rng, shape, bits):
