@@ -416,11 +416,47 @@ __global__ void __launch_bounds__(kThreads, (TM == 1 && AB == 4 && (KIND == 0 ||
         }
     };
 
+    // Chaining epilogue, second half (see the first half in the epilogue below): thread (row, w) owns word w (32 features)
+    // of tile row `row`: it reads the 32 code bytes and moves bit i of each byte into plane i's word four bytes at a time
+    // with one mask and one multiply (((c & (0x01010101 << i)) * (0x10204080 >> i)) >> 28 = the four bits; the partial
+    // products land on distinct bits), appended by a funnel shift.  Replaces one warp ballot per plane and 16 features.
+    // It runs AFTER the first stage barrier of the CTA's next tile (or a barrier of its own after the last tile), so a
+    // tile costs no barrier of its own for it; the code matrix is double-buffered, which keeps the next epilogue's
+    // writes away from these reads.
+    int64_t pend_m0 = -1;                              // tile whose codes wait to be packed (-1: none); same in all threads
+    int pend_n0 = 0, pend_buf = 0;
+    auto pack_pending = [&]() {
+        if (tid < 2 * kBM) {
+            const int row = tid >> 1, wsel = tid & 1;
+            const int64_t m = pend_m0 + row;
+            if (m < p.Mg) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(smem + 2 * BUF_VEC) +
+                                                                   pend_buf * (kBM * kBN)) + row * 4 + wsel * 2;
+                const uint4 lo4 = src[0], hi4 = src[1];
+                const uint32_t c4[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+                const int word0 = (pend_n0 >> 5) + wsel;
+                uint32_t *dst = p.next_planes + (m * p.next_bits) * (int64_t)p.next_kw + word0;
+                const bool clear_pad = wsel == 0 && pend_n0 + kBN >= p.Ng;   // the last feature tile clears the row's padding words
+                for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
+                    const uint32_t mask = 0x01010101u << i, mul = 0x10204080u >> i;
+                    uint32_t word = 0u;
+#pragma unroll
+                    for (int g = 7; g >= 0; --g) word = __funnelshift_l((c4[g] & mask) * mul, word, 4);
+                    if (word0 < p.next_kw) *dst = word;
+                    if (clear_pad)
+                        for (int wz = (pend_n0 >> 5) + 2; wz < p.next_kw; ++wz) dst[wz - word0] = 0u;
+                }
+            }
+        }
+        pend_m0 = -1;
+    };
+
     int tile = blockIdx.x;
     if (tile >= p.ntiles) return;
     TileSrc cur = prep_tile(tile);
     issue_stage(cur, 0, 0);
     int buf = 0;
+    int code_buf = 0;                                  // code matrix that the next epilogue writes
 
     for (;;) {
         int acc[TM][4];
@@ -435,6 +471,9 @@ __global__ void __launch_bounds__(kThreads, (TM == 1 && AB == 4 && (KIND == 0 ||
             cp_async_wait_all();
             recode_stage(stage, buf);
             __syncthreads();   // everybody's units are in place, and everybody is done reading buf^1
+            if constexpr (FUSED) {
+                if (pend_m0 >= 0) pack_pending();          // the previous tile's code matrix is complete as well
+            }
             if (stage + 1 < p.nstages) {
                 issue_stage(cur, stage + 1, buf ^ 1);
             } else if (next_tile < p.ntiles) {
@@ -581,7 +620,7 @@ __global__ void __launch_bounds__(kThreads, (TM == 1 && AB == 4 && (KIND == 0 ||
                 // Next layer's encoder on the fp32 result (Alg. 1 forward: scale, then MBitEncoder), first half: the
                 // codes of this thread's outputs go to the tile's code matrix in shared memory, one byte each
                 // (0 outside the problem, so that padding bits come out as 0).
-                uint8_t *codes = reinterpret_cast<uint8_t *>(smem + 2 * BUF_VEC);        // [kBM][64]
+                uint8_t *codes = reinterpret_cast<uint8_t *>(smem + 2 * BUF_VEC) + code_buf * (kBM * kBN);   // [kBM][64]
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int n = n0 + tx + 16 * c;
@@ -591,36 +630,17 @@ __global__ void __launch_bounds__(kThreads, (TM == 1 && AB == 4 && (KIND == 0 ||
             }
         }
         if (FUSED && p.next_planes != nullptr) {
-            // Second half: thread (row, w) owns word w (32 features) of tile row `row`: it reads the 32 code bytes and
-            // moves bit i of each byte into plane i's word four bytes at a time with one mask and one multiply
-            // (((c & (0x01010101 << i)) * (0x10204080 >> i)) >> 28 = the four bits; the partial products land on
-            // distinct bits), appended by a funnel shift.  Replaces one warp ballot per plane and 16 features.
-            __syncthreads();                       // the code matrix is complete (the next tile's stage barriers
-                                                   // order these reads before its epilogue writes)
-            if (tid < 2 * kBM) {
-                const int row = tid >> 1, wsel = tid & 1;
-                const int64_t m = m0 + row;
-                if (m < p.Mg) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(smem + 2 * BUF_VEC) + row * 4 + wsel * 2;
-                    const uint4 lo4 = src[0], hi4 = src[1];
-                    const uint32_t c4[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
-                    const int word0 = (n0 >> 5) + wsel;
-                    uint32_t *dst = p.next_planes + (m * p.next_bits) * (int64_t)p.next_kw + word0;
-                    const bool clear_pad = wsel == 0 && n0 + kBN >= p.Ng;   // the last feature tile clears the row's padding words
-                    for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
-                        const uint32_t mask = 0x01010101u << i, mul = 0x10204080u >> i;
-                        uint32_t word = 0u;
-#pragma unroll
-                        for (int g = 7; g >= 0; --g) word = __funnelshift_l((c4[g] & mask) * mul, word, 4);
-                        if (word0 < p.next_kw) *dst = word;
-                        if (clear_pad)
-                            for (int wz = (n0 >> 5) + 2; wz < p.next_kw; ++wz) dst[wz - word0] = 0u;
-                    }
-                }
-            }
+            pend_m0 = m0; pend_n0 = n0; pend_buf = code_buf;      // packed after the next barrier
+            code_buf ^= 1;
         }
         tile = next_tile;
         if (tile >= p.ntiles) break;
+    }
+    if constexpr (FUSED) {
+        if (pend_m0 >= 0) {                                // the last tile's codes
+            __syncthreads();
+            pack_pending();
+        }
     }
 }
 
@@ -704,7 +724,7 @@ template <int AB, int WB, int CONV, int TM, bool FUSED>
 inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     constexpr int kBM = 16 * TM;
     constexpr size_t ext = (CONV == 3) ? ((size_t)kStageChunks * (AB * kBM + WB * kBN) + 3u) / 4u * 16u : 0u;   // ninth words
-    constexpr size_t smem = 2u * (kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u + ext) + (FUSED ? (size_t)kBM * kBN : 0u);   // + the chaining epilogue's code matrix
+    constexpr size_t smem = 2u * (kStageChunks * 2u * (AB * kBM + WB * kBN) * 16u + ext) + (FUSED ? 2u * (size_t)kBM * kBN : 0u);   // + the chaining epilogue's two code matrices
     if (smem > 48u * 1024u &&
         cudaFuncSetAttribute(bgemm_tiled_kernel<AB, WB, CONV, TM, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)
