@@ -106,6 +106,8 @@ __global__ void __launch_bounds__(kThreads) pointwise_kernel(const Params p) {
     constexpr int WARPS = kThreads / 32;
     uint4 *rows_s = smem4;                                                     // [WARPS][32 rows][AB] plane words (4 per plane)
     uint32_t *w_s = reinterpret_cast<uint32_t *>(smem4 + WARPS * 32 * AB);     // [WB][KW][Ng]
+    // FUSED: per warp two 32 x 32 matrices of code bytes (one per feature block of the item), 16-byte aligned
+    uint8_t *codes_all = reinterpret_cast<uint8_t *>(w_s + ((WB * KW * p.Ng + 3) & ~3));
     for (int idx = threadIdx.x; idx < WB * KW * p.Ng; idx += kThreads) {
         const int n = idx % p.Ng, jk = idx / p.Ng;
         const int j = jk / KW, k = jk - j * KW;
@@ -116,6 +118,7 @@ __global__ void __launch_bounds__(kThreads) pointwise_kernel(const Params p) {
     constexpr int AMAX = (1 << AB) - 1, PROD = AMAX * ((1 << WB) - 1);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint4 *mine_s = rows_s + warp * 32 * AB;
+    uint8_t *codes_s = codes_all + warp * 2048;
     const int64_t warp0 = (int64_t)blockIdx.x * WARPS + warp;
     const int64_t nwarps = (int64_t)gridDim.x * WARPS;
     const int64_t nbatches = (p.Mg + 31) / 32;
@@ -185,30 +188,53 @@ __global__ void __launch_bounds__(kThreads) pointwise_kernel(const Params p) {
                     if (p.out) p.out[row * p.ldo + n[h]] = y;
                 }
                 if (FUSED && p.next_planes != nullptr) {
-                    // Next layer's encoder: the 32 lanes hold 32 consecutive features of one row, i.e. exactly one
-                    // word of each plane; a ballot per plane assembles it (features beyond Ng give 0 bits).
+                    // Next layer's encoder, first half: the code of this output, one byte, into the warp's code matrix
+                    // [block h][row rr][feature lane] (0 beyond Ng, so that padding bits come out as 0)
                     const uint32_t code = n_ok[h] ? qnn_code_bits(y, p.next_inv2s, p.next_half, p.next_lo, p.next_hi) : 0u;
+                    codes_s[(h * 32 + rr) * 32 + lane] = (uint8_t)code;
+                }
+            }
+        }
+        if (FUSED && p.next_planes != nullptr) {
+            // Second half: lane L owns row L of the batch: its 32 code bytes per feature block are one word of each
+            // plane, gathered four bytes at a time with one mask and one multiply
+            // (((c & (0x01010101 << i)) * (0x10204080 >> i)) >> 28 = the four bits) and a funnel shift.
+            __syncwarp();
+            if (lane < rows_here) {
+                const int64_t row = batch * 32 + lane;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1 && !two) break;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(codes_s + (h * 32 + lane) * 32);
+                    const uint4 lo4 = src[0], hi4 = src[1];
+                    const uint32_t c4[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
                     uint32_t *dst = p.next_planes + (row * p.next_bits) * (int64_t)p.next_kw + (cb + h);
-                    for (int i = 0; i < p.next_bits; ++i) {
-                        const uint32_t word = __ballot_sync(0xffffffffu, (code >> i) & 1u);
-                        if (lane == 0) dst[(int64_t)i * p.next_kw] = word;
-                        // the warp that holds the row's last feature block also clears the padding words of the row
-                        if (cb + h == ncb - 1 && lane > 0 && cb + h + lane < p.next_kw) dst[(int64_t)i * p.next_kw + lane] = 0u;
+                    const bool clear_pad = cb + h == ncb - 1;                  // the row's last feature block: clear the padding words
+                    for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
+                        const uint32_t mask = 0x01010101u << i, mul = 0x10204080u >> i;
+                        uint32_t word = 0u;
+#pragma unroll
+                        for (int g = 7; g >= 0; --g) word = __funnelshift_l((c4[g] & mask) * mul, word, 4);
+                        *dst = word;
+                        if (clear_pad)
+                            for (int wz = ncb; wz < p.next_kw; ++wz) dst[wz - (cb + h)] = 0u;
                     }
                 }
             }
+            __syncwarp();                                                      // before the next item overwrites the matrix
         }
     }
 }
 
-inline size_t smem_bytes(int ab, int wb, int kw, int Ng) {
-    return (size_t)(kThreads / 32) * 32 * ab * 16 + (size_t)wb * kw * Ng * 4;
+inline size_t smem_bytes(int ab, int wb, int kw, int Ng, bool fused = false) {
+    const size_t weights = ((size_t)wb * kw * Ng + 3) / 4 * 16;               // rounded up to 16 bytes
+    return (size_t)(kThreads / 32) * 32 * ab * 16 + weights + (fused ? (size_t)(kThreads / 32) * 2048 : 0);
 }
 
 // usable when a row is at most 4 words per plane and the weights of all features fit the default shared memory
 inline bool applicable(int ab, int wb, int Kg, int Ng) {
     if (ab > 4 || wb > 4 || Kg > 128) return false;
-    return smem_bytes(ab, wb, (Kg + 31) / 32, Ng) <= 48u * 1024u;
+    return smem_bytes(ab, wb, (Kg + 31) / 32, Ng, true) <= 48u * 1024u;
 }
 
 template <int AB, int WB, int KW>
@@ -228,7 +254,7 @@ inline int launch(const Params &p_in, cudaStream_t st) {
     int64_t blocks = (items + kThreads / 32 - 1) / (kThreads / 32);
     if (blocks > (int64_t)sms * 4) blocks = (int64_t)sms * 4;
     if (p.ch_gamma != nullptr || p.next_planes != nullptr)
-        pointwise_kernel<AB, WB, KW, true><<<(int)blocks, kThreads, smem_bytes(AB, WB, KW, p.Ng), st>>>(p);
+        pointwise_kernel<AB, WB, KW, true><<<(int)blocks, kThreads, smem_bytes(AB, WB, KW, p.Ng, true), st>>>(p);
     else
         pointwise_kernel<AB, WB, KW, false><<<(int)blocks, kThreads, smem_bytes(AB, WB, KW, p.Ng), st>>>(p);
     return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA;

@@ -82,7 +82,7 @@ def test_fc_short_rows_padded_leading_dimension_and_single_outputs():
 @pytest.mark.parametrize("Mg,Ng,Kg,ab,wb,nb", [(70, 17, 64, 3, 3, 3), (33, 130, 96, 1, 1, 1), (200, 64, 128, 4, 4, 4),
                                                (45, 100, 33, 2, 3, 8), (129, 257, 100, 3, 2, 2)])
 def test_fc_short_rows_chained(Mg, Ng, Kg, ab, wb, nb):
-    """The chaining epilogue of the short-reduction kernel: next-layer planes (one ballot per plane and 32 features,
+    """The chaining epilogue of the short-reduction kernel: next-layer planes (code bytes gathered into words per row,
     padding words cleared) bit-identical to the oracle's quantize + pack of the oracle's fp32 result, with and
     without the fp32 output, with and without the per-feature affine."""
     import torch
