@@ -121,6 +121,30 @@ def test_composite_calls_check_every_argument_before_their_first_copy_or_launch(
         assert call(scale=0.0) == qnn.E_SCALE and call(flags=2) == qnn.E_ARG and call(ab=9) == qnn.E_ARG
 
 
+def test_popcounts_per_output_mirror_the_dispatch(qnn):
+    """The roofline helper: popcount instructions per output element of the kernel that serves a layer."""
+    f = qnn.lib.qnn_popcounts_per_output
+    # fully-connected, Kg = 4096: 128 words = 16 groups of 8 words at 4 popcounts, for each of the ab*wb pairs
+    assert f(2, 2, 0, 1, 1, 4096, 4096) == 4 * 16 * 4 and f(1, 1, 0, 1, 1, 4096, 4096) == 16 * 4
+    assert f(2, 2, 0, 1, 1, 512, 256) == 4 * 2 * 4                       # the small FC layer: 16 words
+    # 3x3 convolutions: 9-word groups (4 popcounts per channel word) up to 128 channels, 8-word groups beyond
+    assert f(3, 3, 1, 3, 3, 64, 64) == 9 * 2 * 4 and f(4, 4, 1, 3, 3, 128, 128) == 16 * 4 * 4
+    assert f(2, 2, 1, 3, 3, 256, 256) == 4 * 9 * 4                       # 72 words = 9 groups of 8
+    assert f(5, 3, 1, 3, 3, 64, 64) == 15 * (2 * 4 + 2)                  # 18 words: two groups and a tail of two words
+    # short reductions: the adder tree across plane pairs stops at W/2 adders (W = ab*wb*words)
+    assert f(3, 3, 1, 1, 1, 64, 128) == 9 and f(3, 3, 1, 1, 1, 128, 256) == 18 and f(4, 4, 0, 1, 1, 128, 64) == 32
+    assert f(1, 1, 0, 1, 1, 32, 8) == 1
+    # whole patch in one word (first layer on 3 channels): 10 popcounts at 4 x 4 bits, 7 at 3 x 3, one per pair otherwise
+    assert f(4, 4, 1, 3, 3, 3, 64) == 10 and f(3, 3, 1, 3, 3, 3, 64) == 7 and f(2, 4, 1, 3, 3, 3, 64) == 8
+    assert f(0, 2, 0, 1, 1, 64, 8) == 0 and f(2, 2, 0, 3, 3, 64, 8) == 0 and f(2, 9, 1, 3, 3, 64, 8) == 0
+
+
+def test_status_calls_check_their_arguments_on_the_host(qnn):
+    assert qnn.lib.qnn_selftest_bounded_wait(0, None) == qnn.E_ARG
+    assert qnn.lib.qnn_selftest_bounded_wait(1 << 20, None) == qnn.E_ARG
+    assert qnn.lib.qnn_last_device_status(None) == qnn.E_ARG and qnn.lib.qnn_tensor_path_status(None) == qnn.E_ARG
+
+
 def test_importing_binding_without_library_fails_loudly(tmp_path, monkeypatch):
     import importlib.util
     src = (ROOT / "paper_2106_09886_b200" / "qnn.py").read_text()
