@@ -27,7 +27,9 @@ constexpr int kBN = 64, kThreads = 256;
 // default rows per thread: 4 (BM = 64) for ab <= 2, 2 (BM = 32) for ab = 3, 4, 1 (BM = 16) for ab >= 5 (so that
 // TM*ab*8 operand words never exceed 64 registers); ab <= 2 also has a TM = 2
 // instantiation, used when halving the tile fills the SMs' CTA slots more evenly, and ab = 4 a TM = 1 one that runs
-// three CTAs per SM (fully-connected layers and 3x3 convolutions with 9-word groups, see launch_tiled).
+// three CTAs per SM (fully-connected layers and 3x3 convolutions with 9-word groups, see launch_tiled).  One-bit
+// activations (32 operand registers at TM = 4) also run three CTAs per SM: with a single plane the staging, re-coding
+// and barrier of a stage weigh twice what they do at two bits, and a third CTA hides them (+3 to +6%).
 template <int AB> struct TileM { static constexpr int TM = (AB <= 2) ? 4 : (AB <= 4 ? 2 : 1); };
 constexpr int kStageChunks = 2;                   // groups of 8 words per stage
 constexpr int kStageWords = 8 * kStageChunks;     // words per (row, plane) per stage
@@ -170,7 +172,7 @@ __device__ __forceinline__ void pair9(const uint32_t (&ta)[9], const uint32_t (&
 // KIND: 0 = fully-connected operand, 1 = convolution gather, 3 = 3x3 convolution gather with 9-word groups, 2 = dilated / transposed convolution gather (its
 // own instantiation: carrying that index arithmetic in the plain convolution cost it up to 15%).
 template <int AB, int WB, int KIND, int TM, bool FUSED>
-__global__ void __launch_bounds__(kThreads, (TM == 1 && AB == 4 && (KIND == 0 || KIND == 3)) ? 3 : 2) bgemm_tiled_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, ((TM == 1 && AB == 4 && (KIND == 0 || KIND == 3)) || (AB == 1 && KIND != 2)) ? 3 : 2) bgemm_tiled_kernel(const Params p) {
     constexpr bool CONV = KIND != 0, GENERAL = KIND == 2, G9 = KIND == 3;
     // multiply-shift division in the tile bookkeeping: convolutions with ab <= 4 only (the fully-connected kernels
     // divide once per tile, and both they and the 16-row-tile kernels for ab >= 5 ran 2-5% slower with it compiled
@@ -752,7 +754,7 @@ inline int launch_tiled_tmf(const Params &p, int sms, cudaStream_t st) {
     // hides the first-stage latency that would otherwise dominate.  Long reductions: one CTA per tile measured
     // about 5% faster (the hardware's dynamic block placement balances better than the static walk).
     const bool persistent = q.nstages <= 3;
-    const int per_sm = (TM == 1 && AB == 4 && (CONV == 0 || CONV == 3)) ? 3 : 2;
+    const int per_sm = ((TM == 1 && AB == 4 && (CONV == 0 || CONV == 3)) || (AB == 1 && CONV != 2)) ? 3 : 2;
     const int grid = (persistent && q.ntiles > per_sm * sms) ? per_sm * sms : q.ntiles;
     bgemm_tiled_kernel<AB, WB, CONV, TM, FUSED><<<grid, kThreads, smem, st>>>(q);
     return cudaGetLastError() == cudaSuccess ? QNN_OK : QNN_E_CUDA;
