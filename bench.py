@@ -456,10 +456,18 @@ def configs_leg(torch, qnn, dev, peaks, mp, mp_kind, quick=False):
                     "roofline": {"bound": "alu (per layer: see layers)", "frac": roof_ms / conv_ms,
                                  "what": "sum of the layers' roofline times / sum of their measured convolution times"}}
 
-    # the paper's efficiency experiment: 8192^3, 1..6 bits, against the Eq. 16 cost model (shape of the curve; the
-    # fp32 kernel it is a speed-up over is one of the paper's comparison systems and is not built)
+    # the paper's efficiency experiment (Section 5.4, Fig. 7): 8192^3, 1..6 bits, set against the plain
+    # one-thread-per-output fp32 kernel of the same size and against the Eq. 16 cost model
     sweep, base = [], None
     n8 = 8192
+    fa = torch.randn(n8, n8, device="cuda")
+    fb = torch.randn(n8, n8, device="cuda")
+    fc = torch.empty(n8, n8, device="cuda")
+    naive_ms = st.median(rc._time_calls(lambda i: qnn.probe_naive_sgemm(fa, fb, fc), 2, 1))
+    del fa, fb, fc
+    res["naive_fp32_8192"] = {"what": "qnn_probe_naive_sgemm: one thread per output, one fma per step, no tiling "
+                                      "(the comparison line of the paper's efficiency figure; not a product path)",
+                              "ms": naive_ms, "tflops": 2.0 * n8 ** 3 / naive_ms / 1e9}
     for b in range(1, 7):
         r = rc.time_gemm(n8, n8, n8, b, b, reps=3, warmup=2, sets=1)
         ms = r["ms_median"]
@@ -468,6 +476,7 @@ def configs_leg(torch, qnn, dev, peaks, mp, mp_kind, quick=False):
         sweep.append({"bits": b, "ms": ms, "binary_tops": r["binary_tops"], "equiv_int_gops": r["equiv_int_gops"],
                       "time_vs_1bit": ms / base, "eq16_cost_vs_1bit": eq16_model_speedup(n8, 1, 1) / eq16_model_speedup(n8, b, b),
                       "eq16_speedup_model": eq16_model_speedup(n8, b, b),
+                      "speedup_vs_naive_fp32": naive_ms / ms,
                       "roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac")}})
     res["sweep_8192_bits_1_to_6"] = sweep
     return res

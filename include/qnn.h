@@ -397,8 +397,14 @@ int qnn_fc_forward_noalloc(const float *x, int64_t Mg, int Kg, int64_t ldx, int 
  * C = Kg, Cout = Ng) or qnn_bconv2d (is_conv != 0) runs for such a layer issues per output element, all ab*wb plane
  * pairs together (0 = arguments out of range): the popcount pipe is the scarce unit of the contraction, so
  * outputs * that number / the popcount rate of probe variant 0 is the layer's bit-operation roofline time.
+ * qnn_probe_naive_sgemm enqueues the plain fp32 product that the efficiency experiment (Section 5.4, Fig. 7, Eq. 16)
+ * sets the bit-plane product against: c[m][n] = sum_k a[m][k] * b[k][n], device pointers, all three row-major and
+ * dense, one thread per output, one fused multiply-add per reduction step in increasing k, nothing tiled.  A
+ * comparison line only: no product path calls it.  QNN_E_ARG on null pointers or sizes <= 0, QNN_E_RANGE when
+ * m > 8 * 65535.
  */
 int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream);
+int qnn_probe_naive_sgemm(const float *a, const float *b, float *c, int m, int n, int k, void *stream);
 int64_t qnn_popcounts_per_output(int ab, int wb, int is_conv, int R, int S, int C, int Cout);
 int qnn_probe_copy(void *dst, const void *src, size_t bytes, void *stream);
 

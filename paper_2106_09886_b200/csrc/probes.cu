@@ -119,7 +119,29 @@ __global__ void __launch_bounds__(256) probe_copy_kernel(uint4 *__restrict__ dst
         dst[i] = src[i];
 }
 
+// The plain fp32 product the efficiency experiment (Section 5.4, Fig. 7) times the bit-plane product against: one
+// thread per output element, one multiply-add per step of the reduction, operands straight from global memory, no
+// tiling, no shared memory, no tensor cores.  c[m][n] = sum_k a[m][k] * b[k][n], all row-major.
+__global__ void __launch_bounds__(256) probe_naive_sgemm_kernel(const float *__restrict__ a, const float *__restrict__ b,
+                                                                float *__restrict__ c, int m, int n, int k) {
+    const int col = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int row = blockIdx.y * 8 + (threadIdx.x >> 5);
+    if (row >= m || col >= n) return;
+    const float *ar = a + (size_t)row * k;
+    float acc = 0.f;
+    for (int i = 0; i < k; ++i) acc = fmaf(ar[i], b[(size_t)i * n + col], acc);
+    c[(size_t)row * n + col] = acc;
+}
+
 }  // namespace
+
+extern "C" int qnn_probe_naive_sgemm(const float *a, const float *b, float *c, int m, int n, int k, void *stream) {
+    if (!a || !b || !c || m <= 0 || n <= 0 || k <= 0) return QNN_E_ARG;
+    if ((m + 7) / 8 > 65535) return QNN_E_RANGE;
+    dim3 grid((n + 31) / 32, (m + 7) / 8);
+    probe_naive_sgemm_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(a, b, c, m, n, k);
+    return qnn_launch_status();
+}
 
 extern "C" int qnn_probe_bitops(int variant, int iters, int blocks, int32_t *sink, double *word_ops, void *stream) {
     if (!sink || iters <= 0 || blocks <= 0 || (variant < 0 || variant > 4)) return QNN_E_ARG;

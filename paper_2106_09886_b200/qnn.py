@@ -25,7 +25,7 @@ EXPORTS = [
     "qnn_bgemm_backward_weights_workspace", "qnn_bgemm_backward_weights", "qnn_bconv2d_backward_data_workspace",
     "qnn_bconv2d_backward_data", "qnn_bconv2d_backward_weights_workspace", "qnn_bconv2d_backward_weights", "qnn_unpack_codes_f32",
     "qnn_tensor_path_status", "qnn_last_device_status", "qnn_selftest_bounded_wait", "qnn_bgemm_int8_tensor_workspace", "qnn_bgemm_int8_tensor",
-    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_copy", "qnn_popcounts_per_output",
+    "qnn_absmax_f32", "qnn_fc_forward_host", "qnn_fc_forward_host_pipelined", "qnn_fc_forward_noalloc", "qnn_probe_bitops", "qnn_probe_naive_sgemm", "qnn_probe_copy", "qnn_popcounts_per_output",
 ]
 NOALLOC_SCRATCH_BYTES = 8 << 20
 
@@ -89,6 +89,7 @@ def _load() -> C.CDLL:
     lib.qnn_fc_forward_noalloc.argtypes = [p, i64, i, i64, i, f, u, p, i, i, f, p, i64, p]
     lib.qnn_probe_bitops.argtypes = [i, i, i, p, C.POINTER(C.c_double), p]
     lib.qnn_probe_copy.argtypes = [p, p, sz, p]
+    lib.qnn_probe_naive_sgemm.argtypes = [p, p, p, i, i, i, p]
     return lib
 
 
@@ -466,3 +467,19 @@ def weights_views(packed: torch.Tensor, n_out: int, taps: int, c_in: int, bits: 
     nplane = n_out * bits * kw
     as_i32 = packed.view(torch.int32)
     return as_i32[:nplane].view(n_out, bits, kw), as_i32[nplane:nplane + n_out * taps].view(n_out, taps)
+
+
+def probe_naive_sgemm(a: torch.Tensor, b: torch.Tensor, c: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """c = a @ b by the plain one-thread-per-output fp32 kernel (comparison line of Section 5.4); a [m, k], b [k, n]."""
+    m, k = a.shape
+    n = b.shape[1]
+    if b.shape[0] != k or a.dtype != torch.float32 or b.dtype != torch.float32:
+        raise QnnError(E_ARG, "qnn_probe_naive_sgemm")
+    if not (a.is_contiguous() and b.is_contiguous()):
+        raise QnnError(E_ARG, "qnn_probe_naive_sgemm: dense row-major operands")
+    if c is None:
+        c = torch.empty((m, n), dtype=torch.float32, device=a.device)
+    if tuple(c.shape) != (m, n) or c.dtype != torch.float32 or not c.is_contiguous():
+        raise QnnError(E_ARG, "qnn_probe_naive_sgemm: dense row-major [m, n] fp32 output")
+    _check(lib.qnn_probe_naive_sgemm(_ptr(a), _ptr(b), _ptr(c), m, n, k, _stream(stream)), "qnn_probe_naive_sgemm")
+    return c

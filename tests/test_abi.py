@@ -90,6 +90,9 @@ def test_argument_errors_are_reported_before_any_launch(qnn):
     assert lib.qnn_absmax_f32(p, 0, p, None) == qnn.E_ARG
     assert lib.qnn_absmax_f32(None, 4, p, None) == qnn.E_ARG
     assert lib.qnn_probe_copy(p, p, 24, None) == qnn.E_ARG
+    assert lib.qnn_probe_naive_sgemm(p, p, None, 4, 4, 4, None) == qnn.E_ARG
+    assert lib.qnn_probe_naive_sgemm(p, p, p, 4, 0, 4, None) == qnn.E_ARG
+    assert lib.qnn_probe_naive_sgemm(p, p, p, 8 * 65535 + 1, 4, 4, None) == qnn.E_RANGE
 
 
 def test_composite_calls_check_every_argument_before_their_first_copy_or_launch(qnn):
