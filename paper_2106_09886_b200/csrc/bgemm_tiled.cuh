@@ -428,26 +428,27 @@ __global__ void __launch_bounds__(kThreads, ((TM == 1 && AB == 4 && (KIND == 0 |
     int64_t pend_m0 = -1;                              // tile whose codes wait to be packed (-1: none); same in all threads
     int pend_n0 = 0, pend_buf = 0;
     auto pack_pending = [&]() {
-        if (tid < 2 * kBM) {
-            const int row = tid >> 1, wsel = tid & 1;
-            const int64_t m = pend_m0 + row;
-            if (m < p.Mg) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(smem + 2 * BUF_VEC) +
-                                                                   pend_buf * (kBM * kBN)) + row * 4 + wsel * 2;
-                const uint4 lo4 = src[0], hi4 = src[1];
-                const uint32_t c4[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
-                const int word0 = (pend_n0 >> 5) + wsel;
-                uint32_t *dst = p.next_planes + (m * p.next_bits) * (int64_t)p.next_kw + word0;
-                const bool clear_pad = wsel == 0 && pend_n0 + kBN >= p.Ng;   // the last feature tile clears the row's padding words
-                for (int i = 0; i < p.next_bits; ++i, dst += p.next_kw) {
-                    const uint32_t mask = 0x01010101u << i, mul = 0x10204080u >> i;
-                    uint32_t word = 0u;
+        // one (row, word of the tile, plane) per thread: 2 * kBM units per plane, kThreads / (2 * kBM) planes at a time
+        constexpr int PLANES_AT_ONCE = kThreads / (2 * kBM);
+        const int unit = tid % (2 * kBM);
+        const int row = unit >> 1, wsel = unit & 1;
+        const int64_t m = pend_m0 + row;
+        if (m < p.Mg) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(smem + 2 * BUF_VEC) +
+                                                               pend_buf * (kBM * kBN)) + row * 4 + wsel * 2;
+            const uint4 lo4 = src[0], hi4 = src[1];
+            const uint32_t c4[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+            const int word0 = (pend_n0 >> 5) + wsel;
+            const bool clear_pad = wsel == 0 && pend_n0 + kBN >= p.Ng;   // the last feature tile clears the row's padding words
+            for (int i = tid / (2 * kBM); i < p.next_bits; i += PLANES_AT_ONCE) {
+                uint32_t *dst = p.next_planes + (m * p.next_bits + i) * (int64_t)p.next_kw + word0;
+                const uint32_t mask = 0x01010101u << i, mul = 0x10204080u >> i;
+                uint32_t word = 0u;
 #pragma unroll
-                    for (int g = 7; g >= 0; --g) word = __funnelshift_l((c4[g] & mask) * mul, word, 4);
-                    if (word0 < p.next_kw) *dst = word;
-                    if (clear_pad)
-                        for (int wz = (pend_n0 >> 5) + 2; wz < p.next_kw; ++wz) dst[wz - word0] = 0u;
-                }
+                for (int g = 7; g >= 0; --g) word = __funnelshift_l((c4[g] & mask) * mul, word, 4);
+                if (word0 < p.next_kw) *dst = word;
+                if (clear_pad)
+                    for (int wz = (pend_n0 >> 5) + 2; wz < p.next_kw; ++wz) dst[wz - word0] = 0u;
             }
         }
         pend_m0 = -1;
