@@ -194,36 +194,49 @@ __global__ void __launch_bounds__(256) conv_g_t_kernel(const float *__restrict__
 
 // Activation planes -> the copies of the transposed codes that the implicit weight gradient reads (ConvWeightGather):
 // qas[s*st + rho][c][n][a'][j] = qa[n][(a' + qmin)*st + rho][j*st - pad + s][c] where that pixel is inside the image and
-// j < Wo, else 0; a' = 0 .. Hq - 1, j = 0 .. Wq - 1.  One thread per (n, a', j) and (copy, channel word): consecutive
-// threads write consecutive j.
+// j < Wo, else 0; a' = 0 .. Hq - 1, j = 0 .. Wq - 1.  One thread per (n, a', four consecutive j) and (copy, channel word):
+// consecutive threads write consecutive j.
 template <int BITS>
 __global__ void __launch_bounds__(256) conv_codes_shift_kernel(const uint32_t *__restrict__ planes, long long a_pitch, ConvGeom g,
                                                               int Hq, int Wq, int qmin, float *__restrict__ qas) {
-    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    // four consecutive j per thread (Wq is a multiple of 4): every store is 16 bytes, a warp writes 512 contiguous bytes
+    const int wq4 = Wq >> 2;
+    const long long idx4 = (long long)blockIdx.x * 256 + threadIdx.x;
     const long long rows_total = (long long)g.N * Hq;
-    if (idx >= rows_total * Wq) return;
-    const long long row = idx / Wq;                       // (n, a')
-    const int j = (int)(idx - row * Wq);
+    if (idx4 >= rows_total * wq4) return;
+    const long long row = idx4 / wq4;                     // (n, a')
+    const int j0 = (int)(idx4 - row * wq4) * 4;
     const long long n = row / Hq;
     const int copy = blockIdx.y / g.cw, cwi = blockIdx.y % g.cw;
     const int s = copy / g.stride, rho = copy - s * g.stride;
     const int h = ((int)(row - n * Hq) + qmin) * g.stride + rho;
-    const int wi = j * g.stride - g.pad + s;
-    const bool inside = h >= 0 && h < g.H && j < g.Wo && wi >= 0 && wi < g.W;
-    uint32_t w[BITS];
+    const bool row_inside = h >= 0 && h < g.H;
+    uint32_t w[4][BITS];
+    bool inside[4];
 #pragma unroll
-    for (int b = 0; b < BITS; ++b)
-        w[b] = inside ? __ldg(planes + (((n * g.H + h) * g.W + wi) * BITS + b) * a_pitch + cwi) : 0u;
-    const float amax = (float)((1 << BITS) - 1);
+    for (int k = 0; k < 4; ++k) {
+        const int j = j0 + k, wi = j * g.stride - g.pad + s;
+        inside[k] = row_inside && j < g.Wo && wi >= 0 && wi < g.W;
+#pragma unroll
+        for (int b = 0; b < BITS; ++b)
+            w[k][b] = inside[k] ? __ldg(planes + (((n * g.H + h) * g.W + wi) * BITS + b) * a_pitch + cwi) : 0u;
+    }
+    // code 2t - amax as a float without a conversion: the bits of 2^23 + 2t, minus (2^23 + amax); both exact
+    const float bias = 8388608.0f + (float)((1 << BITS) - 1);
     const int ncol = min(32, g.C - cwi * 32);
     const long long cstride = rows_total * Wq;
-    float *o = qas + ((long long)copy * g.C + cwi * 32) * cstride + idx;
-#pragma unroll 8
+    float *o = qas + ((long long)copy * g.C + cwi * 32) * cstride + row * Wq + j0;
+#pragma unroll 4
     for (int c = 0; c < 32; ++c) {
-        int t = 0;
+        float v[4];
 #pragma unroll
-        for (int b = 0; b < BITS; ++b) t |= (int)((w[b] >> c) & 1u) << b;
-        if (c < ncol) o[c * cstride] = inside ? (float)(2 * t) - amax : 0.0f;
+        for (int k = 0; k < 4; ++k) {
+            uint32_t t2 = 0u;
+#pragma unroll
+            for (int b = 0; b < BITS; ++b) t2 |= ((w[k][b] >> c) & 1u) << (b + 1);
+            v[k] = inside[k] ? __int_as_float((int)(0x4B000000u | t2)) - bias : 0.0f;
+        }
+        if (c < ncol) *reinterpret_cast<float4 *>(o + c * cstride) = make_float4(v[0], v[1], v[2], v[3]);
     }
 }
 
@@ -445,11 +458,17 @@ extern "C" int qnn_bconv2d_backward_weights(const float *g, const uint32_t *a_pl
         float *gt = static_cast<float *>(workspace);                    // [Cout][N][Ho][Wq]
         float *qas = reinterpret_cast<float *>(static_cast<char *>(workspace) + round256((size_t)Cout * rows * Wq * 4));   // [S*stride][C][N][Hq][Wq]
         void *split_ws = reinterpret_cast<char *>(qas) + round256((size_t)copies * C * N * Hq * Wq * 4);
-        const dim3 ggrid((unsigned)rows, (unsigned)qnn_ceil_div(Cout, 32), (unsigned)qnn_ceil_div(Wq, 32));
-        conv_g_t_kernel<<<ggrid, 256, 0, st>>>(g, Cout, cg.Wo, Wq, rows, gt);
+        if (Wq == cg.Wo && qnn_ceil_div(cg.Mg, 32) <= 65535) {
+            // no row padding: gt[co][pixel] is the plain transpose of g[pixel][co], whole 32 x 32 tiles throughout
+            const dim3 tgrid((unsigned)qnn_ceil_div(Cout, 32), (unsigned)qnn_ceil_div(cg.Mg, 32));
+            transpose_f32_kernel<<<tgrid, 256, 0, st>>>(g, cg.Mg, (long long)Cout, (long long)Cout, gt, cg.Mg);
+        } else {
+            const dim3 ggrid((unsigned)rows, (unsigned)qnn_ceil_div(Cout, 32), (unsigned)qnn_ceil_div(Wq, 32));
+            conv_g_t_kernel<<<ggrid, 256, 0, st>>>(g, Cout, cg.Wo, Wq, rows, gt);
+        }
         int rc = qnn_launch_status();
         if (rc != QNN_OK) return rc;
-        const dim3 sgrid((unsigned)qnn_ceil_div((long long)N * Hq * Wq, 256), (unsigned)(copies * cg.cw));
+        const dim3 sgrid((unsigned)qnn_ceil_div((long long)N * Hq * (Wq / 4), 256), (unsigned)(copies * cg.cw));
         const long long a_pitch = qnn_row_words_i(C);
 #define CONV_S_CASE(B) case B: conv_codes_shift_kernel<B><<<sgrid, 256, 0, st>>>(a_planes, a_pitch, cg, (int)Hq, (int)Wq, pl.qmin, qas); break;
         switch (ab) {

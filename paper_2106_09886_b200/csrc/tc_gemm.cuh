@@ -758,11 +758,21 @@ ConvWgradPlan conv_wgrad_plan(int N, int C, int Cout, int R, int S, int stride, 
     pl.nkb = (long long)N * pl.kb_per_image;
     pl.bn = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
     pl.tiles_c = (C + pl.bn - 1) / pl.bn;
-    // about two work items per SM (sized for 148 SMs so that workspace queries and calls agree), at least four blocks each
+    // at most about two work items per SM (sized for 148 SMs so that workspace queries and calls agree), at least
+    // four blocks each; among those the fewest parts whose rounds are within 3 % of the best filled (every part
+    // writes, and the sum re-reads, one partial result)
     const long long tiles = (((long long)Cout + BM - 1) / BM) * R * S * pl.tiles_c;
-    long long want = (2 * 148) / tiles;
-    if (want > pl.nkb / 4) want = pl.nkb / 4;
-    if (want > 64) want = 64;
+    long long most = (2 * 148) / tiles;
+    if (most > pl.nkb / 4) most = pl.nkb / 4;
+    if (most > 64) most = 64;
+    auto fill = [&](long long parts) {
+        const long long items = tiles * parts;
+        return (double)items / (double)((items + 147) / 148 * 148);
+    };
+    double best = 0.0;
+    for (long long parts = 1; parts <= most; ++parts) best = fill(parts) > best ? fill(parts) : best;
+    long long want = 1;
+    while (want < most && fill(want) < best - 0.03) ++want;
     if (want < 2) {
         pl.ksplit = 1; pl.kb_per_split = (int)pl.nkb;
     } else {
