@@ -45,3 +45,7 @@ def test_bench_line_has_the_contract_keys():
         for L in c[net]["layers"]:
             assert L["roofline"]["bound"] in ("alu", "hbm") and 0.05 < L["roofline"]["frac"] < 1.2, L
     assert abs(c["sweep_8192_bits_1_to_6"][1]["eq16_speedup_model"] - 15.13) < 0.01        # Eq. 16's printed 2-bit value
+    # the plain fp32 kernel of the efficiency figure is timed in the same leg; the bit-plane product beats it at every width
+    assert c["naive_fp32_8192"]["ms"] > 0
+    for e in c["sweep_8192_bits_1_to_6"]:
+        assert abs(e["speedup_vs_naive_fp32"] - c["naive_fp32_8192"]["ms"] / e["ms"]) < 1e-9 and e["speedup_vs_naive_fp32"] > 1.0
