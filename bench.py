@@ -510,6 +510,33 @@ def cpu_baseline_leg():
             "equiv_int_gops": 2.0 * rows * N_SQ * N_SQ / dt / 1e9}
 
 
+def cpu_popcount_leg(sweep):
+    """The method's own CPU form beside the efficiency sweep (Section 5.4): Eq. 8 on packed planes as the oracle
+    writes it (plain C, the compiler's popcount builtin, OpenMP over rows; nothing vectorised by hand), timed on a
+    bounded sample of the 8192^3 product for 1..6 bits."""
+    import oracle
+    n8, rows = 8192, 32
+    kw = oracle.row_words(n8)
+    rng = np.random.default_rng(8192)
+    out = []
+    for b in range(1, 7):
+        pa = rng.integers(0, 2 ** 32, size=(rows, b, kw), dtype=np.uint64).astype(np.uint32)
+        pw = rng.integers(0, 2 ** 32, size=(n8, b, kw), dtype=np.uint64).astype(np.uint32)
+        oracle.fc_bitplanes(pa[:2], pw, n8)
+        t0 = time.perf_counter()
+        oracle.fc_bitplanes(pa, pw, n8)
+        dt = time.perf_counter() - t0
+        e = {"bits": b, "sample_ms": dt * 1e3, "binary_tops": binary_ops(rows, n8, n8, b, b) / dt / 1e12,
+             "full_size_ms": dt * 1e3 * n8 / rows}
+        gpu = next((s for s in sweep if s.get("bits") == b), None) if sweep else None
+        if gpu:
+            e["gpu_speedup"] = e["full_size_ms"] / gpu["ms"]
+        out.append(e)
+    return {"what": "oracle.fc_bitplanes (Eq. 8 with xor + popcount on packed planes, plain C, OpenMP over rows)",
+            "cores": oracle.num_threads(), "sample": f"{rows} of {n8} rows against all {n8} columns, K = {n8}, one call per width",
+            "bits_1_to_6": out}
+
+
 def run_gpu(args):
     import torch
     from paper_2106_09886_b200 import build as lib_build
@@ -682,6 +709,8 @@ def run_gpu(args):
             line["configs"]["clocks"] = sampler2.stop(t_c0, time.time())
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline_leg()
+            sweep = line.get("configs", {}).get("sweep_8192_bits_1_to_6") if isinstance(line.get("configs"), dict) else None
+            line["cpu_popcount_8192"] = cpu_popcount_leg(sweep)
         print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()

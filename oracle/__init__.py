@@ -59,6 +59,7 @@ def _load():
         lib.oracle_pack_planes.argtypes = [p, c.c_size_t, c.c_size_t, c.c_int, p]
         lib.oracle_fc.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, p]
         lib.oracle_fc_sampled.argtypes = [p, p, c.c_size_t, c.c_size_t, p, p, p]
+        lib.oracle_fc_bitplanes.argtypes = [p, p, c.c_size_t, c.c_size_t, c.c_size_t, c.c_int, c.c_int, p]
         lib.oracle_conv_out_dim.argtypes = [c.c_int] * 4
         lib.oracle_conv_backward_data.argtypes = [p, p] + [c.c_int] * 11 + [c.c_float, p]
         lib.oracle_conv_backward_weights.argtypes = [p, p] + [c.c_int] * 11 + [c.c_float, p]
@@ -123,6 +124,18 @@ def fc(qa: np.ndarray, qw: np.ndarray) -> np.ndarray:
     assert Kg == Kg2
     acc = np.empty((Mg, Ng), dtype=np.int32)
     _check(_load().oracle_fc(_ptr(qa), _ptr(qw), Mg, Ng, Kg, _ptr(acc)), "fc")
+    return acc
+
+
+def fc_bitplanes(a_planes: np.ndarray, w_planes: np.ndarray, Kg: int) -> np.ndarray:
+    """Eq. 8 on packed planes: a_planes [Mg, ab, row_words(Kg)], w_planes [Ng, wb, row_words(Kg)] -> int32 [Mg, Ng]."""
+    a_planes = np.ascontiguousarray(a_planes, dtype=np.uint32)
+    w_planes = np.ascontiguousarray(w_planes, dtype=np.uint32)
+    Mg, ab, kw = a_planes.shape
+    Ng, wb, kw2 = w_planes.shape
+    assert kw == kw2 == row_words(Kg)
+    acc = np.empty((Mg, Ng), dtype=np.int32)
+    _check(_load().oracle_fc_bitplanes(_ptr(a_planes), _ptr(w_planes), Mg, Ng, Kg, ab, wb, _ptr(acc)), "fc_bitplanes")
     return acc
 
 

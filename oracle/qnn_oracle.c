@@ -20,7 +20,9 @@
  *
  * It also writes the canonical bit-plane storage (Eq. 3 / Eq. 7: plane m holds
  * c_m of every element, one bit per element, +1 stored as 1) so that packed
- * planes can be compared word for word.
+ * planes can be compared word for word, and states Eq. 8 itself on those
+ * planes (oracle_fc_bitplanes: one xor and one popcount per word and plane
+ * pair), which must agree exactly with the plain product of step 2.
  *
  * Floating point: the quantizer decides an integer from binary32 data, so the
  * decision is fixed to one binary32 evaluation order: v = fma(x, 1/(2s), 2^(b-1))
@@ -123,6 +125,35 @@ int oracle_fc(const int16_t *qa, const int16_t *qw, size_t Mg, size_t Ng, size_t
             int64_t s = 0;
             for (size_t k = 0; k < Kg; ++k)
                 s += (int64_t)qa[(size_t)m * Kg + k] * (int64_t)qw[n * Kg + k];
+            if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
+            acc[(size_t)m * Ng + n] = (int32_t)s;
+        }
+    }
+    return bad ? ORACLE_E_RANGE : ORACLE_OK;
+}
+
+/* Eq. 8 written out on the packed planes (the decomposition itself, not its result's plain definition):
+ * acc[m][n] = sum_i sum_j 2^(i+j) * (Kg - 2 * popcount(a_i[m] xor w_j[n])), planes as oracle_pack_planes lays them out
+ * ([rows][bits][words], padding bits zero in both operands, so they never differ).  One xor and one popcount per
+ * 32-bit word and plane pair, nothing blocked or combined.  Serves as a second, independent statement of oracle_fc
+ * (the two must agree exactly) and as the CPU form of the method that the efficiency experiment (Section 5.4) times. */
+int oracle_fc_bitplanes(const uint32_t *a_planes, const uint32_t *w_planes, size_t Mg, size_t Ng, size_t Kg, int ab, int wb,
+                        int32_t *acc) {
+    if (!a_planes || !w_planes || !acc || ab < 1 || ab > 8 || wb < 1 || wb > 8) return ORACLE_E_ARG;
+    const size_t kw = oracle_row_words(Kg);
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (ptrdiff_t m = 0; m < (ptrdiff_t)Mg; ++m) {
+        for (size_t n = 0; n < Ng; ++n) {
+            int64_t s = 0;
+            for (int i = 0; i < ab; ++i)
+                for (int j = 0; j < wb; ++j) {
+                    const uint32_t *a = a_planes + ((size_t)m * ab + i) * kw;
+                    const uint32_t *w = w_planes + (n * wb + j) * kw;
+                    int64_t differ = 0;
+                    for (size_t x = 0; x < kw; ++x) differ += __builtin_popcount(a[x] ^ w[x]);
+                    s += ((int64_t)Kg - 2 * differ) * ((int64_t)1 << (i + j));
+                }
             if (s > INT32_MAX || s < INT32_MIN) bad |= 1;
             acc[(size_t)m * Ng + n] = (int32_t)s;
         }

@@ -40,3 +40,18 @@ def test_reference_arm_prints_one_line_from_rank0_only():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["cpu_baseline"]["kind"] == "oracle" and d["value"] > 0
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["unit"] == "binary TOPS" and d["n_gpus"] == 2
+
+
+def test_cpu_popcount_comparator_leg_reports_all_six_widths():
+    """The CPU form of the method timed beside the efficiency sweep: six widths, times that grow with the number of
+    plane pairs, and the speed-up against a given GPU sweep computed from the full-size figures."""
+    sys.path.insert(0, str(ROOT))
+    import bench
+    sweep = [{"bits": b, "ms": 2.0 * b * b} for b in range(1, 7)]
+    r = bench.cpu_popcount_leg(sweep)
+    rows = r["bits_1_to_6"]
+    assert [e["bits"] for e in rows] == [1, 2, 3, 4, 5, 6] and r["cores"] >= 1
+    assert rows[5]["sample_ms"] > rows[0]["sample_ms"] > 0
+    for e in rows:
+        assert abs(e["full_size_ms"] - e["sample_ms"] * 256) < 1e-6 * e["full_size_ms"]
+        assert abs(e["gpu_speedup"] - e["full_size_ms"] / (2.0 * e["bits"] ** 2)) < 1e-9 * e["gpu_speedup"]

@@ -24,7 +24,9 @@ GEOMS = [(2, 6, 5, 3, 4, 3, 3, 1, 1), (1, 9, 9, 40, 6, 3, 3, 2, 1), (3, 8, 8, 64
          # w), many images of 7 x 7 (tiles that span images), more than 256 channels (several channel tiles)
          (2, 11, 10, 8, 12, 5, 4, 3, 2), (1, 3, 150, 16, 8, 3, 3, 1, 1), (37, 7, 7, 24, 40, 3, 3, 1, 1), (2, 6, 6, 300, 20, 3, 3, 2, 1),
          # a 7 x 7 kernel at stride 2 (a network's stem): the weight gradient's strided copies of the codes, two row parities
-         (2, 16, 16, 8, 12, 7, 7, 2, 3)]
+         (2, 16, 16, 8, 12, 7, 7, 2, 3),
+         # output rows of a multiple of four columns (no row padding: the gradient goes through the plain transpose)
+         (3, 8, 8, 20, 12, 3, 3, 1, 1)]
 
 
 def _codes(rng, shape, bits):

@@ -43,6 +43,9 @@ MUTATIONS = {
     "conv_backward_data_taps_transposed": ("plane_of(qw[(((size_t)co * R + r) * S + s) * C + c], wb, j);", "plane_of(qw[(((size_t)co * S + s) * R + r) * C + c], wb, j);"),
     "conv_backward_weights_drops_alpha": ("part += ((double)alpha * (double)g[(((size_t)n * Ho + ho) * Wo + wo) * Cout + co]) *", "part += ((double)g[(((size_t)n * Ho + ho) * Wo + wo) * Cout + co]) *"),
     "conv_backward_data_ignores_stride": ("const int hi = ho * stride - pad + r, wi = wo * stride - pad + s;\n                            if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;\n                            double *dst", "const int hi = ho - pad + r, wi = wo - pad + s;\n                            if (hi < 0 || hi >= H || wi < 0 || wi >= W) continue;\n                            double *dst"),
+    "bitplanes_plane_weight": ("s += ((int64_t)Kg - 2 * differ) * ((int64_t)1 << (i + j));", "s += ((int64_t)Kg - 2 * differ) * ((int64_t)1 << (i * j));"),
+    "bitplanes_counts_agreements": ("s += ((int64_t)Kg - 2 * differ) *", "s += (2 * differ - (int64_t)Kg) *"),
+    "bitplanes_weight_plane_index": ("const uint32_t *w = w_planes + (n * wb + j) * kw;", "const uint32_t *w = w_planes + (n * wb + (wb - 1 - j)) * kw;"),
     "scale_in_double": ("out[i] = (float)acc[i] * alpha;", "out[i] = (float)((double)acc[i] * (double)alpha * (1.0 + 1e-6));"),
 }
 

@@ -203,6 +203,23 @@ def test_eq8_branch_identity(ab, wb, Kg):
     assert np.array_equal(acc, alt)
 
 
+@pytest.mark.parametrize("ab,wb,Kg", [(1, 1, 40), (2, 2, 65), (3, 2, 33), (4, 4, 130), (2, 4, 7), (8, 8, 50), (5, 1, 96), (2, 2, 1)])
+def test_fc_bitplanes_is_eq8_and_agrees_with_the_plain_definition(ab, wb, Kg):
+    """The popcount form of the oracle against three things that are not itself: the literal Python evaluation of
+    Eq. 8, a numpy float64 product of the codes, and the closed form for equal / opposite extreme operands."""
+    rng = np.random.default_rng(ab * 1000 + wb * 37 + Kg)
+    A, B = 2 ** ab - 1, 2 ** wb - 1
+    qa = (2 * rng.integers(0, A + 1, size=(7, Kg)) - A).astype(np.int16)
+    qw = (2 * rng.integers(0, B + 1, size=(5, Kg)) - B).astype(np.int16)
+    pa, pw = oracle.pack_planes(qa, ab), oracle.pack_planes(qw, wb)
+    got = oracle.fc_bitplanes(pa, pw, Kg)
+    assert np.array_equal(got, branch_sum_bruteforce(pa, pw, Kg, ab, wb))
+    assert np.array_equal(got.astype(np.float64), qa.astype(np.float64) @ qw.astype(np.float64).T)
+    hi_a, hi_w = np.full((2, Kg), A, dtype=np.int16), np.full((3, Kg), B, dtype=np.int16)
+    assert np.all(oracle.fc_bitplanes(oracle.pack_planes(hi_a, ab), oracle.pack_planes(hi_w, wb), Kg) == Kg * A * B)
+    assert np.all(oracle.fc_bitplanes(oracle.pack_planes(hi_a, ab), oracle.pack_planes(-hi_w, wb), Kg) == -Kg * A * B)
+
+
 def test_fc_matches_numpy_matmul_ragged():
     rng = np.random.default_rng(5)
     qa = (2 * rng.integers(0, 16, size=(37, 301)) - 15).astype(np.int16)
